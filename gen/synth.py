@@ -10,6 +10,8 @@ weights.
 """
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
 from dataclasses import dataclass, replace
 from typing import Dict, Optional, Tuple
 
@@ -19,7 +21,7 @@ import numpy as np
 _S_LM_HEAD, _S_W1, _S_B1, _S_W2, _S_HT, _S_HD, _S_CSI = 1, 2, 3, 4, 5, 6, 7
 _S_KLEN, _S_MATCH, _S_RANDTOK, _S_Q, _S_U = 8, 9, 10, 11, 12
 
-_CHUNK_ELEMS = 1 << 24  # fixed, so chunked generation is reproducible
+_CHUNK_ELEMS = 1 << 22  # fixed: chunk c of an array is its own Philox stream, so threads can fill it
 
 
 @dataclass(frozen=True)
@@ -40,6 +42,7 @@ class VerifyConfig:
     stochastic: bool = False
     K_lo: int = 0      # ragged windows: K_b ~ U{K_lo..K_hi}
     K_hi: int = 0
+    weight_seed: int = -1  # seed of the model weights; -1: same as seed
 
     @property
     def d_in(self) -> int:
@@ -49,7 +52,8 @@ class VerifyConfig:
         return replace(self, **kw)
 
 
-_8B = dict(H=4096, H_d=2048, d_c=2, d_J=1024, V=128256)
+# one 8B-shaped model (LM head + decision head) serves every 8B workload
+_8B = dict(H=4096, H_d=2048, d_c=2, d_J=1024, V=128256, weight_seed=1000)
 
 CONFIGS: Dict[str, VerifyConfig] = {
     "tiny": VerifyConfig("tiny", B=8, K=4, H=256, H_d=128, d_c=2, d_J=128, V=4096,
@@ -85,14 +89,26 @@ def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
     return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32)
 
 
-def _normal_bf16(g: np.random.Generator, shape: Tuple[int, ...], std: float) -> np.ndarray:
+def _normal_bf16(seed: int, stream: int, shape: Tuple[int, ...], std: float) -> np.ndarray:
+    """bf16 bits of N(0, std); chunk c is drawn from stream (stream, c), independent of thread count."""
     n = int(np.prod(shape))
     out = np.empty(n, dtype=np.uint16)
-    for lo in range(0, n, _CHUNK_ELEMS):
+
+    def fill(c: int) -> None:
+        lo = c * _CHUNK_ELEMS
         hi = min(n, lo + _CHUNK_ELEMS)
+        g = np.random.Generator(np.random.Philox(key=[int(seed), int(stream) + (c << 32)]))
         x = g.standard_normal(hi - lo, dtype=np.float32)
         x *= np.float32(std)
         out[lo:hi] = f32_to_bf16_bits(x)
+
+    chunks = range((n + _CHUNK_ELEMS - 1) // _CHUNK_ELEMS)
+    if len(chunks) > 1:
+        with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as ex:
+            list(ex.map(fill, chunks))
+    else:
+        for c in chunks:
+            fill(c)
     return out.reshape(shape)
 
 
@@ -119,16 +135,17 @@ def make_weights(cfg: VerifyConfig) -> Dict[str, np.ndarray]:
     ordered [h^D | h^T | c] (the order of Eq. 23), each column block drawn from its own
     sub-stream so a different concatenation order is a pure column permutation.
     """
-    lm_head = _normal_bf16(_rng(cfg.seed, _S_LM_HEAD), (cfg.V, cfg.H), 0.02)
+    ws = cfg.weight_seed if cfg.weight_seed >= 0 else cfg.seed
+    lm_head = _normal_bf16(ws, _S_LM_HEAD, (cfg.V, cfg.H), 0.02)
     # hidden-state columns ~ N(0, 1/sqrt(d_in)); CSI columns ~ N(0, 1/128) because the CSI
     # features are consumed unnormalised (tens of dB / Mbps) and would otherwise swamp z
     std1 = 1.0 / np.sqrt(cfg.d_in)
     blocks = []
     for j, (width, std) in enumerate(((cfg.H_d, std1), (cfg.H, std1), (cfg.d_c, 1.0 / 128.0))):
-        blocks.append(_normal_bf16(_rng(cfg.seed, _S_W1 + 100 * (j + 1)), (cfg.d_J, width), std))
+        blocks.append(_normal_bf16(ws, _S_W1 + 100 * (j + 1), (cfg.d_J, width), std))
     W1 = np.ascontiguousarray(np.concatenate(blocks, axis=1))
-    b1 = (_rng(cfg.seed, _S_B1).standard_normal(cfg.d_J, dtype=np.float32) * np.float32(0.1))
-    w2 = (_rng(cfg.seed, _S_W2).standard_normal(cfg.d_J, dtype=np.float32)
+    b1 = (_rng(ws, _S_B1).standard_normal(cfg.d_J, dtype=np.float32) * np.float32(0.1))
+    w2 = (_rng(ws, _S_W2).standard_normal(cfg.d_J, dtype=np.float32)
           * np.float32(1.0 / np.sqrt(cfg.d_J)))
     b2 = np.float32(0.0625)
     return dict(lm_head=lm_head, W1=W1, b1=b1, w2=w2, b2=b2)

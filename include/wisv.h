@@ -1,0 +1,211 @@
+/*
+ * wisv.h - C ABI of the WISV edge-side verifier for one NVIDIA B200 (sm_100a).
+ *
+ * One call verifies a batch of speculative-decoding windows the way the edge
+ * server does in one round of Algorithm 1 of "WISV: Wireless-Informed Semantic
+ * Verification for Distributed Speculative Decoding in Device-Edge LLM
+ * Inference":
+ *
+ *   1. logits of the target model at the K+1 window positions (the LM-head part
+ *      of Verify; Section IV-B: the logits serve mismatch localisation and
+ *      correction) - never written out, only reduced;
+ *   2. per position: argmax, log-sum-exp and the target probability of the draft
+ *      token (Section II-A, greedy verification and Eq. 1);
+ *   3. Localize: the candidate set S of mismatching positions (Section V-C);
+ *   4. the CSI-aware decision head p = sigmoid(w2 . act(W1 [h^D; h^T; c] + b1) + b2)
+ *      (Eqs. 23-25) on full-hidden (FH) or selective-hidden (SH) uploads
+ *      (Section III-B);
+ *   5. the earliest position of S whose rejection probability reaches tau
+ *      (Eq. 27), the accepted length and the correction / bonus token (Algorithm 1,
+ *      full-accept and commit-and-correct branches; Section III-A step 4).
+ *
+ * Indexing.  Request b has a draft window of K_b tokens (K_b <= 64).  Tokens are
+ * addressed by t = k_off[b] + i (i = 0..K_b-1, T = sum K_b) and window rows by
+ * r = k_off[b] + b + i (i = 0..K_b, R = T + B).  Row i < K_b holds the target's
+ * final hidden state whose logits predict draft token i; row K_b yields the
+ * bonus token of a full accept.  accept_len counts accepted draft tokens
+ * (the paper's j-hat minus one, or K_b), correction_token = argmax of row
+ * accept_len in both branches.
+ *
+ * Numerics.  Hidden states are rounded to bf16 (nearest even) before every
+ * matrix product; weights are bf16; accumulation and everything after the
+ * products is fp32.  CSI features and the CSI columns of W1 enter in fp32.
+ *
+ * Conventions.  Every function returns 0 (WISV_OK) or a negative error code; no
+ * function throws, aborts or prints.  Pointers marked "dev" are CUDA device
+ * pointers owned by the caller; the library never frees them.  The weights are
+ * borrowed for the lifetime of the context (the LM head is not copied).  The
+ * context owns its workspace, a repacked copy of W1 and its TMA descriptors.
+ * wisv_verify only enqueues work on the given stream: results are valid once
+ * the caller has synchronised that stream.  A context serves one call at a time
+ * (calls on one context must be stream-ordered).  There is no CPU fallback: on a
+ * device that is not compute capability 10.x wisv_create fails with WISV_EARCH.
+ */
+#ifndef WISV_H_
+#define WISV_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define WISV_VERSION 100
+
+/* error codes */
+#define WISV_OK         0
+#define WISV_EINVAL    -1   /* NULL pointer, bad enum, bad mode bits */
+#define WISV_ESHAPE    -2   /* dimension out of the supported range */
+#define WISV_EALIGN    -3   /* pointer or pitch not aligned as documented */
+#define WISV_ECAPACITY -4   /* batch exceeds the capacities given at create */
+#define WISV_ECUDA     -5   /* a CUDA runtime / driver call failed */
+#define WISV_EARCH     -6   /* current device is not sm_100 */
+#define WISV_ENOMEM    -7   /* allocation failed */
+#define WISV_EDEVICE   -8   /* a kernel reported a pipeline time-out (see wisv_device_error) */
+
+/* activation of the decision head */
+#define WISV_ACT_RELU 0     /* Eq. 25 as printed */
+#define WISV_ACT_GELU 1     /* exact erf form */
+
+/* mode bits of wisv_batch.mode */
+#define WISV_MODE_FH           0u  /* draft_hidden is dense [T, H_d] */
+#define WISV_MODE_SH           1u  /* draft_hidden is packed [M_sel, H_d] with sel_off / sel_pos */
+#define WISV_ACCEPT_GREEDY     0u  /* S = { i : draft token != argmax } */
+#define WISV_ACCEPT_STOCHASTIC 2u  /* S = { i : !(u_i < min(1, p_T(y_i) / q_i)) }  (Eq. 1) */
+
+/* per-request status bits written by the device */
+#define WISV_ST_MISSING_HIDDEN 1   /* a position of S had no uploaded hidden state: rejected greedily */
+#define WISV_ST_BAD_TOKEN      2   /* a draft token id was outside [0, V): clamped */
+#define WISV_ST_NONFINITE      4   /* a non-finite log-sum-exp or head logit was seen */
+#define WISV_ST_BAD_SELECT     8   /* a sel_pos entry was outside [0, K_b): ignored */
+
+#define WISV_MAX_K   64
+#define WISV_MAX_DC  16
+
+typedef struct wisv_ctx wisv_ctx;
+
+typedef struct {
+    int32_t H;              /* target hidden size; H % 8 == 0 */
+    int32_t V;              /* vocabulary size */
+    int32_t H_d;            /* drafter hidden size; H_d % 8 == 0 */
+    int32_t d_c;            /* CSI features, 0..WISV_MAX_DC */
+    int32_t d_J;            /* decision-head hidden width */
+    int32_t act;            /* WISV_ACT_* */
+    int32_t head_row_shift; /* 0: h^T_i is window row i (the row scored against draft token i); 1: row i+1 */
+    float   tau;            /* default threshold: reject iff p >= tau; 0 = greedy, > 1 = accept all */
+    int32_t max_requests;   /* capacity: B */
+    int32_t max_rows;       /* capacity: R = T + B */
+    int32_t max_sel;        /* capacity: M_sel (SH); 0 = max_rows */
+} wisv_config;
+
+typedef struct {
+    const void*  lm_head;   /* dev bf16 [V, H] row-major, 16-byte aligned */
+    const void*  W1;        /* dev bf16 [d_J, H_d + H + d_c] row-major, columns [h^D | h^T | c] (Eq. 23) */
+    const float* b1;        /* dev fp32 [d_J] */
+    const float* w2;        /* dev fp32 [d_J] */
+    float        b2;
+} wisv_weights;
+
+typedef struct {
+    int32_t B;                     /* requests */
+    int32_t K;                     /* uniform window length, or 0 with k_off != NULL */
+    const int32_t* k_off;          /* dev int32 [B+1] prefix sums of K_b (ragged), or NULL */
+    int32_t T_total;               /* sum of K_b (host-known; = B*K when uniform) */
+    const float*   target_hidden;  /* dev fp32 [R, H] */
+    const int32_t* draft_tokens;   /* dev int32 [T] */
+    const float*   draft_hidden;   /* dev fp32 [T, H_d] (FH) or [M_sel, H_d] (SH) */
+    const int32_t* sel_off;        /* SH: dev int32 [B+1], CSR offsets into sel_pos */
+    const int32_t* sel_pos;        /* SH: dev int32 [M_sel], window-relative positions */
+    int32_t M_sel;                 /* SH: number of uploaded hidden states */
+    const float*   csi;            /* dev fp32 [B, d_c] */
+    const float*   draft_q;        /* stochastic: dev fp32 [T], drafter probability of its token */
+    const float*   uniforms;       /* stochastic: dev fp32 [T], u in [0, 1) */
+    uint32_t mode;                 /* WISV_MODE_* | WISV_ACCEPT_* */
+    float    tau;                  /* NaN: use the context default */
+} wisv_batch;
+
+typedef struct {
+    int32_t*  accept_len;        /* dev [B], required */
+    int32_t*  correction_token;  /* dev [B], required */
+    int32_t*  argmax;            /* dev [R], optional */
+    float*    lse;               /* dev [R], optional */
+    float*    p_draft;           /* dev [T], optional: target probability of each draft token */
+    float*    head_prob;         /* dev [T] (FH) or [M_sel] (SH), optional */
+    uint64_t* mismatch_mask;     /* dev [B], optional: bit i set iff position i is in S */
+    int32_t*  n_mismatch;        /* dev [B], optional: |S| (m_r of Section IV-A) */
+    int32_t*  status;            /* dev [B], optional: WISV_ST_* bits */
+} wisv_result;
+
+/*
+ * Create a verifier context on the current CUDA device (Algorithm 1's Require
+ * line: decision head g_theta, threshold tau; the LM head belongs to the target
+ * model T).  Validates dimensions and alignment, allocates the workspace for the
+ * stated capacities, splits W1 into a bf16 [d_J, H_d+H] block and an fp32
+ * [d_J, d_c] CSI block (device-to-device, on the default stream, synchronised
+ * before returning) and encodes the TMA descriptors.  *out is NULL on failure.
+ */
+int wisv_create(const wisv_config* cfg, const wisv_weights* weights, wisv_ctx** out);
+
+/*
+ * Enqueue one verification round (Algorithm 1, from Verify's logits to the
+ * feedback pair) for a batch on `cuda_stream` (a cudaStream_t; NULL = default
+ * stream).  All pointers in `batch` and `result` are device pointers.  Host-side
+ * argument errors are returned before anything is launched; conditions only the
+ * device can see are reported through result->status.  Does not synchronise.
+ */
+int wisv_verify(wisv_ctx* ctx, const wisv_batch* batch, const wisv_result* result, void* cuda_stream);
+
+/*
+ * Same round with HOST buffers: every pointer in `batch` and `result` is host
+ * memory (pinned memory makes the copies asynchronous).  Inputs are copied to
+ * staging buffers owned by the context (allocated on first use), the round is
+ * run, the requested results are copied back and the stream is synchronised
+ * before returning.  Returns WISV_EDEVICE if a kernel reported a time-out.
+ */
+int wisv_verify_host(wisv_ctx* ctx, const wisv_batch* batch, const wisv_result* result, void* cuda_stream);
+
+/* Free the context and everything it owns.  The caller must have synchronised. */
+int wisv_destroy(wisv_ctx* ctx);
+
+/*
+ * Read (and clear) the device error word: non-zero if a bounded wait inside a
+ * kernel gave up.  Synchronises the given stream first.
+ */
+int wisv_device_error(wisv_ctx* ctx, void* cuda_stream, int32_t* flags);
+
+/*
+ * Per-stage device timing.  After wisv_profile_enable(ctx, n) the library
+ * records CUDA events around each kernel of the next calls (ring of n calls);
+ * wisv_profile_read synchronises and returns, for stage s (0 = pack/cast,
+ * 1 = LM head, 2 = decision head, 3 = merge + scan), the elapsed milliseconds
+ * of up to `cap` recorded calls, oldest first.  n = 0 disables profiling.
+ */
+int wisv_profile_enable(wisv_ctx* ctx, int32_t n_calls);
+int wisv_profile_read(wisv_ctx* ctx, int32_t stage, float* ms, int32_t cap, int32_t* n_out);
+
+/* Number of kernels this context has launched so far. */
+int64_t wisv_launch_count(const wisv_ctx* ctx);
+
+/*
+ * Launch geometry the next wisv_verify would use for a batch with R window rows
+ * and P head positions: vocabulary rows per LM-head tile, LM-head tiles, CTAs.
+ * Any output pointer may be NULL.
+ */
+int wisv_plan(const wisv_ctx* ctx, int32_t R, int32_t P, int32_t* lm_tile_n, int32_t* lm_tiles,
+              int32_t* lm_ctas, int32_t* head_tile_n, int32_t* head_tiles, int32_t* head_ctas);
+
+/*
+ * Bring-up / test hook: the raw fp32 logits L = bf16(target_hidden) . lm_head^T
+ * of R rows (Algorithm 1, Verify), written to logits_out (dev fp32 [R, V]) by the
+ * same TMA + tcgen05 main loop with a store epilogue.  target_hidden: dev fp32
+ * [R, H].  Not used by wisv_verify, which never materialises logits.
+ */
+int wisv_debug_logits(wisv_ctx* ctx, const float* target_hidden, int32_t R, float* logits_out, void* cuda_stream);
+
+const char* wisv_strerror(int code);
+int wisv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WISV_H_ */

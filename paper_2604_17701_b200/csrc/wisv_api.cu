@@ -1,0 +1,655 @@
+// Host side of the WISV verifier library: context, argument validation, launch
+// plan and the C ABI declared in include/wisv.h.  One verification round is four
+// stream-ordered launches: pack -> LM-head GEMM+reduce -> decision-head
+// GEMM+reduce -> merge/localize/scan.  Control never returns to the host between
+// them and nothing is synchronised.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "../../include/wisv.h"
+#include "wisv_aux.cuh"
+#include "wisv_gemm.cuh"
+
+using namespace wisv;
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+constexpr int kNumTileVariants = kMaxTileN / 16;   // tile_n = 16, 32, ..., 256
+constexpr int kStages = 4;                         // profiled stages per call
+
+struct Plan {
+    int tile_n, m_tiles, n_tiles, ctas, stages;
+    size_t smem;
+};
+
+struct HostStaging {
+    float* target_hidden = nullptr; int32_t* draft_tokens = nullptr; float* draft_hidden = nullptr;
+    int32_t* k_off = nullptr; int32_t* sel_off = nullptr; int32_t* sel_pos = nullptr; float* csi = nullptr;
+    float* draft_q = nullptr; float* uniforms = nullptr;
+    int32_t* accept_len = nullptr; int32_t* correction = nullptr; int32_t* argmax = nullptr; float* lse = nullptr;
+    float* p_draft = nullptr; float* head_prob = nullptr; unsigned long long* mask = nullptr;
+    int32_t* n_mismatch = nullptr; int32_t* status = nullptr;
+    bool ready = false;
+};
+
+}  // namespace
+
+struct wisv_ctx {
+    wisv_config cfg;
+    wisv_weights w;
+    int device = 0;
+    int sm_count = 0;
+    int max_smem = 0;
+    int max_pos = 0;          // capacity of evaluated head positions
+    int rows_alloc = 0;       // max_rows rounded up to the tile height
+    int pos_alloc = 0;
+    // workspace
+    __nv_bfloat16* X = nullptr;       // [rows_alloc, H]
+    __nv_bfloat16* Z = nullptr;       // [pos_alloc, H_d + H]
+    __nv_bfloat16* W1p = nullptr;     // [d_J, H_d + H]
+    float* W1c = nullptr;             // [d_J, d_c]
+    float4* lm_part = nullptr;
+    size_t lm_part_elems = 0;
+    float* head_part = nullptr;
+    size_t head_part_elems = 0;
+    int32_t* row_tok = nullptr; int32_t* row_flag = nullptr; float* tok_logit = nullptr;
+    int32_t* pos_req = nullptr; int32_t* pos_i = nullptr;
+    int32_t* err = nullptr;
+    // TMA descriptors
+    CUtensorMap tmX, tmZ;
+    CUtensorMap tmW[kNumTileVariants];
+    CUtensorMap tmW1[kNumTileVariants];
+    // profiling
+    int prof_n = 0;
+    long long prof_calls = 0;
+    cudaEvent_t* prof_ev = nullptr;   // [prof_n][kStages + 1]
+    long long launches = 0;
+    HostStaging hs;
+};
+
+namespace {
+
+#define WISV_CUDA(call)                                   \
+    do {                                                  \
+        cudaError_t e_ = (call);                          \
+        if (e_ != cudaSuccess) { (void)cudaGetLastError(); return WISV_ECUDA; } \
+    } while (0)
+
+int encode_2d(EncodeTiledFn fn, CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer,
+              uint32_t box_inner, uint32_t box_outer)
+{
+    cuuint64_t dims[2] = {inner, outer};
+    cuuint64_t strides[1] = {inner * 2};            // bytes between rows (bf16)
+    cuuint32_t box[2] = {box_inner, box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? WISV_OK : WISV_ECUDA;
+}
+
+int round_up(int x, int m) { return (x + m - 1) / m * m; }
+
+size_t gemm_smem_bytes(int tile_n, int stages, int d_c)
+{
+    return 1024 + (size_t)stages * gemm_stage_bytes(tile_n) + gemm_tail_bytes(tile_n, d_c);
+}
+
+int stages_for(const wisv_ctx* c, int tile_n, int d_c, int k_blocks)
+{
+    const size_t fixed = 1024 + gemm_tail_bytes(tile_n, d_c);
+    int s = (int)(((size_t)c->max_smem - fixed) / gemm_stage_bytes(tile_n));
+    if (s > kMaxStages) s = kMaxStages;
+    (void)k_blocks;
+    return s;
+}
+
+double wave_eff(long long tiles, int sms)
+{
+    const long long waves = (tiles + sms - 1) / sms;
+    return (double)tiles / (double)(waves * sms);
+}
+
+// LM head: with a single row tile the kernel streams the weights once and is
+// HBM-bound, so the tile height over the vocabulary is chosen to fill the last
+// wave of CTAs; with many row tiles it is tensor-bound and takes the largest tile.
+Plan plan_lm(const wisv_ctx* c, int R)
+{
+    Plan p{};
+    const int V = c->cfg.V;
+    p.m_tiles = (R + kTileM - 1) / kTileM;
+    int best = 0;
+    if (p.m_tiles == 1) {
+        double best_eff = -1.0;
+        for (int tn = 64; tn <= kMaxTileN; tn += 16) {
+            const long long tiles = (V + tn - 1) / tn;
+            const double e = wave_eff(tiles, c->sm_count);
+            if (e >= best_eff - 1e-9) { best_eff = e > best_eff ? e : best_eff; best = tn; }
+        }
+    } else {
+        best = V >= kMaxTileN ? kMaxTileN : round_up(V, 16);
+    }
+    if (best > round_up(V, 16)) best = round_up(V, 16);
+    p.tile_n = best;
+    p.n_tiles = (V + best - 1) / best;
+    const long long tiles = (long long)p.m_tiles * p.n_tiles;
+    p.ctas = (int)(tiles < c->sm_count ? tiles : c->sm_count);
+    p.stages = stages_for(c, best, 0, 0);
+    p.smem = gemm_smem_bytes(best, p.stages, 0);
+    return p;
+}
+
+Plan plan_head(const wisv_ctx* c, int P)
+{
+    Plan p{};
+    const int N = c->cfg.d_J;
+    p.m_tiles = (P + kTileM - 1) / kTileM;
+    int best = 16;
+    if (p.m_tiles >= 8) {
+        best = N >= kMaxTileN ? kMaxTileN : round_up(N, 16);
+    } else {
+        double best_eff = -1.0;
+        for (int tn = 16; tn <= kMaxTileN; tn *= 2) {
+            const long long tiles = (long long)p.m_tiles * ((N + tn - 1) / tn);
+            const double e = wave_eff(tiles, c->sm_count);
+            if (e >= best_eff - 1e-9) { best_eff = e > best_eff ? e : best_eff; best = tn; }
+        }
+    }
+    if (best > round_up(N, 16)) best = round_up(N, 16);
+    p.tile_n = best;
+    p.n_tiles = (N + best - 1) / best;
+    const long long tiles = (long long)p.m_tiles * p.n_tiles;
+    p.ctas = (int)(tiles < c->sm_count ? tiles : c->sm_count);
+    p.stages = stages_for(c, best, c->cfg.d_c, 0);
+    p.smem = gemm_smem_bytes(best, p.stages, c->cfg.d_c);
+    return p;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+void free_ctx(wisv_ctx* c)
+{
+    if (!c) return;
+    cudaFree(c->X); cudaFree(c->Z); cudaFree(c->W1p); cudaFree(c->W1c); cudaFree(c->lm_part);
+    cudaFree(c->head_part); cudaFree(c->row_tok); cudaFree(c->row_flag); cudaFree(c->tok_logit);
+    cudaFree(c->pos_req); cudaFree(c->pos_i); cudaFree(c->err);
+    if (c->prof_ev) {
+        for (int i = 0; i < c->prof_n * (kStages + 1); ++i) cudaEventDestroy(c->prof_ev[i]);
+        free(c->prof_ev);
+    }
+    HostStaging& h = c->hs;
+    cudaFree(h.target_hidden); cudaFree(h.draft_tokens); cudaFree(h.draft_hidden); cudaFree(h.k_off);
+    cudaFree(h.sel_off); cudaFree(h.sel_pos); cudaFree(h.csi); cudaFree(h.draft_q); cudaFree(h.uniforms);
+    cudaFree(h.accept_len); cudaFree(h.correction); cudaFree(h.argmax); cudaFree(h.lse); cudaFree(h.p_draft);
+    cudaFree(h.head_prob); cudaFree(h.mask); cudaFree(h.n_mismatch); cudaFree(h.status);
+    (void)cudaGetLastError();
+    delete c;
+}
+
+template <typename T>
+int dev_alloc(T** p, size_t n)
+{
+    void* q = nullptr;
+    if (cudaMalloc(&q, (n ? n : 1) * sizeof(T)) != cudaSuccess) { (void)cudaGetLastError(); return WISV_ENOMEM; }
+    *p = static_cast<T*>(q);
+    return WISV_OK;
+}
+
+int validate_batch(const wisv_ctx* c, const wisv_batch* b, const wisv_result* r, int* T_out, int* R_out, int* P_out)
+{
+    if (!c || !b || !r) return WISV_EINVAL;
+    if (b->B < 0 || b->K < 0) return WISV_ESHAPE;
+    if (b->mode & ~3u) return WISV_EINVAL;
+    const bool sh = (b->mode & WISV_MODE_SH) != 0;
+    const bool stoch = (b->mode & WISV_ACCEPT_STOCHASTIC) != 0;
+    if (b->K == 0 && !b->k_off && b->B > 0 && b->T_total != 0) return WISV_EINVAL;
+    if (b->K > WISV_MAX_K) return WISV_ESHAPE;
+    long long T = b->k_off ? (long long)b->T_total : (long long)b->B * b->K;
+    if (b->k_off && b->K != 0) return WISV_EINVAL;
+    if (!b->k_off && b->T_total != 0 && b->T_total != T) return WISV_ESHAPE;
+    if (T < 0 || T > (long long)WISV_MAX_K * b->B) return WISV_ESHAPE;
+    const long long R = T + b->B;
+    if (b->B > c->cfg.max_requests || R > c->cfg.max_rows) return WISV_ECAPACITY;
+    long long P = T;
+    if (sh) {
+        if (b->M_sel < 0) return WISV_ESHAPE;
+        if (b->M_sel > c->max_pos || b->M_sel > T) return b->M_sel > T ? WISV_ESHAPE : WISV_ECAPACITY;
+        P = b->M_sel;
+        if (b->B > 0 && !b->sel_off) return WISV_EINVAL;
+        if (P > 0 && !b->sel_pos) return WISV_EINVAL;
+    }
+    if (P > c->max_pos) return WISV_ECAPACITY;
+    if (b->B > 0) {
+        if (!b->target_hidden || !r->accept_len || !r->correction_token) return WISV_EINVAL;
+        if (T > 0 && !b->draft_tokens) return WISV_EINVAL;
+        if (P > 0 && (!b->draft_hidden || (c->cfg.d_c > 0 && !b->csi))) return WISV_EINVAL;
+        if (stoch && T > 0 && (!b->draft_q || !b->uniforms)) return WISV_EINVAL;
+        if (!aligned16(b->target_hidden) || (P > 0 && !aligned16(b->draft_hidden))) return WISV_EALIGN;
+    }
+    if (!(b->tau != b->tau) && b->tau < 0.0f) return WISV_EINVAL;
+    *T_out = (int)T; *R_out = (int)R; *P_out = (int)P;
+    return WISV_OK;
+}
+
+template <int EPI>
+int launch_gemm(wisv_ctx* c, const CUtensorMap& tA, const CUtensorMap& tB, const GemmParams& gp, const Plan& pl,
+                cudaStream_t st)
+{
+    gemm_rowreduce_kernel<EPI><<<pl.ctas, kGemmThreads, pl.smem, st>>>(tA, tB, gp);
+    WISV_CUDA(cudaGetLastError());
+    c->launches++;
+    return WISV_OK;
+}
+
+GemmParams base_params(const wisv_ctx* c, const Plan& pl, int rows, int n_total, int kdim)
+{
+    GemmParams gp;
+    memset(&gp, 0, sizeof gp);
+    gp.rows = rows; gp.n_total = n_total; gp.k_blocks = (kdim + kBlockK - 1) / kBlockK;
+    gp.tile_n = pl.tile_n; gp.m_tiles = pl.m_tiles; gp.n_tiles = pl.n_tiles; gp.stages = pl.stages;
+    gp.err = c->err;
+    return gp;
+}
+
+}  // namespace
+
+extern "C" {
+
+int wisv_version(void) { return WISV_VERSION; }
+
+const char* wisv_strerror(int code)
+{
+    switch (code) {
+        case WISV_OK: return "ok";
+        case WISV_EINVAL: return "invalid argument";
+        case WISV_ESHAPE: return "dimension out of range";
+        case WISV_EALIGN: return "pointer or pitch misaligned";
+        case WISV_ECAPACITY: return "batch exceeds the context capacity";
+        case WISV_ECUDA: return "CUDA call failed";
+        case WISV_EARCH: return "device is not sm_100";
+        case WISV_ENOMEM: return "out of memory";
+        case WISV_EDEVICE: return "a kernel reported a pipeline time-out";
+        default: return "unknown error";
+    }
+}
+
+int wisv_create(const wisv_config* cfg, const wisv_weights* w, wisv_ctx** out)
+{
+    if (out) *out = nullptr;
+    if (!cfg || !w || !out) return WISV_EINVAL;
+    if (!w->lm_head || !w->W1 || !w->b1 || !w->w2) return WISV_EINVAL;
+    if (cfg->act != WISV_ACT_RELU && cfg->act != WISV_ACT_GELU) return WISV_EINVAL;
+    if (cfg->head_row_shift != 0 && cfg->head_row_shift != 1) return WISV_EINVAL;
+    if (!(cfg->tau >= 0.0f)) return WISV_EINVAL;
+    if (cfg->H < 64 || cfg->H % 8 || cfg->H_d < 8 || cfg->H_d % 8 || cfg->V < 1 || cfg->d_J < 1) return WISV_ESHAPE;
+    if (cfg->d_c < 0 || cfg->d_c > WISV_MAX_DC) return WISV_ESHAPE;
+    if (cfg->max_requests < 1 || cfg->max_rows < cfg->max_requests || cfg->max_sel < 0) return WISV_ESHAPE;
+    if ((long long)cfg->max_rows > (long long)(WISV_MAX_K + 1) * cfg->max_requests) return WISV_ESHAPE;
+    if (!aligned16(w->lm_head)) return WISV_EALIGN;
+
+    int dev = 0;
+    WISV_CUDA(cudaGetDevice(&dev));
+    cudaDeviceProp prop;
+    WISV_CUDA(cudaGetDeviceProperties(&prop, dev));
+    if (prop.major != 10) return WISV_EARCH;
+
+    // every GEMM instantiation may use the full opt-in shared memory
+    WISV_CUDA(cudaFuncSetAttribute(gemm_rowreduce_kernel<EPI_LMHEAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)prop.sharedMemPerBlockOptin));
+    WISV_CUDA(cudaFuncSetAttribute(gemm_rowreduce_kernel<EPI_HEAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)prop.sharedMemPerBlockOptin));
+    WISV_CUDA(cudaFuncSetAttribute(gemm_rowreduce_kernel<EPI_RAW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)prop.sharedMemPerBlockOptin));
+
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    WISV_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+    if (!fn || qres != cudaDriverEntryPointSuccess) return WISV_ECUDA;
+    EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(fn);
+
+    wisv_ctx* c = new (std::nothrow) wisv_ctx();
+    if (!c) return WISV_ENOMEM;
+    c->cfg = *cfg;
+    c->w = *w;
+    c->device = dev;
+    c->sm_count = prop.multiProcessorCount;
+    c->max_smem = (int)prop.sharedMemPerBlockOptin;
+    const int max_T = cfg->max_rows - 1;
+    c->max_pos = cfg->max_sel > 0 ? (cfg->max_sel > max_T ? cfg->max_sel : max_T) : max_T;
+    if (c->max_pos < 1) c->max_pos = 1;
+    c->rows_alloc = round_up(cfg->max_rows, kTileM);
+    c->pos_alloc = round_up(c->max_pos, kTileM);
+    const int hd_h = cfg->H_d + cfg->H;
+
+    // partial buffers sized for the worst plan at any row count up to the capacity
+    size_t lm_elems = 0, head_elems = 0;
+    {
+        const int r1 = cfg->max_rows < kTileM ? cfg->max_rows : kTileM;
+        Plan a = plan_lm(c, r1);
+        lm_elems = (size_t)r1 * a.n_tiles;
+        // the single-tile plan may pick any tile height >= 64
+        const size_t worst1 = (size_t)r1 * ((cfg->V + 63) / 64);
+        if (worst1 > lm_elems) lm_elems = worst1;
+        if (cfg->max_rows > kTileM) {
+            Plan b = plan_lm(c, cfg->max_rows);
+            const size_t e = (size_t)cfg->max_rows * b.n_tiles;
+            if (e > lm_elems) lm_elems = e;
+        }
+        head_elems = (size_t)c->max_pos * ((cfg->d_J + 15) / 16);
+    }
+    c->lm_part_elems = lm_elems;
+    c->head_part_elems = head_elems;
+
+    int rc = WISV_OK;
+    do {
+        if ((rc = dev_alloc(&c->X, (size_t)c->rows_alloc * cfg->H))) break;
+        if ((rc = dev_alloc(&c->Z, (size_t)c->pos_alloc * hd_h))) break;
+        if ((rc = dev_alloc(&c->W1p, (size_t)cfg->d_J * hd_h))) break;
+        if ((rc = dev_alloc(&c->W1c, (size_t)cfg->d_J * (cfg->d_c > 0 ? cfg->d_c : 1)))) break;
+        if ((rc = dev_alloc(&c->lm_part, lm_elems))) break;
+        if ((rc = dev_alloc(&c->head_part, head_elems))) break;
+        if ((rc = dev_alloc(&c->row_tok, (size_t)c->rows_alloc))) break;
+        if ((rc = dev_alloc(&c->row_flag, (size_t)c->rows_alloc))) break;
+        if ((rc = dev_alloc(&c->tok_logit, (size_t)c->rows_alloc))) break;
+        if ((rc = dev_alloc(&c->pos_req, (size_t)c->pos_alloc))) break;
+        if ((rc = dev_alloc(&c->pos_i, (size_t)c->pos_alloc))) break;
+        if ((rc = dev_alloc(&c->err, 1))) break;
+        if (cudaMemset(c->X, 0, (size_t)c->rows_alloc * cfg->H * 2) != cudaSuccess ||
+            cudaMemset(c->Z, 0, (size_t)c->pos_alloc * hd_h * 2) != cudaSuccess ||
+            cudaMemset(c->err, 0, sizeof(int32_t)) != cudaSuccess) { rc = WISV_ECUDA; break; }
+
+        split_w1_kernel<<<cfg->d_J, 256>>>(static_cast<const __nv_bfloat16*>(w->W1), c->W1p, c->W1c, cfg->d_J, hd_h,
+                                           cfg->d_c);
+        if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) { rc = WISV_ECUDA; break; }
+        c->launches++;
+
+        if ((rc = encode_2d(encode, &c->tmX, c->X, (uint64_t)cfg->H, (uint64_t)c->rows_alloc, kBlockK, kTileM))) break;
+        if ((rc = encode_2d(encode, &c->tmZ, c->Z, (uint64_t)hd_h, (uint64_t)c->pos_alloc, kBlockK, kTileM))) break;
+        for (int i = 0; i < kNumTileVariants && rc == WISV_OK; ++i) {
+            const uint32_t tn = 16u * (i + 1);
+            rc = encode_2d(encode, &c->tmW[i], w->lm_head, (uint64_t)cfg->H, (uint64_t)cfg->V, kBlockK, tn);
+            if (rc == WISV_OK)
+                rc = encode_2d(encode, &c->tmW1[i], c->W1p, (uint64_t)hd_h, (uint64_t)cfg->d_J, kBlockK, tn);
+        }
+    } while (0);
+    if (rc != WISV_OK) { free_ctx(c); return rc; }
+    *out = c;
+    return WISV_OK;
+}
+
+int wisv_destroy(wisv_ctx* ctx)
+{
+    if (!ctx) return WISV_EINVAL;
+    free_ctx(ctx);
+    return WISV_OK;
+}
+
+int wisv_plan(const wisv_ctx* c, int32_t R, int32_t P, int32_t* lm_tile_n, int32_t* lm_tiles, int32_t* lm_ctas,
+              int32_t* head_tile_n, int32_t* head_tiles, int32_t* head_ctas)
+{
+    if (!c || R < 1 || P < 0) return WISV_EINVAL;
+    const Plan a = plan_lm(c, R);
+    if (lm_tile_n) *lm_tile_n = a.tile_n;
+    if (lm_tiles) *lm_tiles = a.m_tiles * a.n_tiles;
+    if (lm_ctas) *lm_ctas = a.ctas;
+    const Plan h = plan_head(c, P > 0 ? P : 1);
+    if (head_tile_n) *head_tile_n = h.tile_n;
+    if (head_tiles) *head_tiles = P > 0 ? h.m_tiles * h.n_tiles : 0;
+    if (head_ctas) *head_ctas = P > 0 ? h.ctas : 0;
+    return WISV_OK;
+}
+
+int64_t wisv_launch_count(const wisv_ctx* c) { return c ? c->launches : 0; }
+
+int wisv_verify(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda_stream)
+{
+    int T = 0, R = 0, P = 0;
+    const int vrc = validate_batch(c, b, r, &T, &R, &P);
+    if (vrc != WISV_OK) return vrc;
+    if (b->B == 0) return WISV_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const bool sh = (b->mode & WISV_MODE_SH) != 0;
+    const bool stoch = (b->mode & WISV_ACCEPT_STOCHASTIC) != 0;
+    const wisv_config& cf = c->cfg;
+
+    cudaEvent_t* ev = nullptr;
+    if (c->prof_n > 0) ev = c->prof_ev + (size_t)(c->prof_calls % c->prof_n) * (kStages + 1);
+
+    BatchIndex ix{b->B, b->k_off ? 0 : b->K, b->k_off};
+
+    // ---- 1. pack: bf16 window rows, head input rows, row -> token map
+    if (ev) WISV_CUDA(cudaEventRecord(ev[0], st));
+    PackParams pp;
+    memset(&pp, 0, sizeof pp);
+    pp.ix = ix; pp.R = R; pp.P = P; pp.H = cf.H; pp.H_d = cf.H_d; pp.V = cf.V; pp.shift = cf.head_row_shift;
+    pp.mode_sh = sh ? 1 : 0;
+    pp.target_hidden = b->target_hidden; pp.draft_hidden = b->draft_hidden; pp.draft_tokens = b->draft_tokens;
+    pp.sel_off = b->sel_off; pp.sel_pos = b->sel_pos;
+    pp.X = c->X; pp.Z = c->Z; pp.row_tok = c->row_tok; pp.row_flag = c->row_flag; pp.tok_logit = c->tok_logit;
+    pp.pos_req = c->pos_req; pp.pos_i = c->pos_i;
+    pack_kernel<<<R + P, 256, 0, st>>>(pp);
+    WISV_CUDA(cudaGetLastError());
+    c->launches++;
+
+    // ---- 2. LM head: logits reduced on the fly
+    if (ev) WISV_CUDA(cudaEventRecord(ev[1], st));
+    const Plan pl = plan_lm(c, R);
+    if ((size_t)R * pl.n_tiles > c->lm_part_elems) return WISV_ECAPACITY;
+    {
+        GemmParams gp = base_params(c, pl, R, cf.V, cf.H);
+        gp.lm_part = c->lm_part; gp.row_tok = c->row_tok; gp.tok_logit = c->tok_logit;
+        const int rc = launch_gemm<EPI_LMHEAD>(c, c->tmX, c->tmW[pl.tile_n / 16 - 1], gp, pl, st);
+        if (rc != WISV_OK) return rc;
+    }
+
+    // ---- 3. decision head on the evaluated positions
+    if (ev) WISV_CUDA(cudaEventRecord(ev[2], st));
+    Plan ph{};
+    if (P > 0) {
+        ph = plan_head(c, P);
+        if ((size_t)P * ph.n_tiles > c->head_part_elems) return WISV_ECAPACITY;
+        GemmParams gp = base_params(c, ph, P, cf.d_J, cf.H_d + cf.H);
+        gp.head_part = c->head_part; gp.b1 = c->w.b1; gp.w2 = c->w.w2; gp.w1c = c->W1c; gp.csi = b->csi;
+        gp.pos_req = c->pos_req; gp.d_c = cf.d_c; gp.act = cf.act;
+        const int rc = launch_gemm<EPI_HEAD>(c, c->tmZ, c->tmW1[ph.tile_n / 16 - 1], gp, ph, st);
+        if (rc != WISV_OK) return rc;
+    }
+
+    // ---- 4. merge, localize, scan, emit
+    if (ev) WISV_CUDA(cudaEventRecord(ev[3], st));
+    TailParams tp;
+    memset(&tp, 0, sizeof tp);
+    tp.ix = ix; tp.P = P; tp.V = cf.V; tp.n_tiles_lm = pl.n_tiles; tp.n_tiles_head = ph.n_tiles; tp.mode_sh = sh ? 1 : 0;
+    tp.stochastic = stoch ? 1 : 0; tp.b2 = c->w.b2; tp.tau = (b->tau != b->tau) ? cf.tau : b->tau;
+    tp.lm_part = c->lm_part; tp.tok_logit = c->tok_logit; tp.row_flag = c->row_flag; tp.draft_tokens = b->draft_tokens;
+    tp.head_part = c->head_part; tp.pos_i = c->pos_i; tp.sel_off = b->sel_off; tp.draft_q = b->draft_q;
+    tp.uniforms = b->uniforms;
+    tp.accept_len = r->accept_len; tp.correction = r->correction_token; tp.argmax = r->argmax; tp.lse = r->lse;
+    tp.p_draft = r->p_draft; tp.head_prob = r->head_prob;
+    tp.mismatch_mask = reinterpret_cast<unsigned long long*>(r->mismatch_mask); tp.n_mismatch = r->n_mismatch;
+    tp.status = r->status;
+    tail_kernel<<<b->B, 256, 0, st>>>(tp);
+    WISV_CUDA(cudaGetLastError());
+    c->launches++;
+    if (ev) { WISV_CUDA(cudaEventRecord(ev[4], st)); c->prof_calls++; }
+    return WISV_OK;
+}
+
+int wisv_debug_logits(wisv_ctx* c, const float* target_hidden, int32_t R, float* logits_out, void* cuda_stream)
+{
+    if (!c || !target_hidden || !logits_out) return WISV_EINVAL;
+    if (R < 1 || R > c->cfg.max_rows) return WISV_ECAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    // rows are cast with the pack kernel, as a batch of R one-row windows without tokens
+    PackParams pp;
+    memset(&pp, 0, sizeof pp);
+    pp.ix = BatchIndex{R, 0, nullptr}; pp.R = R; pp.P = 0; pp.H = c->cfg.H; pp.H_d = c->cfg.H_d; pp.V = c->cfg.V;
+    pp.target_hidden = target_hidden; pp.X = c->X; pp.row_tok = c->row_tok; pp.row_flag = c->row_flag;
+    pp.tok_logit = c->tok_logit;
+    pack_kernel<<<R, 256, 0, st>>>(pp);
+    WISV_CUDA(cudaGetLastError());
+    c->launches++;
+    const Plan pl = plan_lm(c, R);
+    GemmParams gp = base_params(c, pl, R, c->cfg.V, c->cfg.H);
+    gp.raw_out = logits_out;
+    return launch_gemm<EPI_RAW>(c, c->tmX, c->tmW[pl.tile_n / 16 - 1], gp, pl, st);
+}
+
+int wisv_device_error(wisv_ctx* c, void* cuda_stream, int32_t* flags)
+{
+    if (!c || !flags) return WISV_EINVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    WISV_CUDA(cudaStreamSynchronize(st));
+    int32_t v = 0;
+    WISV_CUDA(cudaMemcpy(&v, c->err, sizeof v, cudaMemcpyDeviceToHost));
+    if (v != 0) WISV_CUDA(cudaMemset(c->err, 0, sizeof v));
+    *flags = v;
+    return WISV_OK;
+}
+
+int wisv_profile_enable(wisv_ctx* c, int32_t n_calls)
+{
+    if (!c || n_calls < 0 || n_calls > 4096) return WISV_EINVAL;
+    if (c->prof_ev) {
+        for (int i = 0; i < c->prof_n * (kStages + 1); ++i) cudaEventDestroy(c->prof_ev[i]);
+        free(c->prof_ev);
+        c->prof_ev = nullptr;
+    }
+    c->prof_n = 0;
+    c->prof_calls = 0;
+    if (n_calls == 0) return WISV_OK;
+    c->prof_ev = static_cast<cudaEvent_t*>(calloc((size_t)n_calls * (kStages + 1), sizeof(cudaEvent_t)));
+    if (!c->prof_ev) return WISV_ENOMEM;
+    for (int i = 0; i < n_calls * (kStages + 1); ++i) WISV_CUDA(cudaEventCreate(&c->prof_ev[i]));
+    c->prof_n = n_calls;
+    return WISV_OK;
+}
+
+int wisv_profile_read(wisv_ctx* c, int32_t stage, float* ms, int32_t cap, int32_t* n_out)
+{
+    if (!c || !ms || !n_out || stage < 0 || stage >= kStages || cap < 0) return WISV_EINVAL;
+    *n_out = 0;
+    if (c->prof_n == 0) return WISV_OK;
+    const long long have = c->prof_calls < c->prof_n ? c->prof_calls : c->prof_n;
+    const long long first = c->prof_calls - have;
+    int n = 0;
+    for (long long k = first; k < c->prof_calls && n < cap; ++k) {
+        cudaEvent_t* ev = c->prof_ev + (size_t)(k % c->prof_n) * (kStages + 1);
+        WISV_CUDA(cudaEventSynchronize(ev[kStages]));
+        float t = 0.0f;
+        WISV_CUDA(cudaEventElapsedTime(&t, ev[stage], ev[stage + 1]));
+        ms[n++] = t;
+    }
+    *n_out = n;
+    return WISV_OK;
+}
+
+int wisv_verify_host(wisv_ctx* c, const wisv_batch* hb, const wisv_result* hr, void* cuda_stream)
+{
+    if (!c || !hb || !hr) return WISV_EINVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    HostStaging& h = c->hs;
+    const wisv_config& cf = c->cfg;
+    const int maxB = cf.max_requests, maxR = cf.max_rows, maxT = cf.max_rows - 1 > 0 ? cf.max_rows - 1 : 1;
+    if (!h.ready) {
+        int rc = WISV_OK;
+        do {
+            if ((rc = dev_alloc(&h.target_hidden, (size_t)maxR * cf.H))) break;
+            if ((rc = dev_alloc(&h.draft_tokens, (size_t)maxT))) break;
+            if ((rc = dev_alloc(&h.draft_hidden, (size_t)c->max_pos * cf.H_d))) break;
+            if ((rc = dev_alloc(&h.k_off, (size_t)maxB + 1))) break;
+            if ((rc = dev_alloc(&h.sel_off, (size_t)maxB + 1))) break;
+            if ((rc = dev_alloc(&h.sel_pos, (size_t)c->max_pos))) break;
+            if ((rc = dev_alloc(&h.csi, (size_t)maxB * (cf.d_c > 0 ? cf.d_c : 1)))) break;
+            if ((rc = dev_alloc(&h.draft_q, (size_t)maxT))) break;
+            if ((rc = dev_alloc(&h.uniforms, (size_t)maxT))) break;
+            if ((rc = dev_alloc(&h.accept_len, (size_t)maxB))) break;
+            if ((rc = dev_alloc(&h.correction, (size_t)maxB))) break;
+            if ((rc = dev_alloc(&h.argmax, (size_t)maxR))) break;
+            if ((rc = dev_alloc(&h.lse, (size_t)maxR))) break;
+            if ((rc = dev_alloc(&h.p_draft, (size_t)maxT))) break;
+            if ((rc = dev_alloc(&h.head_prob, (size_t)c->max_pos))) break;
+            if ((rc = dev_alloc(&h.mask, (size_t)maxB))) break;
+            if ((rc = dev_alloc(&h.n_mismatch, (size_t)maxB))) break;
+            if ((rc = dev_alloc(&h.status, (size_t)maxB))) break;
+        } while (0);
+        if (rc != WISV_OK) return rc;
+        h.ready = true;
+    }
+    // the device-side view of the batch, validated before any copy
+    wisv_batch db = *hb;
+    wisv_result dr;
+    memset(&dr, 0, sizeof dr);
+    db.k_off = hb->k_off ? h.k_off : nullptr;
+    db.target_hidden = hb->target_hidden ? h.target_hidden : nullptr;
+    db.draft_tokens = hb->draft_tokens ? h.draft_tokens : nullptr;
+    db.draft_hidden = hb->draft_hidden ? h.draft_hidden : nullptr;
+    db.sel_off = hb->sel_off ? h.sel_off : nullptr;
+    db.sel_pos = hb->sel_pos ? h.sel_pos : nullptr;
+    db.csi = hb->csi ? h.csi : nullptr;
+    db.draft_q = hb->draft_q ? h.draft_q : nullptr;
+    db.uniforms = hb->uniforms ? h.uniforms : nullptr;
+    dr.accept_len = hr->accept_len ? h.accept_len : nullptr;
+    dr.correction_token = hr->correction_token ? h.correction : nullptr;
+    dr.argmax = hr->argmax ? h.argmax : nullptr;
+    dr.lse = hr->lse ? h.lse : nullptr;
+    dr.p_draft = hr->p_draft ? h.p_draft : nullptr;
+    dr.head_prob = hr->head_prob ? h.head_prob : nullptr;
+    dr.mismatch_mask = hr->mismatch_mask ? reinterpret_cast<uint64_t*>(h.mask) : nullptr;
+    dr.n_mismatch = hr->n_mismatch ? h.n_mismatch : nullptr;
+    dr.status = hr->status ? h.status : nullptr;
+    int T = 0, R = 0, P = 0;
+    const int vrc = validate_batch(c, &db, &dr, &T, &R, &P);
+    if (vrc != WISV_OK) return vrc;
+    if (hb->B == 0) return WISV_OK;
+    const int B = hb->B;
+    const bool sh = (hb->mode & WISV_MODE_SH) != 0;
+    const bool stoch = (hb->mode & WISV_ACCEPT_STOCHASTIC) != 0;
+#define H2D(dst, src, n) \
+    do { if ((src) && (n) > 0) WISV_CUDA(cudaMemcpyAsync((dst), (src), (size_t)(n), cudaMemcpyHostToDevice, st)); } while (0)
+#define D2H(dst, src, n) \
+    do { if ((dst) && (n) > 0) WISV_CUDA(cudaMemcpyAsync((dst), (src), (size_t)(n), cudaMemcpyDeviceToHost, st)); } while (0)
+    H2D(h.k_off, hb->k_off, sizeof(int32_t) * (B + 1));
+    H2D(h.target_hidden, hb->target_hidden, sizeof(float) * (size_t)R * cf.H);
+    H2D(h.draft_tokens, hb->draft_tokens, sizeof(int32_t) * (size_t)T);
+    H2D(h.draft_hidden, hb->draft_hidden, sizeof(float) * (size_t)P * cf.H_d);
+    if (sh) {
+        H2D(h.sel_off, hb->sel_off, sizeof(int32_t) * (B + 1));
+        H2D(h.sel_pos, hb->sel_pos, sizeof(int32_t) * (size_t)P);
+    }
+    H2D(h.csi, hb->csi, sizeof(float) * (size_t)B * cf.d_c);
+    if (stoch) {
+        H2D(h.draft_q, hb->draft_q, sizeof(float) * (size_t)T);
+        H2D(h.uniforms, hb->uniforms, sizeof(float) * (size_t)T);
+    }
+    const int rc = wisv_verify(c, &db, &dr, cuda_stream);
+    if (rc != WISV_OK) return rc;
+    D2H(hr->accept_len, h.accept_len, sizeof(int32_t) * B);
+    D2H(hr->correction_token, h.correction, sizeof(int32_t) * B);
+    D2H(hr->argmax, h.argmax, sizeof(int32_t) * (size_t)R);
+    D2H(hr->lse, h.lse, sizeof(float) * (size_t)R);
+    D2H(hr->p_draft, h.p_draft, sizeof(float) * (size_t)T);
+    D2H(hr->head_prob, h.head_prob, sizeof(float) * (size_t)P);
+    D2H(hr->mismatch_mask, h.mask, sizeof(uint64_t) * B);
+    D2H(hr->n_mismatch, h.n_mismatch, sizeof(int32_t) * B);
+    D2H(hr->status, h.status, sizeof(int32_t) * B);
+#undef H2D
+#undef D2H
+    int32_t dev_err = 0;
+    WISV_CUDA(cudaMemcpyAsync(&dev_err, c->err, sizeof dev_err, cudaMemcpyDeviceToHost, st));
+    WISV_CUDA(cudaStreamSynchronize(st));
+    if (dev_err != 0) { (void)cudaMemset(c->err, 0, sizeof dev_err); return WISV_EDEVICE; }
+    return WISV_OK;
+}
+
+}  // extern "C"

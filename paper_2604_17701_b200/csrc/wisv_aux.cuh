@@ -1,0 +1,263 @@
+// The small kernels around the two GEMMs:
+//   pack_kernel  - rounds the fp32 hidden states to bf16 (nearest even) and builds
+//                  the decision head's input rows z = [h^D ; h^T] for every evaluated
+//                  position (all T in full-hidden mode, the packed list in
+//                  selective-hidden mode), plus the row -> draft-token map.
+//   tail_kernel  - per request: merges the LM-head partials into argmax / log-sum-exp,
+//                  forms the candidate set S, finishes the head probabilities, finds
+//                  the first rejected position and emits the feedback pair.
+//   split_w1_kernel - one-time repack of W1 into a TMA-legal bf16 block and an fp32 CSI block.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <math_constants.h>
+#include <stdint.h>
+
+namespace wisv {
+
+struct BatchIndex {
+    int32_t B, K;               // K > 0: uniform windows; K == 0: ragged, k_off given
+    const int32_t* k_off;       // [B+1] or nullptr
+    __device__ __forceinline__ int koff(int b) const { return k_off ? k_off[b] : b * K; }
+    __device__ __forceinline__ int roff(int b) const { return koff(b) + b; }
+    // request owning token t (largest b with koff(b) <= t)
+    __device__ int req_of_token(int t) const {
+        if (!k_off) return K > 0 ? min(t / K, B - 1) : 0;
+        int lo = 0, hi = B - 1;
+        while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (k_off[mid] <= t) lo = mid; else hi = mid - 1; }
+        return lo;
+    }
+    // request owning window row r (largest b with roff(b) <= r)
+    __device__ int req_of_row(int r) const {
+        if (!k_off) return min(r / (K + 1), B - 1);
+        int lo = 0, hi = B - 1;
+        while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (k_off[mid] + mid <= r) lo = mid; else hi = mid - 1; }
+        return lo;
+    }
+};
+
+struct PackParams {
+    BatchIndex ix;
+    int32_t R, P, H, H_d, V, shift, mode_sh;
+    const float* target_hidden;   // [R, H]
+    const float* draft_hidden;    // [P, H_d]
+    const int32_t* draft_tokens;  // [T]
+    const int32_t* sel_off;       // [B+1] (SH)
+    const int32_t* sel_pos;       // [P]   (SH)
+    __nv_bfloat16* X;             // [R, H]
+    __nv_bfloat16* Z;             // [P, H_d + H]
+    int32_t* row_tok;             // [R] clamped draft token or -1
+    int32_t* row_flag;            // [R] WISV_ST_BAD_TOKEN or 0
+    float* tok_logit;             // [R]
+    int32_t* pos_req;             // [P]
+    int32_t* pos_i;               // [P] window position or -1 when the list entry is invalid
+};
+
+__device__ __forceinline__ void cast_row(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, int n) {
+    // n % 8 == 0; 8 floats in, one 16-byte store out
+    for (int i = threadIdx.x * 8; i < n; i += blockDim.x * 8) {
+        const float4 a = *reinterpret_cast<const float4*>(src + i);
+        const float4 b = *reinterpret_cast<const float4*>(src + i + 4);
+        __nv_bfloat162 o[4];
+        o[0] = __floats2bfloat162_rn(a.x, a.y);
+        o[1] = __floats2bfloat162_rn(a.z, a.w);
+        o[2] = __floats2bfloat162_rn(b.x, b.y);
+        o[3] = __floats2bfloat162_rn(b.z, b.w);
+        *reinterpret_cast<uint4*>(dst + i) = *reinterpret_cast<const uint4*>(o);
+    }
+}
+
+__global__ void __launch_bounds__(256) pack_kernel(const PackParams p)
+{
+    __shared__ int s_src_row;
+    const int blk = blockIdx.x;
+    if (blk < p.R) {
+        const int r = blk;
+        if (threadIdx.x == 0) {
+            const int b = p.ix.req_of_row(r);
+            const int i = r - p.ix.roff(b);
+            const int Kb = p.ix.koff(b + 1) - p.ix.koff(b);
+            int tok = -1, flag = 0;
+            if (i < Kb) {
+                tok = p.draft_tokens[p.ix.koff(b) + i];
+                if (tok < 0 || tok >= p.V) { flag = 2; tok = tok < 0 ? 0 : p.V - 1; }
+            }
+            p.row_tok[r] = tok;
+            p.row_flag[r] = flag;
+            p.tok_logit[r] = 0.0f;
+        }
+        cast_row(p.target_hidden + (size_t)r * p.H, p.X + (size_t)r * p.H, p.H);
+    } else {
+        const int j = blk - p.R;          // evaluated position
+        if (threadIdx.x == 0) {
+            int b, i;
+            if (p.mode_sh) {
+                int lo = 0, hi = p.ix.B - 1;
+                while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (p.sel_off[mid] <= j) lo = mid; else hi = mid - 1; }
+                b = lo;
+                i = p.sel_pos[j];
+            } else {
+                b = p.ix.req_of_token(j);
+                i = j - p.ix.koff(b);
+            }
+            const int Kb = p.ix.koff(b + 1) - p.ix.koff(b);
+            const bool good = (i >= 0 && i < Kb);
+            p.pos_req[j] = b;
+            p.pos_i[j] = good ? i : -1;
+            s_src_row = p.ix.roff(b) + (good ? i + p.shift : 0);
+        }
+        __syncthreads();
+        const size_t zw = (size_t)(p.H_d + p.H);
+        cast_row(p.draft_hidden + (size_t)j * p.H_d, p.Z + (size_t)j * zw, p.H_d);
+        cast_row(p.target_hidden + (size_t)s_src_row * p.H, p.Z + (size_t)j * zw + p.H_d, p.H);
+    }
+}
+
+// W1 [d_J, H_d + H + d_c] bf16 -> W1p [d_J, H_d + H] bf16 (16-byte pitch) and W1c [d_J, d_c] fp32
+__global__ void split_w1_kernel(const __nv_bfloat16* __restrict__ W1, __nv_bfloat16* __restrict__ W1p,
+                                float* __restrict__ W1c, int d_J, int hd_h, int d_c)
+{
+    const int j = blockIdx.x;
+    const size_t src = (size_t)j * (hd_h + d_c);
+    for (int k = threadIdx.x; k < hd_h; k += blockDim.x) W1p[(size_t)j * hd_h + k] = W1[src + k];
+    for (int c = threadIdx.x; c < d_c; c += blockDim.x) W1c[(size_t)j * d_c + c] = __bfloat162float(W1[src + hd_h + c]);
+}
+
+struct TailParams {
+    BatchIndex ix;
+    int32_t P, V, n_tiles_lm, n_tiles_head, mode_sh, stochastic;
+    float b2, tau;
+    const float4* lm_part;        // [R][n_tiles_lm]
+    const float* tok_logit;       // [R]
+    const int32_t* row_flag;      // [R]
+    const int32_t* draft_tokens;  // [T]
+    const float* head_part;       // [P][n_tiles_head]
+    const int32_t* pos_i;         // [P]
+    const int32_t* sel_off;       // [B+1] (SH)
+    const float* draft_q;         // [T] (stochastic)
+    const float* uniforms;        // [T] (stochastic)
+    int32_t* accept_len; int32_t* correction; int32_t* argmax; float* lse; float* p_draft; float* head_prob;
+    unsigned long long* mismatch_mask; int32_t* n_mismatch; int32_t* status;
+};
+
+struct RowStat { float mx; int idx; float sum; };
+
+__device__ __forceinline__ void merge_stat(RowStat& a, float mx, int idx, float sum) {
+    if (mx == -CUDART_INF_F && sum == 0.0f) return;               // empty
+    if (mx > a.mx) {
+        a.sum = a.sum * expf(a.mx - mx) + sum;                  // exp(-inf) = 0 covers the first merge
+        a.mx = mx; a.idx = idx;
+    } else {
+        a.sum += sum * expf(mx - a.mx);
+        if (mx == a.mx && idx < a.idx) a.idx = idx;               // lowest token id wins ties
+    }
+}
+
+__global__ void __launch_bounds__(256) tail_kernel(const TailParams p)
+{
+    constexpr int kMaxK = 64;
+    __shared__ int s_arg[kMaxK + 1];
+    __shared__ float s_lse[kMaxK + 1];
+    __shared__ float s_prob[kMaxK];
+    __shared__ int s_has[kMaxK];
+    __shared__ int s_flag;
+
+    const int b = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    const int k0 = p.ix.koff(b);
+    const int Kb = min(p.ix.koff(b + 1) - k0, kMaxK);
+    const int r0 = k0 + b;
+
+    if (threadIdx.x < kMaxK) { s_has[threadIdx.x] = 0; s_prob[threadIdx.x] = 0.0f; }
+    if (threadIdx.x == 0) s_flag = 0;
+    __syncthreads();
+
+    // ---- merge the per-tile (max, argidx, sumexp) partials of each window row
+    int flag = 0;
+    for (int i = warp; i <= Kb; i += nwarps) {
+        const int r = r0 + i;
+        RowStat st{-CUDART_INF_F, 0x7fffffff, 0.0f};
+        const float4* part = p.lm_part + (size_t)r * p.n_tiles_lm;
+        for (int n = lane; n < p.n_tiles_lm; n += 32) {
+            const float4 v = part[n];
+            merge_stat(st, v.x, __float_as_int(v.y), v.z);
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const float omx = __shfl_xor_sync(0xffffffffu, st.mx, off);
+            const int oidx = __shfl_xor_sync(0xffffffffu, st.idx, off);
+            const float osum = __shfl_xor_sync(0xffffffffu, st.sum, off);
+            merge_stat(st, omx, oidx, osum);
+        }
+        const float l = st.mx + logf(st.sum);
+        if (lane == 0) {
+            s_arg[i] = st.idx;
+            s_lse[i] = l;
+            if (p.argmax) p.argmax[r] = st.idx;
+            if (p.lse) p.lse[r] = l;
+            if (!isfinite(l)) flag |= 4;
+            flag |= p.row_flag[r];
+        }
+    }
+
+    // ---- finish the decision head: s = b2 + sum of per-tile partial dot products
+    int e0, e1;
+    if (p.mode_sh) { e0 = max(p.sel_off[b], 0); e1 = min(p.sel_off[b + 1], p.P); } else { e0 = k0; e1 = k0 + Kb; }
+    for (int e = e0 + warp; e < e1; e += nwarps) {
+        float s = 0.0f;
+        const float* hp = p.head_part + (size_t)e * p.n_tiles_head;
+        for (int n = lane; n < p.n_tiles_head; n += 32) s += hp[n];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+        s += p.b2;
+        const float prob = 1.0f / (1.0f + expf(-s));
+        if (lane == 0) {
+            if (p.head_prob) p.head_prob[e] = prob;
+            const int i = p.pos_i[e];
+            if (i >= 0 && i < Kb) { s_prob[i] = prob; s_has[i] = 1; } else { flag |= 8; }
+            if (!isfinite(s)) flag |= 4;
+        }
+    }
+    if (flag) atomicOr(&s_flag, flag);
+    __syncthreads();
+
+    // ---- Localize, first-reject scan, emission (one warp; windows hold at most 64 tokens)
+    if (warp == 0) {
+        unsigned cand_bits[2], rej_bits[2];
+        int missing = 0;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int i = lane + 32 * h;
+            bool cand = false, rej = false;
+            if (i < Kb) {
+                const int t = k0 + i;
+                const float pd = expf(p.tok_logit[r0 + i] - s_lse[i]);
+                if (p.p_draft) p.p_draft[t] = pd;
+                if (p.stochastic) {
+                    const float alpha = fminf(1.0f, pd / p.draft_q[t]);
+                    cand = !(p.uniforms[t] < alpha);
+                } else {
+                    cand = p.draft_tokens[t] != s_arg[i];
+                }
+                const bool has = s_has[i] != 0;
+                rej = cand && (!has || s_prob[i] >= p.tau);
+                if (cand && !has) missing = 1;
+            }
+            cand_bits[h] = __ballot_sync(0xffffffffu, cand);
+            rej_bits[h] = __ballot_sync(0xffffffffu, rej);
+        }
+        missing = __any_sync(0xffffffffu, missing);
+        if (lane == 0) {
+            const unsigned long long rej = (unsigned long long)rej_bits[0] | ((unsigned long long)rej_bits[1] << 32);
+            const unsigned long long cnd = (unsigned long long)cand_bits[0] | ((unsigned long long)cand_bits[1] << 32);
+            const int A = rej ? (__ffsll((long long)rej) - 1) : Kb;
+            p.accept_len[b] = A;
+            p.correction[b] = s_arg[A];
+            if (p.mismatch_mask) p.mismatch_mask[b] = cnd;
+            if (p.n_mismatch) p.n_mismatch[b] = __popcll(cnd);
+            if (p.status) p.status[b] = s_flag | (missing ? 1 : 0);
+        }
+    }
+}
+
+}  // namespace wisv

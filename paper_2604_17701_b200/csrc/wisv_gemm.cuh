@@ -1,0 +1,323 @@
+// Persistent, warp-specialised bf16 GEMM for sm_100a whose epilogue reduces each
+// output row over the N dimension instead of storing it:
+//
+//   D[row, n] = sum_k A[row, k] * Bw[n, k]      A: activations (rows x K), Bw: weights (N x K)
+//
+// * LM-head epilogue: per (row, N-tile) the running max, its lowest column index
+//   and sum exp(D - max) (the pieces of argmax / log-sum-exp), plus the one logit
+//   at the row's draft token.  The logits never leave TMEM / registers.
+// * Decision-head epilogue: per (row, N-tile) the partial dot product
+//   sum_n w2[n] * act(D[row, n] + b1[n] + W1c[n, :] . csi[row]).
+// * Raw epilogue (bring-up / tests): D written to global memory.
+//
+// One CTA per SM loops over (m, n) tiles.  Warp 0 streams A and Bw tiles with TMA
+// into a ring of shared-memory stages, warp 1 issues tcgen05.mma (M = 128,
+// N = tile_n, K = 16) into one of two TMEM accumulators, warps 2-5 drain the other
+// accumulator with tcgen05.ld and run the epilogue, so the epilogue of tile i
+// overlaps the main loop of tile i+1.  Every wait is bounded.
+#pragma once
+
+#include <math_constants.h>
+
+#include "wisv_ptx.cuh"
+
+namespace wisv {
+
+constexpr int kTileM = 128;          // rows per tile = TMEM lanes
+constexpr int kBlockK = 64;          // bf16 elements per 128-byte swizzled row
+constexpr int kUmmaK = 16;
+constexpr int kMaxTileN = 256;
+constexpr int kAccCols = 256;        // TMEM columns per accumulator stage
+constexpr int kTmemCols = 512;
+constexpr int kGemmThreads = 192;
+constexpr int kEpiThreads = 128;
+constexpr int kMaxStages = 12;
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s
+constexpr int kMaxDc = 16;
+
+enum { EPI_LMHEAD = 0, EPI_HEAD = 1, EPI_RAW = 2 };
+
+struct GemmParams {
+    int32_t rows;        // valid rows of A
+    int32_t n_total;     // rows of Bw (vocabulary size or d_J)
+    int32_t k_blocks;    // ceil(K / 64)
+    int32_t tile_n;      // Bw rows per tile: multiple of 16, <= 256
+    int32_t m_tiles, n_tiles;
+    int32_t stages;
+    int32_t* err;        // device error word (bit 0: a bounded wait gave up)
+    // LM-head epilogue
+    float4* lm_part;          // [rows][n_tiles] = {max, bits(argidx), sumexp, 0}
+    const int32_t* row_tok;   // [rows] draft token of the row or -1
+    float* tok_logit;         // [rows]
+    // decision-head epilogue
+    float* head_part;         // [rows][n_tiles]
+    const float* b1;          // [n_total]
+    const float* w2;          // [n_total]
+    const float* w1c;         // [n_total][d_c] fp32 CSI columns of W1
+    const float* csi;         // [B][d_c]
+    const int32_t* pos_req;   // [rows] request of each position
+    int32_t d_c;
+    int32_t act;              // 0 ReLU, 1 exact GELU
+    // raw epilogue
+    float* raw_out;           // [rows][n_total]
+};
+
+__host__ __device__ inline uint32_t gemm_stage_bytes(int tile_n) {
+    return static_cast<uint32_t>(kTileM * kBlockK * 2 + tile_n * kBlockK * 2);
+}
+// bytes after the stage ring: barriers + tmem slot + abort flag, then epilogue constants
+__host__ __device__ inline uint32_t gemm_tail_bytes(int tile_n, int d_c) {
+    return 512u + 2u * (static_cast<uint32_t>(tile_n) * static_cast<uint32_t>(2 + d_c) +
+                        static_cast<uint32_t>(kEpiThreads * d_c)) * 4u;
+}
+
+__device__ __forceinline__ float act_apply(float x, int act) {
+    if (act == 0) return fmaxf(x, 0.0f);
+    return 0.5f * x * (1.0f + erff(x * 0.70710678118654752440f));
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                      const GemmParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;
+    uint8_t* smem = smem_raw + pad;                       // 1024-byte aligned: swizzle atoms need it
+    const uint32_t smem_base = raw_addr + pad;
+
+    const uint32_t a_bytes = kTileM * kBlockK * 2;
+    const uint32_t b_bytes = static_cast<uint32_t>(p.tile_n) * kBlockK * 2;
+    const uint32_t stage_bytes = a_bytes + b_bytes;
+    const uint32_t ring_bytes = stage_bytes * static_cast<uint32_t>(p.stages);
+
+    // barriers: full[S], empty[S], acc_full[2], acc_empty[2], drain
+    const uint32_t bar_base = smem_base + ring_bytes;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (kMaxStages + s); };
+    auto acc_full_bar = [&](int s) { return bar_base + 8u * (2 * kMaxStages + s); };
+    auto acc_empty_bar = [&](int s) { return bar_base + 8u * (2 * kMaxStages + 2 + s); };
+    const uint32_t drain_bar = bar_base + 8u * (2 * kMaxStages + 4);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + ring_bytes + 8 * (2 * kMaxStages + 5));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [0] abort, [1] drain scratch
+    float* epi_const = reinterpret_cast<float*>(smem + ring_bytes + 512);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int total_tiles = p.m_tiles * p.n_tiles;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(acc_full_bar(s), 1); mbar_init(acc_empty_bar(s), 4); }
+        mbar_init(drain_bar, 1);
+        abort_flag[0] = 0;
+        abort_flag[1] = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            long long issued = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                const int m = t % p.m_tiles, n = t / p.m_tiles;
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, kWaitLimitNs)) { ok = false; break; }
+                    const uint32_t a_dst = smem_base + stage_bytes * s;
+                    mbar_expect_tx(full_bar(s), stage_bytes);
+                    tma_load_2d(a_dst, &tmA, kb * kBlockK, m * kTileM, full_bar(s));
+                    tma_load_2d(a_dst + a_bytes, &tmB, kb * kBlockK, n * p.tile_n, full_bar(s));
+                    ++issued;
+                    if (++s == p.stages) { s = 0; ph ^= 1u; }
+                }
+            }
+            if (!ok) {
+                // let copies already in flight land before the CTA retires
+                const int inflight = issued < p.stages ? static_cast<int>(issued) : p.stages;
+                int ws = s;
+                uint32_t wph = ph;
+                for (int i = 0; i < inflight; ++i) {
+                    if (--ws < 0) { ws = p.stages - 1; wph ^= 1u; }
+                    mbar_wait_bounded(full_bar(ws), wph, abort_flag + 1, kWaitLimitNs);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = idesc_bf16_f32(kTileM, static_cast<uint32_t>(p.tile_n));
+            int s = 0;
+            uint32_t ph = 0;
+            int local = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++local) {
+                const int as = local & 1;
+                const uint32_t aph = (local >> 1) & 1u;
+                if (!mbar_wait_bounded(acc_empty_bar(as), aph ^ 1u, abort_flag, kWaitLimitNs)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(as * kAccCols);
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!mbar_wait_bounded(full_bar(s), ph, abort_flag, kWaitLimitNs)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_base + stage_bytes * s;
+                    const uint64_t a_desc = smem_desc_k128(a_addr);
+                    const uint64_t b_desc = smem_desc_k128(a_addr + a_bytes);
+#pragma unroll
+                    for (int k = 0; k < kBlockK / kUmmaK; ++k) {
+                        // advancing K by 16 bf16 = 32 bytes = 2 descriptor units inside the swizzle atom
+                        umma_bf16(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(empty_bar(s));       // stage is free once these MMAs have read it
+                    if (++s == p.stages) { s = 0; ph ^= 1u; }
+                }
+                if (ok) umma_commit(acc_full_bar(as));
+            }
+            if (!ok) {
+                // drain whatever was issued before TMEM is released
+                umma_commit(drain_bar);
+                mbar_wait_bounded(drain_bar, 0, abort_flag + 1, kWaitLimitNs);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..5)
+        const int q = warp & 3;                            // TMEM lane quadrant this warp may read
+        const int et = threadIdx.x - 64;                   // 0..127 among epilogue threads
+        int local = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++local) {
+            const int m = t % p.m_tiles, n = t / p.m_tiles;
+            const int as = local & 1;
+            const uint32_t aph = (local >> 1) & 1u;
+            const int row = m * kTileM + q * 32 + lane;
+            const bool valid = row < p.rows;
+            const int n0 = n * p.tile_n;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(as * kAccCols);
+
+            const float* cb1 = nullptr; const float* cw2 = nullptr; const float* cwc = nullptr; const float* ccs = nullptr;
+            if (EPI == EPI_HEAD) {
+                // stage this tile's b1 / w2 / CSI weights and each row's CSI vector
+                // (double-buffered by accumulator stage, so one barrier per tile suffices)
+                float* buf = epi_const + as * (p.tile_n * (2 + p.d_c) + kEpiThreads * p.d_c);
+                float* wb1 = buf; float* ww2 = buf + p.tile_n; float* wwc = buf + 2 * p.tile_n;
+                float* wcs = buf + (2 + p.d_c) * p.tile_n;
+                for (int j = et; j < p.tile_n; j += kEpiThreads) {
+                    const bool in = (n0 + j) < p.n_total;
+                    wb1[j] = in ? p.b1[n0 + j] : 0.0f;
+                    ww2[j] = in ? p.w2[n0 + j] : 0.0f;
+                    for (int c = 0; c < p.d_c; ++c)
+                        wwc[c * p.tile_n + j] = in ? p.w1c[(size_t)(n0 + j) * p.d_c + c] : 0.0f;
+                }
+                const int rq = valid ? p.pos_req[row] : 0;
+                for (int c = 0; c < p.d_c; ++c) wcs[c * kEpiThreads + et] = valid ? p.csi[(size_t)rq * p.d_c + c] : 0.0f;
+                cb1 = wb1; cw2 = ww2; cwc = wwc; ccs = wcs;
+            }
+
+            bool got = mbar_wait_bounded(acc_full_bar(as), aph, abort_flag, kWaitLimitNs);
+            if (EPI == EPI_HEAD) {
+                // barrier over the 128 epilogue threads that also agrees on `got`
+                uint32_t all;
+                asm volatile(
+                    "{\n\t"
+                    ".reg .pred pi, po;\n\t"
+                    "setp.ne.u32 pi, %1, 0;\n\t"
+                    "barrier.cta.red.and.pred po, 1, 128, pi;\n\t"
+                    "selp.u32 %0, 1, 0, po;\n\t"
+                    "}\n"
+                    : "=r"(all) : "r"(got ? 1u : 0u) : "memory");
+                got = all != 0;
+            } else {
+                got = __all_sync(0xffffffffu, got);
+            }
+            if (!got) { ok = false; break; }
+            tc_fence_after();
+
+            float mx = -CUDART_INF_F, sum = 0.0f, hs = 0.0f;
+            int arg = 0;
+            const int tok = (EPI == EPI_LMHEAD && valid) ? p.row_tok[row] : -1;
+
+            for (int c0 = 0; c0 < p.tile_n; c0 += 16) {
+                uint32_t v[16];
+                __syncwarp();                                // tcgen05.ld is warp-collective
+                tmem_ld16(taddr + static_cast<uint32_t>(c0), v);
+                tmem_wait_ld();
+                if (!valid) continue;
+                const int col0 = n0 + c0;
+                if (EPI == EPI_LMHEAD) {
+                    float f[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) f[j] = (col0 + j < p.n_total) ? __uint_as_float(v[j]) : -CUDART_INF_F;
+                    float cm = f[0];
+                    int ci = 0;
+#pragma unroll
+                    for (int j = 1; j < 16; ++j) { if (f[j] > cm) { cm = f[j]; ci = j; } }
+                    if (cm > mx) {                           // strict: earlier (lower) index wins ties
+                        sum *= exp2f((mx - cm) * 1.4426950408889634f);
+                        mx = cm;
+                        arg = col0 + ci;
+                    }
+                    const float base = mx * 1.4426950408889634f;
+                    float acc = 0.0f;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) acc += exp2f(fmaf(f[j], 1.4426950408889634f, -base));
+                    sum += acc;
+                    if (static_cast<unsigned>(tok - col0) < 16u) {
+                        float tl = 0.0f;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) tl = (tok - col0 == j) ? f[j] : tl;
+                        p.tok_logit[row] = tl;
+                    }
+                } else if (EPI == EPI_HEAD) {
+                    float pre[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) pre[j] = __uint_as_float(v[j]) + cb1[c0 + j];
+                    for (int c = 0; c < p.d_c; ++c) {
+                        const float x = ccs[c * kEpiThreads + et];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) pre[j] = fmaf(x, cwc[c * p.tile_n + c0 + j], pre[j]);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) hs = fmaf(cw2[c0 + j], act_apply(pre[j], p.act), hs);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        if (col0 + j < p.n_total) p.raw_out[(size_t)row * p.n_total + col0 + j] = __uint_as_float(v[j]);
+                }
+            }
+            // accumulator drained: hand it back to the MMA warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty_bar(as));
+
+            if (valid) {
+                if (EPI == EPI_LMHEAD)
+                    p.lm_part[(size_t)row * p.n_tiles + n] = make_float4(mx, __int_as_float(arg), sum, 0.0f);
+                else if (EPI == EPI_HEAD)
+                    p.head_part[(size_t)row * p.n_tiles + n] = hs;
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+    if (threadIdx.x == 0 && (abort_flag[0] != 0)) atomicOr(p.err, 1);
+}
+
+}  // namespace wisv

@@ -1,0 +1,316 @@
+"""CUDA path versus the CPU oracle, element by element, through the C ABI."""
+import functools
+
+import numpy as np
+import pytest
+import torch
+
+import gen
+import oracle
+from paper_2604_17701_b200 import cases
+from parity import compare, oracle_ref_argmax, run_oracle
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@functools.lru_cache(maxsize=4)
+def _weights(cfg_key):
+    return gen.make_weights(cfg_key)
+
+
+def _shared_weights(cfg):
+    # weights depend only on the model dimensions and the weight seed
+    key = gen.VerifyConfig("w", B=1, K=1, H=cfg.H, H_d=cfg.H_d, d_c=cfg.d_c, d_J=cfg.d_J, V=cfg.V,
+                           match_rate=0.0, seed=cfg.seed, weight_seed=cfg.weight_seed)
+    return _weights(key)
+
+
+def _small(name="s", **kw):
+    base = dict(B=8, K=4, H=256, H_d=128, d_c=2, d_J=128, V=4096, match_rate=0.5, seed=0)
+    base.update(kw)
+    return gen.VerifyConfig(name, **base)
+
+
+def _run(cfg, *, act=None, tau=None, shift=0, ref_fn=oracle_ref_argmax):
+    case = cases.make_case(cfg, ref_fn, weights=_shared_weights(cfg))
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d, act=act, tau=tau, head_row_shift=shift)
+    out = cases.run(v, d)
+    torch.cuda.synchronize()
+    assert v.device_error() == 0
+    ref = run_oracle(case, act=act, tau=tau, head_row_shift=shift)
+    stats = compare(case, ref, out, cfg.tau if tau is None else tau)
+    v.close()
+    return case, ref, out, stats
+
+
+def test_raw_logits_match_oracle():
+    cfg = _small(B=8, K=4)
+    case = cases.make_case(cfg, oracle_ref_argmax)
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d)
+    L = v.debug_logits(d["target_hidden"]).cpu().numpy()
+    assert v.device_error() == 0
+    ref = oracle.lm_head(case["lm_head"], case["target_hidden"], want_logits=True)["logits"]
+    assert np.max(np.abs(L - ref)) < 2e-4
+    v.close()
+
+
+@pytest.mark.parametrize("act", ["gelu", "relu"])
+@pytest.mark.parametrize("shift", [0, 1])
+def test_tiny_config(act, shift):
+    _run(gen.config("tiny"), act=act, shift=shift)
+
+
+@pytest.mark.parametrize("kw", [
+    dict(V=1000),                              # vocabulary tail inside a tile
+    dict(V=4099, H=72, H_d=40),                # K tail (H not a multiple of 64), odd vocabulary
+    dict(B=1, K=1),                            # smallest window
+    dict(B=3, K=64, V=777),                    # longest window
+    dict(B=40, K=4),                           # R = 200: two row tiles, ragged second tile
+    dict(B=70, K=3, V=600, d_J=200),           # R = 280: three row tiles, head width not a tile multiple
+    dict(B=16, K=0, K_lo=1, K_hi=9),           # ragged windows
+    dict(match_rate=1.0),                      # full-match windows accept K
+    dict(match_rate=0.0),                      # every position a candidate
+    dict(d_c=0),                               # no CSI features
+    dict(d_c=5, d_J=48),                       # odd CSI width
+], ids=lambda kw: "-".join("%s%s" % (k, v) for k, v in kw.items()))
+def test_shapes(kw):
+    _run(_small(**kw))
+
+
+@pytest.mark.parametrize("tau", [0.0, 0.35, 0.65, 1.5])
+def test_thresholds(tau):
+    case, ref, out, _ = _run(_small(B=24, K=6, seed=3), tau=tau)
+    A = out.accept_len.cpu().numpy()
+    if tau > 1:
+        assert np.array_equal(A, case["k_len"])
+
+
+@pytest.mark.parametrize("kw", [dict(), dict(K=0, K_lo=2, K_hi=12, B=32), dict(match_rate=1.0), dict(match_rate=0.0)],
+                         ids=["uniform", "ragged", "emptyS", "fullS"])
+def test_selective_hidden(kw):
+    cfg = _small(mode="SH", seed=5, **{**dict(B=12, K=5), **kw})
+    case, ref, out, _ = _run(cfg)
+    # same decisions as full-hidden upload on the same traffic
+    fh = cases.make_case(cfg.with_(mode="FH"), oracle_ref_argmax, weights=_shared_weights(cfg))
+    d = cases.to_device(fh, DEV)
+    v = cases.make_verifier(d)
+    o2 = cases.run(v, d)
+    assert torch.equal(o2.accept_len, out.accept_len) and torch.equal(o2.correction_token, out.correction_token)
+    v.close()
+
+
+def test_selective_hidden_missing_upload_is_rejected_and_flagged():
+    cfg = _small(mode="SH", B=6, K=5, seed=7, match_rate=0.3)
+    case = cases.make_case(cfg, oracle_ref_argmax)
+    # drop the last uploaded hidden state of every request that has one
+    keep, counts = [], []
+    for b in range(cfg.B):
+        lo, hi = int(case["sel_off"][b]), int(case["sel_off"][b + 1])
+        kept = list(range(lo, max(lo, hi - 1)))
+        keep += kept
+        counts.append(len(kept))
+    keep = np.asarray(keep, np.int64)
+    case["sel_off"] = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    case["sel_pos"] = case["sel_pos"][keep]
+    case["draft_hidden"] = case["draft_hidden"][keep]
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d)
+    out = cases.run(v, d)
+    ref = run_oracle(case)
+    compare(case, ref, out, cfg.tau)
+    st = out.status.cpu().numpy()
+    assert np.array_equal((st & 1) != 0, np.asarray(counts) < ref["n_mismatch"])
+    v.close()
+
+
+def test_stochastic_acceptance():
+    cfg = _small(B=32, K=6, seed=9, stochastic=True)
+    case = cases.make_case(cfg, oracle_ref_argmax)
+    # spread alpha = min(1, p/q) over (0, 1]: q = p_T(y) * U(0.5, 4)
+    base = run_oracle(case)
+    g = np.random.default_rng(1)
+    case["draft_q"] = (base["p_draft"] * g.uniform(0.5, 4.0, size=case["T"])).astype(np.float32)
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d)
+    for tau in (0.0, 0.5):
+        out = cases.run(v, d, tau=tau)
+        ref = run_oracle(case, tau=tau)
+        st = compare(case, ref, out, tau)
+        assert st["tainted_requests"] < cfg.B
+    v.close()
+
+
+def test_bad_token_ids_are_clamped_and_flagged():
+    cfg = _small(B=4, K=4, seed=11)
+    case = cases.make_case(cfg, oracle_ref_argmax)
+    case["draft_tokens"] = case["draft_tokens"].copy()
+    case["draft_tokens"][1] = cfg.V + 5
+    case["draft_tokens"][9] = -3
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d)
+    out = cases.run(v, d)
+    st = out.status.cpu().numpy()
+    assert st[0] & 2 and st[2] & 2 and not (st[1] & 2) and not (st[3] & 2)
+    A = out.accept_len.cpu().numpy()
+    assert np.all(A >= 0) and np.all(A <= 4)
+    v.close()
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    cfg = _small(B=9, K=5, seed=13)
+    case = cases.make_case(cfg, oracle_ref_argmax)
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d)
+    out = cases.run(v, d)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    ho = v.verify_host(pin(case["target_hidden"]), pin(case["draft_tokens"]), pin(case["draft_hidden"]),
+                       pin(case["csi"]), B=cfg.B, K=cfg.K, extras=True)
+    for k in ("accept_len", "correction_token", "argmax", "lse", "p_draft", "head_prob", "n_mismatch", "status"):
+        assert torch.equal(getattr(ho, k), getattr(out, k).cpu()), k
+    v.close()
+
+
+def test_capacity_and_argument_errors():
+    cfg = _small(B=4, K=4)
+    case = cases.make_case(cfg, oracle_ref_argmax)
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d)
+    from paper_2604_17701_b200 import WisvError
+    with pytest.raises(WisvError) as e:
+        v.verify(d["target_hidden"], d["draft_tokens"], d["draft_hidden"], d["csi"], B=5, K=4)
+    assert e.value.code == -4
+    with pytest.raises(WisvError) as e:
+        v.verify(d["target_hidden"], d["draft_tokens"], d["draft_hidden"], d["csi"], B=1, K=65)
+    assert e.value.code == -2
+    with pytest.raises(WisvError) as e:
+        v.verify(None, d["draft_tokens"], d["draft_hidden"], d["csi"], B=4, K=4)
+    assert e.value.code == -1
+    v.close()
+
+
+# ------------------------------------------------------------------ 8B shapes
+
+def _lib_ref(lm_head_bits, target_hidden):
+    return cases.library_ref_argmax(lm_head_bits, target_hidden, device=DEV)
+
+
+def _subset_case(case, reqs):
+    """The same traffic restricted to a few whole requests (requests are independent)."""
+    cfg = case["cfg"]
+    k_len = case["k_len"][reqs]
+    tok_idx = np.concatenate([np.arange(case["k_off"][b], case["k_off"][b + 1]) for b in reqs]).astype(np.int64)
+    row_idx = np.concatenate([np.arange(case["row_off"][b], case["row_off"][b + 1]) for b in reqs]).astype(np.int64)
+    k_off, row_off = gen.row_offsets(k_len)
+    sub = dict(case)
+    sub.update(cfg=cfg.with_(B=len(reqs)), k_len=k_len, k_off=k_off, row_off=row_off, T=int(k_off[-1]),
+               R=int(row_off[-1]), target_hidden=case["target_hidden"][row_idx],
+               draft_tokens=case["draft_tokens"][tok_idx], csi=case["csi"][reqs])
+    if case["sel_off"] is not None:
+        sel_idx = np.concatenate([np.arange(case["sel_off"][b], case["sel_off"][b + 1]) for b in reqs]).astype(np.int64)
+        cnt = np.array([case["sel_off"][b + 1] - case["sel_off"][b] for b in reqs])
+        sub.update(sel_off=np.concatenate([[0], np.cumsum(cnt)]).astype(np.int32), sel_pos=case["sel_pos"][sel_idx],
+                   draft_hidden=case["draft_hidden"][sel_idx])
+        ev_idx = sel_idx
+    else:
+        sub.update(draft_hidden=case["draft_hidden"][tok_idx])
+        ev_idx = tok_idx
+    for k in ("draft_q", "uniforms"):
+        if case[k] is not None:
+            sub[k] = case[k][tok_idx]
+    return sub, row_idx, tok_idx, ev_idx
+
+
+class _Sub:
+    pass
+
+
+def _subset_output(out, reqs, row_idx, tok_idx, ev_idx):
+    s = _Sub()
+    r, t, e, q = (torch.as_tensor(x, device=out.accept_len.device) for x in (row_idx, tok_idx, ev_idx, np.asarray(reqs)))
+    s.accept_len, s.correction_token = out.accept_len[q], out.correction_token[q]
+    s.n_mismatch, s.mismatch_mask, s.status = out.n_mismatch[q], out.mismatch_mask[q], out.status[q]
+    s.argmax, s.lse, s.p_draft, s.head_prob = out.argmax[r], out.lse[r], out.p_draft[t], out.head_prob[e]
+    return s
+
+
+def _check_properties(case, out):
+    """Properties that hold at any size, checked on the full batch."""
+    k_len, k_off, row_off = case["k_len"], case["k_off"], case["row_off"]
+    A = out.accept_len.cpu().numpy()
+    corr = out.correction_token.cpu().numpy()
+    am = out.argmax.cpu().numpy()
+    assert np.all(A >= 0) and np.all(A <= k_len)
+    assert np.array_equal(corr, am[row_off[:-1] + A])              # correction / bonus = argmax of row A
+    assert np.all(np.isfinite(out.lse.cpu().numpy()))
+    assert np.all(out.status.cpu().numpy() & ~1 == 0)
+    if case["draft_q"] is None:
+        rows = np.repeat(row_off[:-1], k_len) + (np.arange(case["T"]) - np.repeat(k_off[:-1], k_len))
+        mism = case["draft_tokens"] != am[rows]
+        first = np.array([next((i for i in range(k_len[b]) if mism[k_off[b] + i]), k_len[b]) for b in range(len(k_len))])
+        assert np.all(A >= first)                                   # the head only extends the greedy span
+        nm = out.n_mismatch.cpu().numpy()
+        cnt = np.add.reduceat(mism.astype(np.int32), k_off[:-1])
+        assert np.array_equal(nm, np.where(k_len > 0, cnt, 0))
+    return A
+
+
+def _sampled_parity(name, n_sample, seed_pick=0):
+    cfg = gen.config(name)
+    case = cases.make_case(cfg, _lib_ref, weights=_shared_weights(cfg))
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d)
+    out = cases.run(v, d)
+    torch.cuda.synchronize()
+    assert v.device_error() == 0
+    A = _check_properties(case, out)
+    B = cfg.B
+    if n_sample >= B:
+        reqs = list(range(B))
+    else:
+        # first, last, requests straddling 128-row tile boundaries, then a seeded random fill
+        picks = {0, B - 1}
+        for edge in range(128, case["R"], 128):
+            picks.add(int(np.searchsorted(case["row_off"], edge, side="right") - 1))
+            if len(picks) >= n_sample // 2:
+                break
+        rest = [b for b in np.random.default_rng(seed_pick).permutation(B) if b not in picks]
+        reqs = sorted(list(picks) + [int(b) for b in rest[:max(0, n_sample - len(picks))]])
+    sub, row_idx, tok_idx, ev_idx = _subset_case(case, reqs)
+    ref = run_oracle(sub)
+    stats = compare(sub, ref, _subset_output(out, reqs, row_idx, tok_idx, ev_idx), cfg.tau)
+    v.close()
+    return case, out, A, stats
+
+
+def test_8b_batch1_full_oracle():
+    _sampled_parity("8b_b1", 1)
+
+
+@pytest.mark.parametrize("name", ["8b_b64_m30", "8b_b64", "8b_b64_m95"])
+def test_8b_batch64_sampled(name):
+    case, out, A, stats = _sampled_parity(name, 6)
+    assert stats["tainted_requests"] < stats["requests"]
+
+
+def test_8b_selective_hidden_sampled():
+    case, out, A, stats = _sampled_parity("8b_sh256", 12)
+    assert stats["tainted_requests"] < stats["requests"]
+
+
+@pytest.mark.parametrize("name", ["8b_b512", "8b_b512_stoch"])
+def test_8b_batch512_sampled(name):
+    case, out, A, stats = _sampled_parity(name, 10)
+    if name == "8b_b512":
+        # i.i.d. per-position accept probability a = r' + (1 - r') P(p < tau): closed-form mean
+        k = 16
+        am = out.argmax.cpu().numpy()
+        rows = np.repeat(case["row_off"][:-1], case["k_len"]) + (np.arange(case["T"]) - np.repeat(case["k_off"][:-1], case["k_len"]))
+        mism = case["draft_tokens"] != am[rows]
+        hp = out.head_prob.cpu().numpy()
+        a = 1.0 - np.mean(mism & (hp >= 0.5))
+        expect = a * (1 - a ** k) / (1 - a)
+        var = np.var(A)
+        assert abs(A.mean() - expect) < 4 * np.sqrt(var / len(A)) + 0.05
