@@ -208,7 +208,7 @@ class Verifier:
         R = T + B
         P = int(sel_pos.shape[0]) if sel_pos is not None else T
         if out is None:
-            out = self._outputs(B, R, T, P, target_hidden.device, extras)
+            out = self._outputs(B, R, T, P, self.device, extras)
         b = self._batch(B=B, K=K, k_off=k_off, T=T, target_hidden=target_hidden, draft_tokens=draft_tokens,
                         draft_hidden=draft_hidden, csi=csi, sel_off=sel_off, sel_pos=sel_pos, draft_q=draft_q,
                         uniforms=uniforms, tau=tau)
