@@ -1,0 +1,389 @@
+#!/usr/bin/env python
+"""Throughput of the WISV edge-side verifier round on B200, next to its CPU oracle.
+
+  python bench.py --gpus N --steps K --warmup W [--workload NAME] [--impl reference]
+
+One step = one whole verification round (pack -> LM head -> decision head ->
+merge/scan) over one batch of seeded synthetic windows.  The default workload is
+the Llama-3-8B-shaped batch-1 verifier (B=1, K=8, H=4096, V=128256).  Prints one
+JSON line: verified draft tokens/s with inputs resident in HBM (`value`), the
+same through the host-buffer entry point with copies inside the timed region
+(`e2e`), the roofline of the dominant kernel (LM head) from CUDA events recorded
+by the library around that kernel, and the oracle timed on the host cores.
+With N > 1 (torchrun) every rank verifies its own batch on its own GPU (requests
+are independent: no data-path collective) and the job-wide rate is reported.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import gen  # noqa: E402
+
+METRIC = "verified draft tokens/s at 8B shape (B×K); % of HBM or bf16 TC roofline"
+UNIT = "draft tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return p, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons sampled while the timed regions run."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.Q,
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is not None:
+            self.p.terminate()
+            try:
+                self.p.wait(timeout=5)
+            except Exception:
+                self.p.kill()
+        try:
+            self.f.flush()
+            self.f.seek(0)
+            sm, mx, reasons = [], [], set()
+            names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+            for line in self.f.read().splitlines():
+                c = [x.strip() for x in line.split(",")]
+                if len(c) < 9:
+                    continue
+                try:
+                    sm.append(float(c[1]))
+                    mx.append(float(c[2]))
+                except ValueError:
+                    continue
+                for n, v in zip(names, c[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            if sm:
+                out = {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                       "samples": len(sm)}
+        finally:
+            self.f.close()
+            try:
+                os.unlink(self.f.name)
+            except OSError:
+                pass
+        return out
+
+
+def pick_requests(case, n):
+    """First, last and a seeded fill: a bounded sample of whole requests."""
+    B = case["cfg"].B
+    if n >= B:
+        return list(range(B))
+    picks = {0, B - 1}
+    rest = [int(b) for b in np.random.default_rng(0).permutation(B) if b not in picks]
+    return sorted(list(picks) + rest[:max(0, n - len(picks))])
+
+
+def subset_case(case, reqs):
+    cfg = case["cfg"]
+    k_len = case["k_len"][reqs]
+    tok = np.concatenate([np.arange(case["k_off"][b], case["k_off"][b + 1]) for b in reqs]).astype(np.int64)
+    row = np.concatenate([np.arange(case["row_off"][b], case["row_off"][b + 1]) for b in reqs]).astype(np.int64)
+    k_off, row_off = gen.row_offsets(k_len)
+    sub = dict(case)
+    sub.update(cfg=cfg.with_(B=len(reqs)), k_len=k_len, k_off=k_off, row_off=row_off, T=int(k_off[-1]),
+               R=int(row_off[-1]), target_hidden=case["target_hidden"][row], draft_tokens=case["draft_tokens"][tok],
+               csi=case["csi"][reqs])
+    if case["sel_off"] is not None:
+        sel = np.concatenate([np.arange(case["sel_off"][b], case["sel_off"][b + 1]) for b in reqs]).astype(np.int64)
+        cnt = [int(case["sel_off"][b + 1] - case["sel_off"][b]) for b in reqs]
+        sub.update(sel_off=np.concatenate([[0], np.cumsum(cnt)]).astype(np.int32), sel_pos=case["sel_pos"][sel],
+                   draft_hidden=case["draft_hidden"][sel])
+    else:
+        sub.update(draft_hidden=case["draft_hidden"][tok])
+    for k in ("draft_q", "uniforms"):
+        if case[k] is not None:
+            sub[k] = case[k][tok]
+    return sub
+
+
+def oracle_round(case):
+    """One verification round of the CPU oracle on a case (test infrastructure, timed as the baseline)."""
+    import oracle
+    cfg = case["cfg"]
+    act = {"relu": oracle.ACT_RELU, "gelu": oracle.ACT_GELU}[cfg.act]
+    return oracle.verify(lm_head_bits=case["lm_head"], W1_bits=case["W1"], b1=case["b1"], w2=case["w2"],
+                         b2=float(case["b2"]), act=act, tau=cfg.tau, k_len=case["k_len"],
+                         target_hidden=case["target_hidden"], draft_tokens=case["draft_tokens"],
+                         draft_hidden=case["draft_hidden"], csi=case["csi"], sel_off=case["sel_off"],
+                         sel_pos=case["sel_pos"], draft_q=case["draft_q"], uniforms=case["uniforms"])
+
+
+def oracle_sample_size(case, rows_budget):
+    """Requests whose window rows add up to about rows_budget."""
+    mean_rows = case["R"] / max(1, case["cfg"].B)
+    return max(1, min(case["cfg"].B, int(rows_budget / mean_rows)))
+
+
+def workload_config(name, rank=0):
+    cfg = gen.config(name)
+    return cfg.with_(seed=cfg.seed + 1000 * rank) if rank else cfg
+
+
+def config_block(cfg, case, extra=None):
+    d = {"workload": cfg.name, "B": cfg.B, "K": cfg.K if cfg.K_hi == 0 else "U{%d..%d}" % (cfg.K_lo, cfg.K_hi),
+         "H": cfg.H, "V": cfg.V, "H_d": cfg.H_d, "d_J": cfg.d_J, "d_c": cfg.d_c, "mode": cfg.mode,
+         "accept": "stochastic" if cfg.stochastic else "greedy", "act": cfg.act, "tau": cfg.tau,
+         "match_rate": cfg.match_rate, "window_rows": case["R"], "draft_tokens": case["T"],
+         "l2": "no flush: every step streams the 1.05 GB bf16 LM head, far larger than the 126 MB L2"}
+    if extra:
+        d.update(extra)
+    return d
+
+
+# ------------------------------------------------------------------------------------- reference arm
+
+def run_reference(args, rank, world):
+    """Time the CPU oracle as it stands on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    import oracle
+    from paper_2604_17701_b200 import cases
+    cfg = workload_config(args.workload)
+    try:
+        import torch
+        prep_dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+    except Exception:
+        prep_dev = "cpu"
+    # input preparation only (which draft tokens are forced to match); the timed work below is the CPU oracle
+    case = cases.make_case(cfg, lambda w, h: cases.library_ref_argmax(w, h, device=prep_dev))
+    n_req = oracle_sample_size(case, args.oracle_rows)
+    sub = subset_case(case, pick_requests(case, n_req))
+    for _ in range(args.warmup):
+        oracle_round(sub)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_round(sub)
+    dt = (time.perf_counter() - t0) / max(1, args.steps)
+    value = sub["T"] / dt
+    sample = "%d of %d requests (%d window rows, %d draft tokens) per step" % (n_req, cfg.B, sub["R"], sub["T"])
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_block(cfg, case, {"sampled_requests": n_req}),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------- CUDA arm
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+    import torch.distributed as dist
+    from paper_2604_17701_b200 import cases
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the verifier has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = "cuda:%d" % local_rank
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    cfg = workload_config(args.workload, rank)
+    case = cases.make_case(cfg, lambda w, h: cases.library_ref_argmax(w, h, device=dev))
+    d = cases.to_device(case, dev)
+    v = cases.make_verifier(d)
+    T, R = case["T"], case["R"]
+    P = T if case["sel_pos"] is None else int(case["sel_pos"].shape[0])
+    out = cases.run(v, d, extras=True)
+    torch.cuda.synchronize()
+    if v.device_error() != 0:
+        raise SystemExit("device reported a pipeline time-out")
+    plan = v.plan(R, P)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def max_over_ranks(x):
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    stream = torch.cuda.current_stream()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+
+    # ---- (1) device-resident inputs, K back-to-back rounds, CUDA events on the launching stream
+    fast_out = cases.run(v, d, extras=False)
+    for _ in range(args.warmup):
+        cases.run(v, d, extras=False, out=fast_out)
+    barrier()
+    n0 = v.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        cases.run(v, d, extras=False, out=fast_out)
+    e1.record(stream)
+    barrier()
+    launches = v.launch_count() - n0
+    ms_step = max_over_ranks(e0.elapsed_time(e1) / args.steps)
+
+    # ---- (2) the same rounds with the library's per-kernel events switched on (roofline of the LM head)
+    prof_steps = min(args.steps, 1000)
+    v.profile_enable(prof_steps)
+    for _ in range(prof_steps):
+        cases.run(v, d, extras=False, out=fast_out)
+    torch.cuda.synchronize()
+    stage_ms = [v.profile_read(s, prof_steps) for s in range(4)]
+    v.profile_enable(0)
+    lm_ms = max_over_ranks(float(np.mean(stage_ms[1])))
+    stage_mean = [float(np.mean(s)) if s else 0.0 for s in stage_ms]
+
+    # ---- (3) end to end through the host-buffer entry point: H2D + round + D2H + sync per step
+    pin = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    hc = {k: pin(case[k]) for k in ("target_hidden", "draft_tokens", "draft_hidden", "csi", "sel_off", "sel_pos",
+                                    "draft_q", "uniforms")}
+    hk = pin(case["k_off"]) if cfg.K_hi > 0 else None
+    hkw = dict(B=cfg.B, K=cfg.K if cfg.K_hi == 0 else 0, k_off=hk, T=T, sel_off=hc["sel_off"],
+               sel_pos=hc["sel_pos"], draft_q=hc["draft_q"], uniforms=hc["uniforms"], extras=False)
+    host_out = v.verify_host(hc["target_hidden"], hc["draft_tokens"], hc["draft_hidden"], hc["csi"], **hkw)
+    e2e_steps = max(3, min(args.steps, 500))
+    for _ in range(min(args.warmup, 10)):
+        v.verify_host(hc["target_hidden"], hc["draft_tokens"], hc["draft_hidden"], hc["csi"], out=host_out, **hkw)
+    barrier()
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        v.verify_host(hc["target_hidden"], hc["draft_tokens"], hc["draft_hidden"], hc["csi"], out=host_out, **hkw)
+    e1.record(stream)
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1) / e2e_steps)
+    h2d = sum(int(t.numel() * t.element_size()) for t in list(hc.values()) + [hk] if t is not None)
+    d2h = 2 * 4 * cfg.B
+    same = bool(torch.equal(host_out.accept_len, fast_out.accept_len.cpu()))
+
+    clocks = sampler.stop() if rank == 0 else None
+
+    if rank == 0:
+        peaks, peak_kind = load_peaks()
+        w_bytes = cfg.V * cfg.H * 2
+        flops = 2.0 * R * cfg.H * cfg.V
+        hbm_bound = R < 256
+        if hbm_bound:
+            achieved = w_bytes / (lm_ms * 1e-3) / 1e9
+            peak = float(peaks["hbm_gbs"])
+            roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                    "traffic": None}
+        else:
+            achieved = flops / (lm_ms * 1e-3) / 1e12
+            long_step = lm_ms > 50.0
+            peak = float(peaks["bf16_tflops_sustained" if long_step else "bf16_tflops"])
+            roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                    "traffic": None}
+        roof.update({"kernel": "gemm_rowreduce_kernel<LM head>", "kernel_ms": lm_ms, "peak_source": peak_kind,
+                     "algorithmic_bytes": w_bytes, "algorithmic_flops": flops,
+                     "stage_ms": {"pack": stage_mean[0], "lm_head": stage_mean[1], "decision_head": stage_mean[2],
+                                  "merge_scan": stage_mean[3]}})
+
+        line = {"metric": METRIC, "value": world * T / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": config_block(cfg, case, {"parallelism": "requests sharded, 1 batch per GPU", "plan": plan}),
+                "clocks": clocks, "gpu_launches": int(launches),
+                "e2e": {"value": world * T / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                        "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps,
+                        "matches_device_path": same},
+                "roofline": roof,
+                "accepted_tokens_per_s": world * float(fast_out.accept_len.sum().item()) / (ms_step * 1e-3),
+                "mean_accept_len": float(out.accept_len.float().mean().item())}
+
+        if world == 1 and not args.no_cpu_baseline:
+            import oracle
+            n_req = oracle_sample_size(case, args.oracle_rows)
+            reqs = pick_requests(case, n_req)
+            sub = subset_case(case, reqs)
+            t0 = time.perf_counter()
+            ref = oracle_round(sub)
+            dt = time.perf_counter() - t0
+            A = out.accept_len.cpu().numpy()[reqs]
+            line["cpu_baseline"] = {
+                "value": sub["T"] / dt, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+                "sample": "%d of %d requests (%d window rows, %d draft tokens), one oracle round, %.1f s"
+                          % (n_req, cfg.B, sub["R"], sub["T"], dt),
+                "accept_len_equal": int(np.sum(A == ref["accept_len"])), "requests_compared": len(reqs)}
+        print(json.dumps(line), flush=True)
+
+    v.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="8b_b1", choices=sorted(gen.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--oracle-rows", type=int, default=None,
+                    help="window rows of oracle work per baseline round (bounds its run time)")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1 and world != args.gpus:
+        raise SystemExit("--gpus must equal WORLD_SIZE under torchrun")
+    if args.impl == "reference":
+        args.steps = 3 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        args.oracle_rows = 64 if args.oracle_rows is None else args.oracle_rows
+        run_reference(args, rank, world)
+    else:
+        big = gen.config(args.workload).B >= 64
+        args.steps = (200 if big else 5000) if args.steps is None else args.steps
+        args.warmup = (5 if big else 50) if args.warmup is None else args.warmup
+        args.warmup = max(3, args.warmup)
+        args.oracle_rows = 160 if args.oracle_rows is None else args.oracle_rows
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()
