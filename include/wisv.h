@@ -202,6 +202,40 @@ int wisv_plan(const wisv_ctx* ctx, int32_t R, int32_t P, int32_t* lm_tile_n, int
  */
 int wisv_debug_logits(wisv_ctx* ctx, const float* target_hidden, int32_t R, float* logits_out, void* cuda_stream);
 
+/*
+ * LM-head reduction without any allocation (the paper has no counterpart: this
+ * entry point exists for deployment, not for the method).
+ *
+ * For callers that are not allowed to allocate device memory - a plug-in inside
+ * a serving process whose framework has reserved the whole GPU for its own pool,
+ * or a latency-critical loop that must stay out of the driver's allocator - and
+ * therefore cannot use wisv_create.  Computes, for R <= WISV_STATIC_MAX_ROWS rows,
+ *     argmax[r] = lowest v maximising  bf16(target_hidden[r]) . lm_head[v]
+ *     lse[r]    = log sum_v exp(that logit)
+ * with the same TMA + tcgen05 kernel as wisv_verify, keeping its scratch (the
+ * bf16 copy of the rows and the per-tile partials) in a fixed array of about
+ * 4 MiB that is part of the library image: every GPU that loads the library
+ * holds it until the process exits.
+ *
+ * lm_head: dev bf16 [V, H] row-major, 16-byte aligned; target_hidden: dev fp32
+ * [R, H], 16-byte aligned; argmax: dev int32 [R]; lse: dev fp32 [R].  Limits:
+ * R <= WISV_STATIC_MAX_ROWS, 64 <= H <= WISV_STATIC_MAX_H with H % 8 == 0,
+ * V <= WISV_STATIC_MAX_V; anything larger returns WISV_ECAPACITY and launches
+ * nothing.  The call only enqueues work on `cuda_stream`; it calls no cudaMalloc,
+ * cudaFree or other allocating routine.  The first call on each device looks up
+ * the array's device address and raises the kernel's shared-memory limit; make
+ * that first call outside any stream capture.  All calls on a device share the
+ * array, which keeps the previous call's contents (each call rewrites what it
+ * reads): calls that may overlap on the GPU race on it, so order them on one
+ * stream or with events.  If a bounded wait inside the kernel gives up, every
+ * argmax is -1 and every lse is NaN.
+ */
+#define WISV_STATIC_MAX_ROWS 128
+#define WISV_STATIC_MAX_H    8192
+#define WISV_STATIC_MAX_V    262144
+int wisv_lm_head_reduce_static(const void* lm_head, int32_t V, int32_t H, const float* target_hidden, int32_t R,
+                               int32_t* argmax, float* lse, void* cuda_stream);
+
 const char* wisv_strerror(int code);
 int wisv_version(void);
 

@@ -6,6 +6,6 @@ memory and the stream handle.  There is no CPU path; if the library is missing
 or the device is not a B200, calls fail loudly.
 """
 from .binding import (  # noqa: F401
-    WisvError, Verifier, VerifyOutput, load_library, exported_symbols,
+    WisvError, Verifier, VerifyOutput, load_library, exported_symbols, lm_head_reduce_static,
     ACT_RELU, ACT_GELU, MODE_FH, MODE_SH, ACCEPT_GREEDY, ACCEPT_STOCHASTIC,
 )

@@ -91,6 +91,8 @@ def load_library(build_if_missing: bool = False):
     lib.wisv_plan.argtypes = [P, C.c_int32, C.c_int32] + [C.POINTER(C.c_int32)] * 6
     lib.wisv_debug_logits.restype = C.c_int
     lib.wisv_debug_logits.argtypes = [P, P, C.c_int32, P, P]
+    lib.wisv_lm_head_reduce_static.restype = C.c_int
+    lib.wisv_lm_head_reduce_static.argtypes = [P, C.c_int32, C.c_int32, P, C.c_int32, P, P, P]
     _lib = lib
     return lib
 
@@ -271,3 +273,22 @@ class Verifier:
         n = C.c_int32(0)
         _check(self.lib.wisv_profile_read(self._h, stage, buf, cap, C.byref(n)), "wisv_profile_read")
         return [buf[i] for i in range(n.value)]
+
+
+def lm_head_reduce_static(lm_head, target_hidden, argmax, lse, stream=None):
+    """wisv_lm_head_reduce_static on torch CUDA tensors the caller has already allocated.
+
+    For callers that may not allocate device memory: nothing is allocated here
+    either - inputs and outputs are the caller's, the scratch lives in the library
+    image.  lm_head: bf16 [V, H]; target_hidden: fp32 [R, H]; argmax: int32 [R];
+    lse: fp32 [R].  Asynchronous on the current (or given) torch stream.
+    """
+    import torch
+    lib = load_library()
+    V, H = lm_head.shape
+    R = target_hidden.shape[0]
+    st = stream if stream is not None else torch.cuda.current_stream(lm_head.device)
+    with torch.cuda.device(lm_head.device):
+        _check(lib.wisv_lm_head_reduce_static(lm_head.data_ptr(), V, H, target_hidden.data_ptr(), R,
+                                              argmax.data_ptr(), lse.data_ptr(), C.c_void_p(st.cuda_stream)),
+               "wisv_lm_head_reduce_static")
