@@ -183,6 +183,16 @@ int wisv_device_error(wisv_ctx* ctx, void* cuda_stream, int32_t* flags);
 int wisv_profile_enable(wisv_ctx* ctx, int32_t n_calls);
 int wisv_profile_read(wisv_ctx* ctx, int32_t stage, float* ms, int32_t cap, int32_t* n_out);
 
+/*
+ * Override the launch plan (0 in a field = choose automatically): vocabulary rows
+ * per LM-head tile and decision-head columns per tile (multiples of 16, <= 256)
+ * and the depth of the shared-memory stage ring (>= 2; capped by what fits).
+ * NULL restores the automatic plan.  The partial buffers are sized for any legal
+ * setting; results do not depend on the plan beyond fp32 summation order.
+ */
+typedef struct { int32_t lm_tile_n, lm_stages, head_tile_n, head_stages; } wisv_tuning;
+int wisv_set_tuning(wisv_ctx* ctx, const wisv_tuning* tuning);
+
 /* Number of kernels this context has launched so far. */
 int64_t wisv_launch_count(const wisv_ctx* ctx);
 

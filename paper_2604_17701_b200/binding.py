@@ -48,6 +48,11 @@ class _Result(C.Structure):
                 ("mismatch_mask", C.c_void_p), ("n_mismatch", C.c_void_p), ("status", C.c_void_p)]
 
 
+class _Tuning(C.Structure):
+    _fields_ = [("lm_tile_n", C.c_int32), ("lm_stages", C.c_int32), ("head_tile_n", C.c_int32),
+                ("head_stages", C.c_int32)]
+
+
 def exported_symbols() -> List[str]:
     """Function names declared in include/wisv.h."""
     text = open(_HEADER).read()
@@ -91,6 +96,8 @@ def load_library(build_if_missing: bool = False):
     lib.wisv_plan.argtypes = [P, C.c_int32, C.c_int32] + [C.POINTER(C.c_int32)] * 6
     lib.wisv_debug_logits.restype = C.c_int
     lib.wisv_debug_logits.argtypes = [P, P, C.c_int32, P, P]
+    lib.wisv_set_tuning.restype = C.c_int
+    lib.wisv_set_tuning.argtypes = [P, C.POINTER(_Tuning)]
     lib.wisv_lm_head_reduce_static.restype = C.c_int
     lib.wisv_lm_head_reduce_static.argtypes = [P, C.c_int32, C.c_int32, P, C.c_int32, P, P, P]
     _lib = lib
@@ -261,6 +268,10 @@ class Verifier:
         _check(self.lib.wisv_plan(self._h, R, P, *[C.byref(x) for x in v]), "wisv_plan")
         keys = ("lm_tile_n", "lm_tiles", "lm_ctas", "head_tile_n", "head_tiles", "head_ctas")
         return dict(zip(keys, (x.value for x in v)))
+
+    def set_tuning(self, lm_tile_n: int = 0, lm_stages: int = 0, head_tile_n: int = 0, head_stages: int = 0):
+        t = _Tuning(lm_tile_n, lm_stages, head_tile_n, head_stages)
+        _check(self.lib.wisv_set_tuning(self._h, C.byref(t)), "wisv_set_tuning")
 
     def launch_count(self) -> int:
         return int(self.lib.wisv_launch_count(self._h))

@@ -25,10 +25,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 constexpr int kNumTileVariants = kMaxTileN / 16;   // tile_n = 16, 32, ..., 256
+constexpr int kNumRowVariants = kTileM / 8;        // a_rows = 8, 16, ..., 128
 constexpr int kStages = 4;                         // profiled stages per call
 
 struct Plan {
     int tile_n, m_tiles, n_tiles, ctas, stages;
+    int a_rows;      // activation rows loaded per tile (8..128)
+    int carry;       // one partial per (row, CTA) instead of per (row, N-tile)
+    int parts;       // partials per row
     size_t smem;
 };
 
@@ -66,7 +70,7 @@ struct wisv_ctx {
     int32_t* pos_req = nullptr; int32_t* pos_i = nullptr;
     int32_t* err = nullptr;
     // TMA descriptors
-    CUtensorMap tmX, tmZ;
+    CUtensorMap tmX[kNumRowVariants], tmZ[kNumRowVariants];   // box heights 8, 16, ..., 128 rows
     CUtensorMap tmW[kNumTileVariants];
     CUtensorMap tmW1[kNumTileVariants];
     // profiling
@@ -74,6 +78,7 @@ struct wisv_ctx {
     long long prof_calls = 0;
     cudaEvent_t* prof_ev = nullptr;   // [prof_n][kStages + 1]
     long long launches = 0;
+    wisv_tuning tune = {0, 0, 0, 0};
     HostStaging hs;
 };
 
@@ -100,18 +105,26 @@ int encode_2d(EncodeTiledFn fn, CUtensorMap* out, const void* base, uint64_t inn
 
 int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
-size_t gemm_smem_bytes(int tile_n, int stages, int d_c)
+size_t gemm_fixed_bytes(int tile_n, int a_rows, int d_c)
 {
-    return 1024 + (size_t)stages * gemm_stage_bytes(tile_n) + gemm_tail_bytes(tile_n, d_c);
+    return 1024 + gemm_tail_bytes(tile_n, d_c) + gemm_overread_bytes(a_rows);
 }
 
-int stages_for(const wisv_ctx* c, int tile_n, int d_c, int k_blocks)
+// stage count, tile geometry -> shared memory; fills stages / smem of the plan
+void finish_plan(const wisv_ctx* c, Plan* p, int d_c, int k_blocks, int forced_stages)
 {
-    const size_t fixed = 1024 + gemm_tail_bytes(tile_n, d_c);
-    int s = (int)(((size_t)c->max_smem - fixed) / gemm_stage_bytes(tile_n));
+    const size_t fixed = gemm_fixed_bytes(p->tile_n, p->a_rows, d_c);
+    const size_t stage = gemm_stage_bytes(p->tile_n, p->a_rows);
+    int s = (int)(((size_t)c->max_smem - fixed) / stage);
     if (s > kMaxStages) s = kMaxStages;
-    (void)k_blocks;
-    return s;
+    if (s > k_blocks * 4 && k_blocks > 0) s = k_blocks * 4 > 2 ? k_blocks * 4 : 2;
+    if (forced_stages >= 2 && forced_stages < s) s = forced_stages;
+    p->stages = s;
+    p->smem = fixed + (size_t)s * stage;
+    const long long tiles = (long long)p->m_tiles * p->n_tiles;
+    p->ctas = (int)(tiles < c->sm_count ? tiles : c->sm_count);
+    p->carry = p->m_tiles == 1 ? 1 : 0;
+    p->parts = p->carry ? p->ctas : p->n_tiles;
 }
 
 double wave_eff(long long tiles, int sms)
@@ -129,23 +142,25 @@ Plan plan_lm(const wisv_ctx* c, int R)
     const int V = c->cfg.V;
     p.m_tiles = (R + kTileM - 1) / kTileM;
     int best = 0;
-    if (p.m_tiles == 1) {
+    if (c->tune.lm_tile_n >= 16 && c->tune.lm_tile_n <= kMaxTileN && c->tune.lm_tile_n % 16 == 0) {
+        best = c->tune.lm_tile_n;
+    } else if (p.m_tiles == 1) {
+        // largest tile whose wave efficiency is within half a percent of the best
         double best_eff = -1.0;
         for (int tn = 64; tn <= kMaxTileN; tn += 16) {
-            const long long tiles = (V + tn - 1) / tn;
-            const double e = wave_eff(tiles, c->sm_count);
-            if (e >= best_eff - 1e-9) { best_eff = e > best_eff ? e : best_eff; best = tn; }
+            const double e = wave_eff((V + tn - 1) / tn, c->sm_count);
+            if (e > best_eff) best_eff = e;
         }
+        for (int tn = 64; tn <= kMaxTileN; tn += 16)
+            if (wave_eff((V + tn - 1) / tn, c->sm_count) >= best_eff - 0.005) best = tn;
     } else {
-        best = V >= kMaxTileN ? kMaxTileN : round_up(V, 16);
+        best = kMaxTileN;
     }
     if (best > round_up(V, 16)) best = round_up(V, 16);
     p.tile_n = best;
     p.n_tiles = (V + best - 1) / best;
-    const long long tiles = (long long)p.m_tiles * p.n_tiles;
-    p.ctas = (int)(tiles < c->sm_count ? tiles : c->sm_count);
-    p.stages = stages_for(c, best, 0, 0);
-    p.smem = gemm_smem_bytes(best, p.stages, 0);
+    p.a_rows = p.m_tiles == 1 ? round_up(R, 8) : kTileM;
+    finish_plan(c, &p, 0, (c->cfg.H + kBlockK - 1) / kBlockK, c->tune.lm_stages);
     return p;
 }
 
@@ -155,8 +170,10 @@ Plan plan_head(const wisv_ctx* c, int P)
     const int N = c->cfg.d_J;
     p.m_tiles = (P + kTileM - 1) / kTileM;
     int best = 16;
-    if (p.m_tiles >= 8) {
-        best = N >= kMaxTileN ? kMaxTileN : round_up(N, 16);
+    if (c->tune.head_tile_n >= 16 && c->tune.head_tile_n <= kMaxTileN && c->tune.head_tile_n % 16 == 0) {
+        best = c->tune.head_tile_n;
+    } else if (p.m_tiles >= 8) {
+        best = kMaxTileN;
     } else {
         double best_eff = -1.0;
         for (int tn = 16; tn <= kMaxTileN; tn *= 2) {
@@ -168,10 +185,8 @@ Plan plan_head(const wisv_ctx* c, int P)
     if (best > round_up(N, 16)) best = round_up(N, 16);
     p.tile_n = best;
     p.n_tiles = (N + best - 1) / best;
-    const long long tiles = (long long)p.m_tiles * p.n_tiles;
-    p.ctas = (int)(tiles < c->sm_count ? tiles : c->sm_count);
-    p.stages = stages_for(c, best, c->cfg.d_c, 0);
-    p.smem = gemm_smem_bytes(best, p.stages, c->cfg.d_c);
+    p.a_rows = p.m_tiles == 1 ? round_up(P, 8) : kTileM;
+    finish_plan(c, &p, c->cfg.d_c, (c->cfg.H_d + c->cfg.H + kBlockK - 1) / kBlockK, c->tune.head_stages);
     return p;
 }
 
@@ -257,6 +272,7 @@ GemmParams base_params(const wisv_ctx* c, const Plan& pl, int rows, int n_total,
     memset(&gp, 0, sizeof gp);
     gp.rows = rows; gp.n_total = n_total; gp.k_blocks = (kdim + kBlockK - 1) / kBlockK;
     gp.tile_n = pl.tile_n; gp.m_tiles = pl.m_tiles; gp.n_tiles = pl.n_tiles; gp.stages = pl.stages;
+    gp.a_rows = pl.a_rows; gp.carry = pl.carry; gp.part_stride = pl.parts;
     gp.err = c->err;
     return gp;
 }
@@ -335,14 +351,11 @@ int wisv_create(const wisv_config* cfg, const wisv_weights* w, wisv_ctx** out)
     size_t lm_elems = 0, head_elems = 0;
     {
         const int r1 = cfg->max_rows < kTileM ? cfg->max_rows : kTileM;
-        Plan a = plan_lm(c, r1);
-        lm_elems = (size_t)r1 * a.n_tiles;
-        // the single-tile plan may pick any tile height >= 64
-        const size_t worst1 = (size_t)r1 * ((cfg->V + 63) / 64);
-        if (worst1 > lm_elems) lm_elems = worst1;
+        // one row tile: at most one partial per (row, CTA), or per 16-row vocabulary tile when tuned
+        lm_elems = (size_t)r1 * ((cfg->V + 15) / 16 < c->sm_count ? (cfg->V + 15) / 16 : c->sm_count);
         if (cfg->max_rows > kTileM) {
             Plan b = plan_lm(c, cfg->max_rows);
-            const size_t e = (size_t)cfg->max_rows * b.n_tiles;
+            const size_t e = (size_t)cfg->max_rows * b.n_tiles;   // automatic plan; a finer tuned tile is refused
             if (e > lm_elems) lm_elems = e;
         }
         head_elems = (size_t)c->max_pos * ((cfg->d_J + 15) / 16);
@@ -373,8 +386,13 @@ int wisv_create(const wisv_config* cfg, const wisv_weights* w, wisv_ctx** out)
         if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) { rc = WISV_ECUDA; break; }
         c->launches++;
 
-        if ((rc = encode_2d(encode, &c->tmX, c->X, (uint64_t)cfg->H, (uint64_t)c->rows_alloc, kBlockK, kTileM))) break;
-        if ((rc = encode_2d(encode, &c->tmZ, c->Z, (uint64_t)hd_h, (uint64_t)c->pos_alloc, kBlockK, kTileM))) break;
+        for (int i = 0; i < kNumRowVariants && rc == WISV_OK; ++i) {
+            const uint32_t rows = 8u * (i + 1);
+            rc = encode_2d(encode, &c->tmX[i], c->X, (uint64_t)cfg->H, (uint64_t)c->rows_alloc, kBlockK, rows);
+            if (rc == WISV_OK)
+                rc = encode_2d(encode, &c->tmZ[i], c->Z, (uint64_t)hd_h, (uint64_t)c->pos_alloc, kBlockK, rows);
+        }
+        if (rc != WISV_OK) break;
         for (int i = 0; i < kNumTileVariants && rc == WISV_OK; ++i) {
             const uint32_t tn = 16u * (i + 1);
             rc = encode_2d(encode, &c->tmW[i], w->lm_head, (uint64_t)cfg->H, (uint64_t)cfg->V, kBlockK, tn);
@@ -411,6 +429,18 @@ int wisv_plan(const wisv_ctx* c, int32_t R, int32_t P, int32_t* lm_tile_n, int32
 
 int64_t wisv_launch_count(const wisv_ctx* c) { return c ? c->launches : 0; }
 
+int wisv_set_tuning(wisv_ctx* c, const wisv_tuning* t)
+{
+    if (!c) return WISV_EINVAL;
+    if (!t) { c->tune = wisv_tuning{0, 0, 0, 0}; return WISV_OK; }
+    const int32_t tn[2] = {t->lm_tile_n, t->head_tile_n};
+    for (int i = 0; i < 2; ++i)
+        if (tn[i] != 0 && (tn[i] < 16 || tn[i] > kMaxTileN || tn[i] % 16)) return WISV_ESHAPE;
+    if (t->lm_stages < 0 || t->head_stages < 0 || t->lm_stages == 1 || t->head_stages == 1) return WISV_ESHAPE;
+    c->tune = *t;
+    return WISV_OK;
+}
+
 int wisv_verify(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda_stream)
 {
     int T = 0, R = 0, P = 0;
@@ -444,11 +474,11 @@ int wisv_verify(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cu
     // ---- 2. LM head: logits reduced on the fly
     if (ev) WISV_CUDA(cudaEventRecord(ev[1], st));
     const Plan pl = plan_lm(c, R);
-    if ((size_t)R * pl.n_tiles > c->lm_part_elems) return WISV_ECAPACITY;
+    if ((size_t)R * pl.parts > c->lm_part_elems) return WISV_ECAPACITY;
     {
         GemmParams gp = base_params(c, pl, R, cf.V, cf.H);
         gp.lm_part = c->lm_part; gp.row_tok = c->row_tok; gp.tok_logit = c->tok_logit;
-        const int rc = launch_gemm<EPI_LMHEAD>(c, c->tmX, c->tmW[pl.tile_n / 16 - 1], gp, pl, st);
+        const int rc = launch_gemm<EPI_LMHEAD>(c, c->tmX[pl.a_rows / 8 - 1], c->tmW[pl.tile_n / 16 - 1], gp, pl, st);
         if (rc != WISV_OK) return rc;
     }
 
@@ -457,11 +487,11 @@ int wisv_verify(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cu
     Plan ph{};
     if (P > 0) {
         ph = plan_head(c, P);
-        if ((size_t)P * ph.n_tiles > c->head_part_elems) return WISV_ECAPACITY;
+        if ((size_t)P * ph.parts > c->head_part_elems) return WISV_ECAPACITY;
         GemmParams gp = base_params(c, ph, P, cf.d_J, cf.H_d + cf.H);
         gp.head_part = c->head_part; gp.b1 = c->w.b1; gp.w2 = c->w.w2; gp.w1c = c->W1c; gp.csi = b->csi;
         gp.pos_req = c->pos_req; gp.d_c = cf.d_c; gp.act = cf.act;
-        const int rc = launch_gemm<EPI_HEAD>(c, c->tmZ, c->tmW1[ph.tile_n / 16 - 1], gp, ph, st);
+        const int rc = launch_gemm<EPI_HEAD>(c, c->tmZ[ph.a_rows / 8 - 1], c->tmW1[ph.tile_n / 16 - 1], gp, ph, st);
         if (rc != WISV_OK) return rc;
     }
 
@@ -469,7 +499,7 @@ int wisv_verify(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cu
     if (ev) WISV_CUDA(cudaEventRecord(ev[3], st));
     TailParams tp;
     memset(&tp, 0, sizeof tp);
-    tp.ix = ix; tp.P = P; tp.V = cf.V; tp.n_tiles_lm = pl.n_tiles; tp.n_tiles_head = ph.n_tiles; tp.mode_sh = sh ? 1 : 0;
+    tp.ix = ix; tp.P = P; tp.V = cf.V; tp.n_tiles_lm = pl.parts; tp.n_tiles_head = ph.parts; tp.mode_sh = sh ? 1 : 0;
     tp.stochastic = stoch ? 1 : 0; tp.b2 = c->w.b2; tp.tau = (b->tau != b->tau) ? cf.tau : b->tau;
     tp.lm_part = c->lm_part; tp.tok_logit = c->tok_logit; tp.row_flag = c->row_flag; tp.draft_tokens = b->draft_tokens;
     tp.head_part = c->head_part; tp.pos_i = c->pos_i; tp.sel_off = b->sel_off; tp.draft_q = b->draft_q;
@@ -502,7 +532,7 @@ int wisv_debug_logits(wisv_ctx* c, const float* target_hidden, int32_t R, float*
     const Plan pl = plan_lm(c, R);
     GemmParams gp = base_params(c, pl, R, c->cfg.V, c->cfg.H);
     gp.raw_out = logits_out;
-    return launch_gemm<EPI_RAW>(c, c->tmX, c->tmW[pl.tile_n / 16 - 1], gp, pl, st);
+    return launch_gemm<EPI_RAW>(c, c->tmX[pl.a_rows / 8 - 1], c->tmW[pl.tile_n / 16 - 1], gp, pl, st);
 }
 
 int wisv_device_error(wisv_ctx* c, void* cuda_stream, int32_t* flags)

@@ -178,7 +178,16 @@ __global__ void __launch_bounds__(256) tail_kernel(const TailParams p)
         const int r = r0 + i;
         RowStat st{-CUDART_INF_F, 0x7fffffff, 0.0f};
         const float4* part = p.lm_part + (size_t)r * p.n_tiles_lm;
-        for (int n = lane; n < p.n_tiles_lm; n += 32) {
+        // four independent loads in flight per lane before the dependent merges
+        int n = lane;
+        for (; n + 96 < p.n_tiles_lm; n += 128) {
+            const float4 v0 = part[n], v1 = part[n + 32], v2 = part[n + 64], v3 = part[n + 96];
+            merge_stat(st, v0.x, __float_as_int(v0.y), v0.z);
+            merge_stat(st, v1.x, __float_as_int(v1.y), v1.z);
+            merge_stat(st, v2.x, __float_as_int(v2.y), v2.z);
+            merge_stat(st, v3.x, __float_as_int(v3.y), v3.z);
+        }
+        for (; n < p.n_tiles_lm; n += 32) {
             const float4 v = part[n];
             merge_stat(st, v.x, __float_as_int(v.y), v.z);
         }

@@ -31,7 +31,7 @@ constexpr int kAccCols = 256;        // TMEM columns per accumulator stage
 constexpr int kTmemCols = 512;
 constexpr int kGemmThreads = 192;
 constexpr int kEpiThreads = 128;
-constexpr int kMaxStages = 12;
+constexpr int kMaxStages = 32;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s
 constexpr int kMaxDc = 16;
 
@@ -44,13 +44,19 @@ struct GemmParams {
     int32_t tile_n;      // Bw rows per tile: multiple of 16, <= 256
     int32_t m_tiles, n_tiles;
     int32_t stages;
+    int32_t a_rows;      // rows of A actually loaded per tile (multiple of 8, <= 128); the MMA still spans
+                         // 128 rows, the rest of its A operand is whatever follows in shared memory and only
+                         // feeds accumulator rows that are never read
+    int32_t carry;       // 1: one row tile, each CTA keeps its running row state across its tiles and
+                         //    writes one partial per (row, CTA); 0: one partial per (row, N-tile)
+    int32_t part_stride; // partials per row (CTAs when carry, else n_tiles)
     int32_t* err;        // device error word (bit 0: a bounded wait gave up)
     // LM-head epilogue
-    float4* lm_part;          // [rows][n_tiles] = {max, bits(argidx), sumexp, 0}
+    float4* lm_part;          // [rows][part_stride] = {max, bits(argidx), sumexp, 0}
     const int32_t* row_tok;   // [rows] draft token of the row or -1
     float* tok_logit;         // [rows]
     // decision-head epilogue
-    float* head_part;         // [rows][n_tiles]
+    float* head_part;         // [rows][part_stride]
     const float* b1;          // [n_total]
     const float* w2;          // [n_total]
     const float* w1c;         // [n_total][d_c] fp32 CSI columns of W1
@@ -62,12 +68,16 @@ struct GemmParams {
     float* raw_out;           // [rows][n_total]
 };
 
-__host__ __device__ inline uint32_t gemm_stage_bytes(int tile_n) {
-    return static_cast<uint32_t>(kTileM * kBlockK * 2 + tile_n * kBlockK * 2);
+__host__ __device__ inline uint32_t gemm_stage_bytes(int tile_n, int a_rows = kTileM) {
+    return static_cast<uint32_t>(a_rows * kBlockK * 2 + tile_n * kBlockK * 2);
+}
+// bytes the MMA may read past the last stage's A slot when fewer than 128 rows are loaded
+__host__ __device__ inline uint32_t gemm_overread_bytes(int a_rows) {
+    return static_cast<uint32_t>((kTileM - a_rows) * kBlockK * 2);
 }
 // bytes after the stage ring: barriers + tmem slot + abort flag, then epilogue constants
 __host__ __device__ inline uint32_t gemm_tail_bytes(int tile_n, int d_c) {
-    return 512u + 2u * (static_cast<uint32_t>(tile_n) * static_cast<uint32_t>(2 + d_c) +
+    return 1024u + 2u * (static_cast<uint32_t>(tile_n) * static_cast<uint32_t>(2 + d_c) +
                         static_cast<uint32_t>(kEpiThreads * d_c)) * 4u;
 }
 
@@ -87,7 +97,7 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     uint8_t* smem = smem_raw + pad;                       // 1024-byte aligned: swizzle atoms need it
     const uint32_t smem_base = raw_addr + pad;
 
-    const uint32_t a_bytes = kTileM * kBlockK * 2;
+    const uint32_t a_bytes = static_cast<uint32_t>(p.a_rows) * kBlockK * 2;
     const uint32_t b_bytes = static_cast<uint32_t>(p.tile_n) * kBlockK * 2;
     const uint32_t stage_bytes = a_bytes + b_bytes;
     const uint32_t ring_bytes = stage_bytes * static_cast<uint32_t>(p.stages);
@@ -101,7 +111,7 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     const uint32_t drain_bar = bar_base + 8u * (2 * kMaxStages + 4);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + ring_bytes + 8 * (2 * kMaxStages + 5));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [0] abort, [1] drain scratch
-    float* epi_const = reinterpret_cast<float*>(smem + ring_bytes + 512);
+    float* epi_const = reinterpret_cast<float*>(smem + ring_bytes + 1024);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -198,6 +208,8 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         const int et = threadIdx.x - 64;                   // 0..127 among epilogue threads
         int local = 0;
         bool ok = true;
+        float mx = -CUDART_INF_F, sum = 0.0f, hs = 0.0f;   // running row state (per tile, or per CTA when carry)
+        int arg = 0;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++local) {
             const int m = t % p.m_tiles, n = t / p.m_tiles;
             const int as = local & 1;
@@ -245,8 +257,7 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             if (!got) { ok = false; break; }
             tc_fence_after();
 
-            float mx = -CUDART_INF_F, sum = 0.0f, hs = 0.0f;
-            int arg = 0;
+            if (!p.carry) { mx = -CUDART_INF_F; sum = 0.0f; hs = 0.0f; arg = 0; }
             const int tok = (EPI == EPI_LMHEAD && valid) ? p.row_tok[row] : -1;
 
             for (int c0 = 0; c0 < p.tile_n; c0 += 16) {
@@ -302,11 +313,22 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty_bar(as));
 
-            if (valid) {
+            if (valid && !p.carry) {
                 if (EPI == EPI_LMHEAD)
-                    p.lm_part[(size_t)row * p.n_tiles + n] = make_float4(mx, __int_as_float(arg), sum, 0.0f);
+                    p.lm_part[(size_t)row * p.part_stride + n] = make_float4(mx, __int_as_float(arg), sum, 0.0f);
                 else if (EPI == EPI_HEAD)
-                    p.head_part[(size_t)row * p.n_tiles + n] = hs;
+                    p.head_part[(size_t)row * p.part_stride + n] = hs;
+            }
+        }
+        if (p.carry && ok) {
+            // one row tile: tiles of this CTA ascend through the vocabulary, so the strict '>' above
+            // already kept the lowest index; a CTA without tiles is never launched
+            const int row = q * 32 + lane;
+            if (row < p.rows) {
+                if (EPI == EPI_LMHEAD)
+                    p.lm_part[(size_t)row * p.part_stride + blockIdx.x] = make_float4(mx, __int_as_float(arg), sum, 0.0f);
+                else if (EPI == EPI_HEAD)
+                    p.head_part[(size_t)row * p.part_stride + blockIdx.x] = hs;
             }
         }
     }
