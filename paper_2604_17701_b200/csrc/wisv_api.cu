@@ -27,12 +27,15 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 constexpr int kNumTileVariants = kMaxTileN / 16;   // tile_n = 16, 32, ..., 256
 constexpr int kNumRowVariants = kTileM / 8;        // a_rows = 8, 16, ..., 128
 constexpr int kStages = 4;                         // profiled stages per call
+constexpr int kSplitTileN = 64;                    // head tile height when K is split over CTAs
 
 struct Plan {
     int tile_n, m_tiles, n_tiles, ctas, stages;
     int a_rows;      // activation rows loaded per tile (8..128)
     int carry;       // one partial per (row, CTA) instead of per (row, N-tile)
     int parts;       // partials per row
+    int k_splits;    // work items per (m, n) tile along K (decision head with one row tile)
+    int kb_per_split;
     size_t smem;
 };
 
@@ -66,6 +69,9 @@ struct wisv_ctx {
     size_t lm_part_elems = 0;
     float* head_part = nullptr;
     size_t head_part_elems = 0;
+    float* splitk_buf = nullptr;      // [sm_count][128][kSplitTileN] raw partial head tiles
+    int32_t* splitk_count = nullptr;  // per (m, n) tile arrival counters, zero between calls
+    int splitk_tiles = 0;
     int32_t* row_tok = nullptr; int32_t* row_flag = nullptr; float* tok_logit = nullptr;
     int32_t* pos_req = nullptr; int32_t* pos_i = nullptr;
     int32_t* err = nullptr;
@@ -121,9 +127,10 @@ void finish_plan(const wisv_ctx* c, Plan* p, int d_c, int k_blocks, int forced_s
     if (forced_stages >= 2 && forced_stages < s) s = forced_stages;
     p->stages = s;
     p->smem = fixed + (size_t)s * stage;
-    const long long tiles = (long long)p->m_tiles * p->n_tiles;
-    p->ctas = (int)(tiles < c->sm_count ? tiles : c->sm_count);
-    p->carry = p->m_tiles == 1 ? 1 : 0;
+    if (p->k_splits < 1) { p->k_splits = 1; p->kb_per_split = k_blocks; }
+    const long long items = (long long)p->m_tiles * p->n_tiles * p->k_splits;
+    p->ctas = (int)(items < c->sm_count ? items : c->sm_count);
+    p->carry = (p->m_tiles == 1 && p->k_splits == 1) ? 1 : 0;
     p->parts = p->carry ? p->ctas : p->n_tiles;
 }
 
@@ -170,8 +177,21 @@ Plan plan_head(const wisv_ctx* c, int P)
     const int N = c->cfg.d_J;
     p.m_tiles = (P + kTileM - 1) / kTileM;
     int best = 16;
+    const int k_blocks = (c->cfg.H_d + c->cfg.H + kBlockK - 1) / kBlockK;
     if (c->tune.head_tile_n >= 16 && c->tune.head_tile_n <= kMaxTileN && c->tune.head_tile_n % 16 == 0) {
         best = c->tune.head_tile_n;
+    } else if (p.m_tiles == 1) {
+        // one row tile: too few column tiles to fill the GPU and every CTA would walk all of K, so K is
+        // split as well: about one work item per SM, partial tiles combined by the last item to finish
+        best = kSplitTileN;
+        const int nt = (N + best - 1) / best;
+        int splits = c->sm_count / nt;
+        if (splits > k_blocks) splits = k_blocks;
+        if (splits > kMaxKSplits) splits = kMaxKSplits;
+        if (splits > 1) {
+            p.kb_per_split = (k_blocks + splits - 1) / splits;
+            p.k_splits = (k_blocks + p.kb_per_split - 1) / p.kb_per_split;     // no empty split
+        }
     } else if (p.m_tiles >= 8) {
         best = kMaxTileN;
     } else {
@@ -186,7 +206,7 @@ Plan plan_head(const wisv_ctx* c, int P)
     p.tile_n = best;
     p.n_tiles = (N + best - 1) / best;
     p.a_rows = p.m_tiles == 1 ? round_up(P, 8) : kTileM;
-    finish_plan(c, &p, c->cfg.d_c, (c->cfg.H_d + c->cfg.H + kBlockK - 1) / kBlockK, c->tune.head_stages);
+    finish_plan(c, &p, c->cfg.d_c, k_blocks, c->tune.head_stages);
     return p;
 }
 
@@ -197,7 +217,7 @@ void free_ctx(wisv_ctx* c)
     if (!c) return;
     cudaFree(c->X); cudaFree(c->Z); cudaFree(c->W1p); cudaFree(c->W1c); cudaFree(c->lm_part);
     cudaFree(c->head_part); cudaFree(c->row_tok); cudaFree(c->row_flag); cudaFree(c->tok_logit);
-    cudaFree(c->pos_req); cudaFree(c->pos_i); cudaFree(c->err);
+    cudaFree(c->pos_req); cudaFree(c->pos_i); cudaFree(c->err); cudaFree(c->splitk_buf); cudaFree(c->splitk_count);
     if (c->prof_ev) {
         for (int i = 0; i < c->prof_n * (kStages + 1); ++i) cudaEventDestroy(c->prof_ev[i]);
         free(c->prof_ev);
@@ -273,6 +293,8 @@ GemmParams base_params(const wisv_ctx* c, const Plan& pl, int rows, int n_total,
     gp.rows = rows; gp.n_total = n_total; gp.k_blocks = (kdim + kBlockK - 1) / kBlockK;
     gp.tile_n = pl.tile_n; gp.m_tiles = pl.m_tiles; gp.n_tiles = pl.n_tiles; gp.stages = pl.stages;
     gp.a_rows = pl.a_rows; gp.carry = pl.carry; gp.part_stride = pl.parts;
+    gp.k_splits = pl.k_splits; gp.kb_per_split = pl.kb_per_split;
+    gp.splitk_buf = c->splitk_buf; gp.splitk_count = c->splitk_count;
     gp.err = c->err;
     return gp;
 }
@@ -377,6 +399,10 @@ int wisv_create(const wisv_config* cfg, const wisv_weights* w, wisv_ctx** out)
         if ((rc = dev_alloc(&c->pos_req, (size_t)c->pos_alloc))) break;
         if ((rc = dev_alloc(&c->pos_i, (size_t)c->pos_alloc))) break;
         if ((rc = dev_alloc(&c->err, 1))) break;
+        c->splitk_tiles = (cfg->d_J + 15) / 16;
+        if ((rc = dev_alloc(&c->splitk_buf, (size_t)c->sm_count * kTileM * kSplitTileN))) break;
+        if ((rc = dev_alloc(&c->splitk_count, (size_t)c->splitk_tiles))) break;
+        if (cudaMemset(c->splitk_count, 0, sizeof(int32_t) * c->splitk_tiles) != cudaSuccess) { rc = WISV_ECUDA; break; }
         if (cudaMemset(c->X, 0, (size_t)c->rows_alloc * cfg->H * 2) != cudaSuccess ||
             cudaMemset(c->Z, 0, (size_t)c->pos_alloc * hd_h * 2) != cudaSuccess ||
             cudaMemset(c->err, 0, sizeof(int32_t)) != cudaSuccess) { rc = WISV_ECUDA; break; }
@@ -542,7 +568,11 @@ int wisv_device_error(wisv_ctx* c, void* cuda_stream, int32_t* flags)
     WISV_CUDA(cudaStreamSynchronize(st));
     int32_t v = 0;
     WISV_CUDA(cudaMemcpy(&v, c->err, sizeof v, cudaMemcpyDeviceToHost));
-    if (v != 0) WISV_CUDA(cudaMemset(c->err, 0, sizeof v));
+    if (v != 0) {
+        // an aborted launch may have left split-K arrival counters half-way
+        WISV_CUDA(cudaMemset(c->err, 0, sizeof v));
+        WISV_CUDA(cudaMemset(c->splitk_count, 0, sizeof(int32_t) * c->splitk_tiles));
+    }
     *flags = v;
     return WISV_OK;
 }

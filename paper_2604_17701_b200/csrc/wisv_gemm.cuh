@@ -32,8 +32,9 @@ constexpr int kTmemCols = 512;
 constexpr int kGemmThreads = 192;
 constexpr int kEpiThreads = 128;
 constexpr int kMaxStages = 32;
-constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s
+constexpr uint64_t kWaitLimitNs = 4000000000ull;   // SM clocks: 2 s at 2 GHz, 3.3 s at 1.2 GHz
 constexpr int kMaxDc = 16;
+constexpr int kMaxKSplits = 16;      // split-K work items per tile (their partial loads are issued together)
 
 enum { EPI_LMHEAD = 0, EPI_HEAD = 1, EPI_RAW = 2 };
 
@@ -50,6 +51,12 @@ struct GemmParams {
     int32_t carry;       // 1: one row tile, each CTA keeps its running row state across its tiles and
                          //    writes one partial per (row, CTA); 0: one partial per (row, N-tile)
     int32_t part_stride; // partials per row (CTAs when carry, else n_tiles)
+    int32_t k_splits;    // decision head only: the K range is cut into k_splits work items per (m, n) tile;
+                         // each item stores its raw fp32 tile, the last one to finish adds them up in
+                         // split order and applies the epilogue (no CTA ever waits for another)
+    int32_t kb_per_split;
+    float* splitk_buf;        // [items][128][tile_n] raw partial pre-activations
+    int32_t* splitk_count;    // [m_tiles * n_tiles], zero between calls (the last item resets it)
     int32_t* err;        // device error word (bit 0: a bounded wait gave up)
     // LM-head epilogue
     float4* lm_part;          // [rows][part_stride] = {max, bits(argidx), sumexp, 0}
@@ -77,7 +84,7 @@ __host__ __device__ inline uint32_t gemm_overread_bytes(int a_rows) {
 }
 // bytes after the stage ring: barriers + tmem slot + abort flag, then epilogue constants
 __host__ __device__ inline uint32_t gemm_tail_bytes(int tile_n, int d_c) {
-    return 1024u + 2u * (static_cast<uint32_t>(tile_n) * static_cast<uint32_t>(2 + d_c) +
+    return 1024u + 4096u + 2u * (static_cast<uint32_t>(tile_n) * static_cast<uint32_t>(2 + d_c) +
                         static_cast<uint32_t>(kEpiThreads * d_c)) * 4u;
 }
 
@@ -111,11 +118,19 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     const uint32_t drain_bar = bar_base + 8u * (2 * kMaxStages + 4);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + ring_bytes + 8 * (2 * kMaxStages + 5));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [0] abort, [1] drain scratch
-    float* epi_const = reinterpret_cast<float*>(smem + ring_bytes + 1024);
+    volatile int* last_flag = abort_flag + 2;                                    // split-K: this CTA finishes the tile
+    float* split_red = reinterpret_cast<float*>(smem + ring_bytes + 1024);     // [128][<= 8] split-K row sums
+    float* epi_const = reinterpret_cast<float*>(smem + ring_bytes + 1024 + 4096);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int total_tiles = p.m_tiles * p.n_tiles;
+    const int total_tiles = p.m_tiles * p.n_tiles * p.k_splits;      // work items
+    // item t -> row tile m (fastest), K split ks, column tile n
+    auto item_m = [&](int t) { return t % p.m_tiles; };
+    auto item_ks = [&](int t) { return (t / p.m_tiles) % p.k_splits; };
+    auto item_n = [&](int t) { return (t / p.m_tiles) / p.k_splits; };
+    auto item_kb0 = [&](int t) { return item_ks(t) * p.kb_per_split; };
+    auto item_kb1 = [&](int t) { const int e = (item_ks(t) + 1) * p.kb_per_split; return e < p.k_blocks ? e : p.k_blocks; };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -144,8 +159,9 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             long long issued = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                const int m = t % p.m_tiles, n = t / p.m_tiles;
-                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                const int m = item_m(t), n = item_n(t);
+                const int kb1 = item_kb1(t);
+                for (int kb = item_kb0(t); kb < kb1; ++kb) {
                     if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, kWaitLimitNs)) { ok = false; break; }
                     const uint32_t a_dst = smem_base + stage_bytes * s;
                     mbar_expect_tx(full_bar(s), stage_bytes);
@@ -180,7 +196,8 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 if (!mbar_wait_bounded(acc_empty_bar(as), aph ^ 1u, abort_flag, kWaitLimitNs)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(as * kAccCols);
-                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                const int kb0 = item_kb0(t), kb1 = item_kb1(t);
+                for (int kb = kb0; kb < kb1; ++kb) {
                     if (!mbar_wait_bounded(full_bar(s), ph, abort_flag, kWaitLimitNs)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_addr = smem_base + stage_bytes * s;
@@ -189,7 +206,7 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 #pragma unroll
                     for (int k = 0; k < kBlockK / kUmmaK; ++k) {
                         // advancing K by 16 bf16 = 32 bytes = 2 descriptor units inside the swizzle atom
-                        umma_bf16(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        umma_bf16(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, ((kb - kb0) | k) != 0 ? 1u : 0u);
                     }
                     umma_commit(empty_bar(s));       // stage is free once these MMAs have read it
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
@@ -211,7 +228,7 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         float mx = -CUDART_INF_F, sum = 0.0f, hs = 0.0f;   // running row state (per tile, or per CTA when carry)
         int arg = 0;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++local) {
-            const int m = t % p.m_tiles, n = t / p.m_tiles;
+            const int m = item_m(t), n = item_n(t);
             const int as = local & 1;
             const uint32_t aph = (local >> 1) & 1u;
             const int row = m * kTileM + q * 32 + lane;
@@ -234,7 +251,9 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                         wwc[c * p.tile_n + j] = in ? p.w1c[(size_t)(n0 + j) * p.d_c + c] : 0.0f;
                 }
                 const int rq = valid ? p.pos_req[row] : 0;
-                for (int c = 0; c < p.d_c; ++c) wcs[c * kEpiThreads + et] = valid ? p.csi[(size_t)rq * p.d_c + c] : 0.0f;
+                // indexed by row within the tile (this thread's TMEM lane), not by thread number
+                for (int c = 0; c < p.d_c; ++c)
+                    wcs[c * kEpiThreads + q * 32 + lane] = valid ? p.csi[(size_t)rq * p.d_c + c] : 0.0f;
                 cb1 = wb1; cw2 = ww2; cwc = wwc; ccs = wcs;
             }
 
@@ -291,12 +310,20 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                         for (int j = 0; j < 16; ++j) tl = (tok - col0 == j) ? f[j] : tl;
                         p.tok_logit[row] = tl;
                     }
+                } else if (EPI == EPI_HEAD && p.k_splits > 1) {
+                    // split K: park the raw partial tile; the last item of this (m, n) tile finishes it
+                    float4* dst = reinterpret_cast<float4*>(
+                        p.splitk_buf + ((size_t)t * kTileM + (q * 32 + lane)) * p.tile_n + c0);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                             __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
                 } else if (EPI == EPI_HEAD) {
                     float pre[16];
 #pragma unroll
                     for (int j = 0; j < 16; ++j) pre[j] = __uint_as_float(v[j]) + cb1[c0 + j];
                     for (int c = 0; c < p.d_c; ++c) {
-                        const float x = ccs[c * kEpiThreads + et];
+                        const float x = ccs[c * kEpiThreads + q * 32 + lane];
 #pragma unroll
                         for (int j = 0; j < 16; ++j) pre[j] = fmaf(x, cwc[c * p.tile_n + c0 + j], pre[j]);
                     }
@@ -313,7 +340,58 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty_bar(as));
 
-            if (valid && !p.carry) {
+            if (EPI == EPI_HEAD && p.k_splits > 1) {
+                // publish this item's partial tile, then find out whether it was the last of its tile
+                __threadfence();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (et == 0) {
+                    const int old = atomicAdd(p.splitk_count + (m * p.n_tiles + n), 1);
+                    const int last = old == p.k_splits - 1;
+                    if (last) atomicExch(p.splitk_count + (m * p.n_tiles + n), 0);   // ready for the next call
+                    *last_flag = last;
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                const bool finisher = *last_flag != 0;
+                if (finisher) {
+                    // The whole epilogue group adds up the split tiles: a warp takes 32 columns of one
+                    // row at a time (coalesced reads, all split loads in flight together), applies the
+                    // head epilogue per column and reduces over the 32 columns with shuffles; the
+                    // per-(row, chunk) sums are then added in chunk order, so the result is deterministic.
+                    __threadfence();
+                    const int chunks = (p.tile_n + 31) / 32;
+                    const int rows_here = min(kTileM, p.rows - m * kTileM);
+                    const int ew = et >> 5;
+                    for (int pair = ew; pair < rows_here * chunks; pair += kEpiThreads / 32) {
+                        const int r = pair / chunks, ch = pair - r * chunks;
+                        const int col = ch * 32 + lane;
+                        float val = 0.0f;
+                        if (col < p.tile_n) {
+                            float x[kMaxKSplits];
+#pragma unroll
+                            for (int ks = 0; ks < kMaxKSplits; ++ks) {
+                                const int it = (n * p.k_splits + ks) * p.m_tiles + m;
+                                x[ks] = ks < p.k_splits
+                                            ? __ldcg(p.splitk_buf + ((size_t)it * kTileM + r) * p.tile_n + col) : 0.0f;
+                            }
+                            float pre = 0.0f;
+#pragma unroll
+                            for (int ks = 0; ks < kMaxKSplits; ++ks) pre += x[ks];      // split order
+                            pre += cb1[col];
+                            for (int c = 0; c < p.d_c; ++c) pre = fmaf(ccs[c * kEpiThreads + r], cwc[c * p.tile_n + col], pre);
+                            val = cw2[col] * act_apply(pre, p.act);
+                        }
+#pragma unroll
+                        for (int off = 16; off > 0; off >>= 1) val += __shfl_xor_sync(0xffffffffu, val, off);
+                        if (lane == 0) split_red[r * chunks + ch] = val;
+                    }
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    if (et < rows_here) {
+                        float tot = 0.0f;
+                        for (int ch = 0; ch < chunks; ++ch) tot += split_red[et * chunks + ch];
+                        p.head_part[(size_t)(m * kTileM + et) * p.part_stride + n] = tot;
+                    }
+                }
+            } else if (valid && !p.carry) {
                 if (EPI == EPI_LMHEAD)
                     p.lm_part[(size_t)row * p.part_stride + n] = make_float4(mx, __int_as_float(arg), sum, 0.0f);
                 else if (EPI == EPI_HEAD)

@@ -61,17 +61,21 @@ __device__ __forceinline__ void fence_proxy_async() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
-// Bounded wait: gives up after `limit_ns` (or as soon as *abort_flag is set by
-// another role), so a broken pipeline ends with an error word, never a hang.
+// Bounded wait: gives up after `limit_cycles` SM clocks (or as soon as *abort_flag
+// is set by another role), so a broken pipeline ends with an error word, never a
+// hang.  The deadline uses the SM's own cycle counter, which is cheap to read; the
+// first polls take no timestamp at all so a short wait costs nothing extra.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
-                                                  volatile int* abort_flag, uint64_t limit_ns) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = globaltimer_ns();
+                                                  volatile int* abort_flag, uint64_t limit_cycles) {
+#pragma unroll 1
+    for (int i = 0; i < 8; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
     uint32_t it = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if ((++it & 0x3FFu) == 0) {
+        if ((++it & 0xFFu) == 0) {
             if (*abort_flag != 0) return false;
-            if (globaltimer_ns() - t0 > limit_ns) { *abort_flag = 1; return false; }
+            if (static_cast<uint64_t>(clock64() - t0) > limit_cycles) { *abort_flag = 1; return false; }
         }
     }
     return true;

@@ -208,6 +208,7 @@ extern "C" int wisv_lm_head_reduce_static(const void* lm_head, int32_t V, int32_
     memset(&gp, 0, sizeof gp);
     gp.rows = R; gp.n_total = V; gp.k_blocks = (H + kBlockK - 1) / kBlockK; gp.tile_n = tile_n;
     gp.m_tiles = 1; gp.n_tiles = n_tiles; gp.a_rows = kTileM; gp.carry = 0; gp.part_stride = n_tiles;
+    gp.k_splits = 1; gp.kb_per_split = gp.k_blocks;
     const size_t fixed = 1024 + gemm_tail_bytes(tile_n, 0);
     int stages = (int)(((size_t)s->max_smem - fixed) / gemm_stage_bytes(tile_n));
     if (stages > kMaxStages) stages = kMaxStages;

@@ -80,6 +80,44 @@ def test_shapes(kw):
     _run(_small(**kw))
 
 
+@pytest.mark.parametrize("kw", [dict(B=2, K=8), dict(B=4, K=4, d_c=3), dict(B=3, K=1, H=72, H_d=40, d_J=50),
+                                dict(B=5, K=3, act="relu"), dict(B=20, K=5, d_J=200)],
+                         ids=["P16", "P16dc3", "P3odd", "P15relu", "P100"])
+def test_split_k_head_matches_single_pass_head(kw):
+    """One row tile of positions: the head GEMM splits K over CTAs; forcing a tile height turns that off."""
+    cfg = _small(seed=17, **kw)
+    case, ref, out, _ = _run(cfg)
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d)
+    v.set_tuning(head_tile_n=16)
+    for _ in range(2):                       # twice: the split-K tile counters must have reset themselves
+        o2 = cases.run(v, d)
+    torch.cuda.synchronize()
+    assert v.device_error() == 0
+    compare(case, ref, o2, cfg.tau)
+    assert float((o2.head_prob - out.head_prob).abs().max()) < 1e-5
+    assert torch.equal(o2.accept_len, out.accept_len)
+    v.set_tuning()
+    o3 = cases.run(v, d)
+    assert torch.equal(o3.head_prob, out.head_prob)      # deterministic from call to call
+    v.close()
+
+
+@pytest.mark.parametrize("tune", [dict(lm_tile_n=64), dict(lm_tile_n=256, lm_stages=2), dict(head_tile_n=64, head_stages=3)],
+                         ids=lambda t: "-".join("%s%s" % kv for kv in t.items()))
+def test_results_do_not_depend_on_the_launch_plan(tune):
+    cfg = _small(B=20, K=5, seed=19)
+    case = cases.make_case(cfg, oracle_ref_argmax)
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d)
+    v.set_tuning(**tune)
+    out = cases.run(v, d)
+    torch.cuda.synchronize()
+    assert v.device_error() == 0
+    compare(case, run_oracle(case), out, cfg.tau)
+    v.close()
+
+
 @pytest.mark.parametrize("tau", [0.0, 0.35, 0.65, 1.5])
 def test_thresholds(tau):
     case, ref, out, _ = _run(_small(B=24, K=6, seed=3), tau=tau)
