@@ -11,6 +11,7 @@
 #include <string.h>
 
 #include <new>
+#include <utility>
 
 #include "../../include/wisv.h"
 #include "wisv_aux.cuh"
@@ -276,12 +277,28 @@ int validate_batch(const wisv_ctx* c, const wisv_batch* b, const wisv_result* r,
     return WISV_OK;
 }
 
+// Launch with programmatic stream serialisation: the kernel may be scheduled while its predecessor in
+// the stream is still running; it synchronises with it through griddepcontrol.wait in device code.
+template <typename... KArgs, typename... Args>
+int launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args)
+{
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    WISV_CUDA(cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...));
+    return WISV_OK;
+}
+
 template <int EPI>
 int launch_gemm(wisv_ctx* c, const CUtensorMap& tA, const CUtensorMap& tB, const GemmParams& gp, const Plan& pl,
                 cudaStream_t st)
 {
-    gemm_rowreduce_kernel<EPI><<<pl.ctas, kGemmThreads, pl.smem, st>>>(tA, tB, gp);
-    WISV_CUDA(cudaGetLastError());
+    const int rc = launch_pdl(gemm_rowreduce_kernel<EPI>, dim3(pl.ctas), dim3(kGemmThreads), pl.smem, st, tA, tB, gp);
+    if (rc != WISV_OK) return rc;
     c->launches++;
     return WISV_OK;
 }
@@ -493,8 +510,10 @@ int wisv_verify(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cu
     pp.sel_off = b->sel_off; pp.sel_pos = b->sel_pos;
     pp.X = c->X; pp.Z = c->Z; pp.row_tok = c->row_tok; pp.row_flag = c->row_flag; pp.tok_logit = c->tok_logit;
     pp.pos_req = c->pos_req; pp.pos_i = c->pos_i;
-    pack_kernel<<<R + P, 256, 0, st>>>(pp);
-    WISV_CUDA(cudaGetLastError());
+    {
+        const int rc = launch_pdl(pack_kernel, dim3(R + P), dim3(256), 0, st, pp);
+        if (rc != WISV_OK) return rc;
+    }
     c->launches++;
 
     // ---- 2. LM head: logits reduced on the fly
@@ -534,8 +553,10 @@ int wisv_verify(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cu
     tp.p_draft = r->p_draft; tp.head_prob = r->head_prob;
     tp.mismatch_mask = reinterpret_cast<unsigned long long*>(r->mismatch_mask); tp.n_mismatch = r->n_mismatch;
     tp.status = r->status;
-    tail_kernel<<<b->B, 256, 0, st>>>(tp);
-    WISV_CUDA(cudaGetLastError());
+    {
+        const int rc = launch_pdl(tail_kernel, dim3(b->B), dim3(256), 0, st, tp);
+        if (rc != WISV_OK) return rc;
+    }
     c->launches++;
     if (ev) { WISV_CUDA(cudaEventRecord(ev[4], st)); c->prof_calls++; }
     return WISV_OK;

@@ -70,6 +70,9 @@ __device__ __forceinline__ void cast_row(const float* __restrict__ src, __nv_bfl
 __global__ void __launch_bounds__(256) pack_kernel(const PackParams p)
 {
     __shared__ int s_src_row;
+    // the previous round's kernels still read the buffers this kernel rewrites
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int blk = blockIdx.x;
     if (blk < p.R) {
         const int r = blk;
@@ -171,6 +174,9 @@ __global__ void __launch_bounds__(256) tail_kernel(const TailParams p)
     if (threadIdx.x < kMaxK) { s_has[threadIdx.x] = 0; s_prob[threadIdx.x] = 0.0f; }
     if (threadIdx.x == 0) s_flag = 0;
     __syncthreads();
+    // partials of the LM-head and decision-head kernels must be complete and visible
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // ---- merge the per-tile (max, argidx, sumexp) partials of each window row
     int flag = 0;

@@ -151,6 +151,14 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    // Everything above overlaps the previous kernel in the stream.  The LM-head and raw kernels read
+    // what the pack kernel wrote, so they wait for it here.  The decision-head kernel also reads only
+    // pack output, which is complete by the time it can be scheduled (the LM-head kernel releases its
+    // dependents only after its own wait); it waits at its end instead, so that "head kernel complete"
+    // implies "LM-head kernel complete" for the merge/scan kernel that follows.
+    if (EPI != EPI_HEAD) griddep_wait();
+    griddep_launch_dependents();
+
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -417,6 +425,7 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         tc_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
     }
+    if (EPI == EPI_HEAD) griddep_wait();
     if (threadIdx.x == 0 && (abort_flag[0] != 0)) atomicOr(p.err, 1);
 }
 
