@@ -1,0 +1,60 @@
+"""The one-process-per-GPU plumbing of bench.py on CPU: two gloo ranks, and the reference arm under torchrun."""
+import json
+import os
+import socket
+import subprocess
+import sys
+import textwrap
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _torchrun(nproc, script_args, env_extra=None, timeout=600):
+    env = dict(os.environ)
+    env.update(env_extra or {})
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(nproc),
+           "--master-addr", "127.0.0.1", "--master-port", str(_free_port())] + script_args
+    return subprocess.run(cmd, cwd=ROOT, env=env, capture_output=True, text=True, timeout=timeout)
+
+
+def test_max_over_ranks_and_sharded_seeds_with_two_gloo_ranks(tmp_path):
+    script = tmp_path / "ranks.py"
+    script.write_text(textwrap.dedent("""
+        import json, os, sys
+        sys.path.insert(0, %r)
+        import bench
+        rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+        r = bench.Ranks(world, backend="gloo")
+        r.barrier()
+        slowest = r.max(1.0 + rank)                       # every rank must learn the slowest rank's time
+        cfg = bench.workload_config("8b_b1", rank)        # each rank verifies its own batch of the same model
+        print(json.dumps({"rank": rank, "max": slowest, "seed": cfg.seed, "weight_seed": cfg.weight_seed,
+                          "value": bench.aggregate(world, 8, slowest)}), flush=True)
+        r.close()
+    """ % ROOT))
+    out = _torchrun(2, [str(script)])
+    assert out.returncode == 0, out.stderr[-2000:]
+    recs = [json.loads(l) for l in out.stdout.splitlines() if l.startswith("{")]
+    assert sorted(r["rank"] for r in recs) == [0, 1]
+    assert all(r["max"] == 2.0 for r in recs)
+    assert len({r["seed"] for r in recs}) == 2 and len({r["weight_seed"] for r in recs}) == 1
+    assert all(abs(r["value"] - 2 * 8 / 2.0e-3) < 1e-9 for r in recs)   # job-wide units / slowest step
+
+
+def test_reference_arm_prints_one_line_from_rank_zero_only():
+    out = _torchrun(2, ["bench.py", "--impl", "reference", "--gpus", "2", "--steps", "1", "--warmup", "0",
+                        "--workload", "tiny", "--oracle-rows", "10"])
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    rec = json.loads(lines[0])
+    assert rec["impl"] == "reference" and rec["n_gpus"] == 2 and rec["gpu_launches"] == 0
+    assert rec["cpu_baseline"]["kind"] == "oracle" and rec["cpu_baseline"]["value"] == rec["value"]
+    assert rec["e2e"]["h2d_bytes_per_step"] == 0 and rec["e2e"]["value"] == rec["value"]
+    assert rec["config"]["workload"] == "tiny" and rec["vs_baseline"] is None
