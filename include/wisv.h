@@ -156,6 +156,29 @@ int wisv_create(const wisv_config* cfg, const wisv_weights* weights, wisv_ctx** 
 int wisv_verify(wisv_ctx* ctx, const wisv_batch* batch, const wisv_result* result, void* cuda_stream);
 
 /*
+ * The selective-hidden protocol in the two steps the paper runs it in (Algorithm 1:
+ * Verify and Localize, then RequestHidden / Upload of the hidden states of S, then the
+ * decision; Section III-B option 2 and the payloads B_req, B_u2 of Eqs. 8-9).
+ *
+ * wisv_localize runs steps 1-3 of the round: it needs B, K / k_off, T_total,
+ * target_hidden, draft_tokens (and draft_q, uniforms for the stochastic test) and
+ * writes any of mismatch_mask, n_mismatch (m_r, what the edge requests from the
+ * device), argmax, lse, p_draft; if accept_len / correction_token are given they
+ * receive the plain greedy result (what the round yields if no hidden state ever
+ * arrives).  The context keeps the per-row argmax and the candidate sets.
+ *
+ * wisv_decide runs steps 4-5 for the batch of the preceding wisv_localize on the same
+ * context (same B, K / k_off pointer and T_total, else WISV_ESHAPE; WISV_EINVAL if no
+ * localize is pending): it needs target_hidden again (h^T is a head input),
+ * draft_hidden with sel_off / sel_pos (WISV_MODE_SH) or dense (WISV_MODE_FH), csi and
+ * tau, and writes accept_len, correction_token and optionally head_prob,
+ * mismatch_mask, n_mismatch, status.  Localize followed by decide gives exactly the
+ * result of one wisv_verify on the same inputs.  Both calls only enqueue work.
+ */
+int wisv_localize(wisv_ctx* ctx, const wisv_batch* batch, const wisv_result* result, void* cuda_stream);
+int wisv_decide(wisv_ctx* ctx, const wisv_batch* batch, const wisv_result* result, void* cuda_stream);
+
+/*
  * Same round with HOST buffers: every pointer in `batch` and `result` is host
  * memory (pinned memory makes the copies asynchronous).  Inputs are copied to
  * staging buffers owned by the context (allocated on first use), the round is

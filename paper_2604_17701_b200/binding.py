@@ -80,7 +80,7 @@ def load_library(build_if_missing: bool = False):
     lib.wisv_create.argtypes = [C.POINTER(_Config), C.POINTER(_Weights), C.POINTER(P)]
     lib.wisv_destroy.restype = C.c_int
     lib.wisv_destroy.argtypes = [P]
-    for name in ("wisv_verify", "wisv_verify_host"):
+    for name in ("wisv_verify", "wisv_verify_host", "wisv_localize", "wisv_decide"):
         f = getattr(lib, name)
         f.restype = C.c_int
         f.argtypes = [P, C.POINTER(_Batch), C.POINTER(_Result), P]
@@ -224,6 +224,44 @@ class Verifier:
         r = self._result(out)
         st = stream if stream is not None else torch.cuda.current_stream(self.device)
         _check(self.lib.wisv_verify(self._h, C.byref(b), C.byref(r), C.c_void_p(st.cuda_stream)), "wisv_verify")
+        return out
+
+    def localize(self, target_hidden, draft_tokens, *, B: int, K: int = 0, k_off=None, T: Optional[int] = None,
+                 draft_q=None, uniforms=None, out: Optional[VerifyOutput] = None, stream=None) -> VerifyOutput:
+        """wisv_localize: LM head, argmax / log-sum-exp and the candidate sets S (first phase of SH)."""
+        torch = self._torch
+        if T is None:
+            T = B * K if k_off is None else int(draft_tokens.shape[0])
+        if out is None:
+            out = self._outputs(B, T + B, T, 0, self.device, True)
+            out.head_prob = None
+        b = self._batch(B=B, K=K, k_off=k_off, T=T, target_hidden=target_hidden, draft_tokens=draft_tokens,
+                        draft_hidden=None, csi=None, sel_off=None, sel_pos=None, draft_q=draft_q,
+                        uniforms=uniforms, tau=None)
+        r = self._result(out)
+        st = stream if stream is not None else torch.cuda.current_stream(self.device)
+        _check(self.lib.wisv_localize(self._h, C.byref(b), C.byref(r), C.c_void_p(st.cuda_stream)), "wisv_localize")
+        return out
+
+    def decide(self, target_hidden, draft_hidden, csi, *, B: int, K: int = 0, k_off=None, T: int,
+               sel_off=None, sel_pos=None, tau: Optional[float] = None, out: Optional[VerifyOutput] = None,
+               stream=None) -> VerifyOutput:
+        """wisv_decide: decision head on the uploaded hidden states and the first-reject scan (second phase)."""
+        torch = self._torch
+        P = int(sel_pos.shape[0]) if sel_pos is not None else T
+        if out is None:
+            out = VerifyOutput(torch.empty(B, dtype=torch.int32, device=self.device),
+                               torch.empty(B, dtype=torch.int32, device=self.device))
+            out.head_prob = torch.empty(P, dtype=torch.float32, device=self.device)
+            out.mismatch_mask = torch.empty(B, dtype=torch.int64, device=self.device)
+            out.n_mismatch = torch.empty(B, dtype=torch.int32, device=self.device)
+            out.status = torch.empty(B, dtype=torch.int32, device=self.device)
+        b = self._batch(B=B, K=K, k_off=k_off, T=T, target_hidden=target_hidden, draft_tokens=None,
+                        draft_hidden=draft_hidden, csi=csi, sel_off=sel_off, sel_pos=sel_pos, draft_q=None,
+                        uniforms=None, tau=tau)
+        r = self._result(out)
+        st = stream if stream is not None else torch.cuda.current_stream(self.device)
+        _check(self.lib.wisv_decide(self._h, C.byref(b), C.byref(r), C.c_void_p(st.cuda_stream)), "wisv_decide")
         return out
 
     def verify_host(self, target_hidden, draft_tokens, draft_hidden, csi, *, B: int, K: int = 0, k_off=None,

@@ -76,6 +76,11 @@ struct wisv_ctx {
     int32_t* row_tok = nullptr; int32_t* row_flag = nullptr; float* tok_logit = nullptr;
     int32_t* pos_req = nullptr; int32_t* pos_i = nullptr;
     int32_t* err = nullptr;
+    int32_t* saved_arg = nullptr;               // [rows_alloc] argmax per row, localize -> decide
+    unsigned long long* saved_mask = nullptr;   // [max_requests] candidate sets, localize -> decide
+    bool loc_valid = false;                     // a localize call is waiting for its decide
+    int loc_B = 0, loc_T = 0, loc_K = 0;
+    const int32_t* loc_k_off = nullptr;
     // TMA descriptors
     CUtensorMap tmX[kNumRowVariants], tmZ[kNumRowVariants];   // box heights 8, 16, ..., 128 rows
     CUtensorMap tmW[kNumTileVariants];
@@ -219,6 +224,7 @@ void free_ctx(wisv_ctx* c)
     cudaFree(c->X); cudaFree(c->Z); cudaFree(c->W1p); cudaFree(c->W1c); cudaFree(c->lm_part);
     cudaFree(c->head_part); cudaFree(c->row_tok); cudaFree(c->row_flag); cudaFree(c->tok_logit);
     cudaFree(c->pos_req); cudaFree(c->pos_i); cudaFree(c->err); cudaFree(c->splitk_buf); cudaFree(c->splitk_count);
+    cudaFree(c->saved_arg); cudaFree(c->saved_mask);
     if (c->prof_ev) {
         for (int i = 0; i < c->prof_n * (kStages + 1); ++i) cudaEventDestroy(c->prof_ev[i]);
         free(c->prof_ev);
@@ -241,7 +247,10 @@ int dev_alloc(T** p, size_t n)
     return WISV_OK;
 }
 
-int validate_batch(const wisv_ctx* c, const wisv_batch* b, const wisv_result* r, int* T_out, int* R_out, int* P_out)
+enum { PHASE_FULL = 0, PHASE_LOCALIZE = 1, PHASE_DECIDE = 2 };
+
+int validate_batch(const wisv_ctx* c, const wisv_batch* b, const wisv_result* r, int* T_out, int* R_out, int* P_out,
+                   int phase = PHASE_FULL)
 {
     if (!c || !b || !r) return WISV_EINVAL;
     if (b->B < 0 || b->K < 0) return WISV_ESHAPE;
@@ -257,7 +266,9 @@ int validate_batch(const wisv_ctx* c, const wisv_batch* b, const wisv_result* r,
     const long long R = T + b->B;
     if (b->B > c->cfg.max_requests || R > c->cfg.max_rows) return WISV_ECAPACITY;
     long long P = T;
-    if (sh) {
+    if (phase == PHASE_LOCALIZE) {
+        P = 0;
+    } else if (sh) {
         if (b->M_sel < 0) return WISV_ESHAPE;
         if (b->M_sel > c->max_pos || b->M_sel > T) return b->M_sel > T ? WISV_ESHAPE : WISV_ECAPACITY;
         P = b->M_sel;
@@ -266,10 +277,11 @@ int validate_batch(const wisv_ctx* c, const wisv_batch* b, const wisv_result* r,
     }
     if (P > c->max_pos) return WISV_ECAPACITY;
     if (b->B > 0) {
-        if (!b->target_hidden || !r->accept_len || !r->correction_token) return WISV_EINVAL;
-        if (T > 0 && !b->draft_tokens) return WISV_EINVAL;
+        if (!b->target_hidden) return WISV_EINVAL;
+        if (phase != PHASE_LOCALIZE && (!r->accept_len || !r->correction_token)) return WISV_EINVAL;
+        if (phase != PHASE_DECIDE && T > 0 && !b->draft_tokens) return WISV_EINVAL;
         if (P > 0 && (!b->draft_hidden || (c->cfg.d_c > 0 && !b->csi))) return WISV_EINVAL;
-        if (stoch && T > 0 && (!b->draft_q || !b->uniforms)) return WISV_EINVAL;
+        if (phase != PHASE_DECIDE && stoch && T > 0 && (!b->draft_q || !b->uniforms)) return WISV_EINVAL;
         if (!aligned16(b->target_hidden) || (P > 0 && !aligned16(b->draft_hidden))) return WISV_EALIGN;
     }
     if (!(b->tau != b->tau) && b->tau < 0.0f) return WISV_EINVAL;
@@ -416,6 +428,8 @@ int wisv_create(const wisv_config* cfg, const wisv_weights* w, wisv_ctx** out)
         if ((rc = dev_alloc(&c->pos_req, (size_t)c->pos_alloc))) break;
         if ((rc = dev_alloc(&c->pos_i, (size_t)c->pos_alloc))) break;
         if ((rc = dev_alloc(&c->err, 1))) break;
+        if ((rc = dev_alloc(&c->saved_arg, (size_t)c->rows_alloc))) break;
+        if ((rc = dev_alloc(&c->saved_mask, (size_t)cfg->max_requests))) break;
         c->splitk_tiles = (cfg->d_J + 15) / 16;
         if ((rc = dev_alloc(&c->splitk_buf, (size_t)c->sm_count * kTileM * kSplitTileN))) break;
         if ((rc = dev_alloc(&c->splitk_count, (size_t)c->splitk_tiles))) break;
@@ -484,11 +498,22 @@ int wisv_set_tuning(wisv_ctx* c, const wisv_tuning* t)
     return WISV_OK;
 }
 
-int wisv_verify(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda_stream)
+}  // extern "C"
+
+namespace {
+
+// One verification round, or one of its two phases (localize: pack rows + LM head + merge;
+// decide: pack positions + decision head + scan on the candidate sets the localize call saved).
+int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda_stream, int phase)
 {
     int T = 0, R = 0, P = 0;
-    const int vrc = validate_batch(c, b, r, &T, &R, &P);
+    const int vrc = validate_batch(c, b, r, &T, &R, &P, phase);
     if (vrc != WISV_OK) return vrc;
+    if (phase == PHASE_DECIDE) {
+        if (!c->loc_valid) return WISV_EINVAL;
+        if (b->B != c->loc_B || T != c->loc_T || (b->k_off ? 0 : b->K) != c->loc_K || b->k_off != c->loc_k_off)
+            return WISV_ESHAPE;
+    }
     if (b->B == 0) return WISV_OK;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const bool sh = (b->mode & WISV_MODE_SH) != 0;
@@ -504,23 +529,24 @@ int wisv_verify(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cu
     if (ev) WISV_CUDA(cudaEventRecord(ev[0], st));
     PackParams pp;
     memset(&pp, 0, sizeof pp);
-    pp.ix = ix; pp.R = R; pp.P = P; pp.H = cf.H; pp.H_d = cf.H_d; pp.V = cf.V; pp.shift = cf.head_row_shift;
+    const int pack_rows = phase == PHASE_DECIDE ? 0 : R;
+    pp.ix = ix; pp.R = pack_rows; pp.P = P; pp.H = cf.H; pp.H_d = cf.H_d; pp.V = cf.V; pp.shift = cf.head_row_shift;
     pp.mode_sh = sh ? 1 : 0;
     pp.target_hidden = b->target_hidden; pp.draft_hidden = b->draft_hidden; pp.draft_tokens = b->draft_tokens;
     pp.sel_off = b->sel_off; pp.sel_pos = b->sel_pos;
     pp.X = c->X; pp.Z = c->Z; pp.row_tok = c->row_tok; pp.row_flag = c->row_flag; pp.tok_logit = c->tok_logit;
     pp.pos_req = c->pos_req; pp.pos_i = c->pos_i;
-    {
-        const int rc = launch_pdl(pack_kernel, dim3(R + P), dim3(256), 0, st, pp);
+    if (pack_rows + P > 0) {
+        const int rc = launch_pdl(pack_kernel, dim3(pack_rows + P), dim3(256), 0, st, pp);
         if (rc != WISV_OK) return rc;
+        c->launches++;
     }
-    c->launches++;
 
     // ---- 2. LM head: logits reduced on the fly
     if (ev) WISV_CUDA(cudaEventRecord(ev[1], st));
     const Plan pl = plan_lm(c, R);
     if ((size_t)R * pl.parts > c->lm_part_elems) return WISV_ECAPACITY;
-    {
+    if (phase != PHASE_DECIDE) {
         GemmParams gp = base_params(c, pl, R, cf.V, cf.H);
         gp.lm_part = c->lm_part; gp.row_tok = c->row_tok; gp.tok_logit = c->tok_logit;
         const int rc = launch_gemm<EPI_LMHEAD>(c, c->tmX[pl.a_rows / 8 - 1], c->tmW[pl.tile_n / 16 - 1], gp, pl, st);
@@ -545,6 +571,7 @@ int wisv_verify(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cu
     TailParams tp;
     memset(&tp, 0, sizeof tp);
     tp.ix = ix; tp.P = P; tp.V = cf.V; tp.n_tiles_lm = pl.parts; tp.n_tiles_head = ph.parts; tp.mode_sh = sh ? 1 : 0;
+    tp.phase = phase; tp.saved_arg = c->saved_arg; tp.saved_mask = c->saved_mask;
     tp.stochastic = stoch ? 1 : 0; tp.b2 = c->w.b2; tp.tau = (b->tau != b->tau) ? cf.tau : b->tau;
     tp.lm_part = c->lm_part; tp.tok_logit = c->tok_logit; tp.row_flag = c->row_flag; tp.draft_tokens = b->draft_tokens;
     tp.head_part = c->head_part; tp.pos_i = c->pos_i; tp.sel_off = b->sel_off; tp.draft_q = b->draft_q;
@@ -559,7 +586,31 @@ int wisv_verify(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cu
     }
     c->launches++;
     if (ev) { WISV_CUDA(cudaEventRecord(ev[4], st)); c->prof_calls++; }
+    if (phase == PHASE_LOCALIZE) {
+        c->loc_valid = true; c->loc_B = b->B; c->loc_T = T; c->loc_K = b->k_off ? 0 : b->K; c->loc_k_off = b->k_off;
+    } else {
+        c->loc_valid = false;
+    }
     return WISV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int wisv_verify(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda_stream)
+{
+    return run_round(c, b, r, cuda_stream, PHASE_FULL);
+}
+
+int wisv_localize(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda_stream)
+{
+    return run_round(c, b, r, cuda_stream, PHASE_LOCALIZE);
+}
+
+int wisv_decide(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda_stream)
+{
+    return run_round(c, b, r, cuda_stream, PHASE_DECIDE);
 }
 
 int wisv_debug_logits(wisv_ctx* c, const float* target_hidden, int32_t R, float* logits_out, void* cuda_stream)

@@ -129,6 +129,9 @@ __global__ void split_w1_kernel(const __nv_bfloat16* __restrict__ W1, __nv_bfloa
 struct TailParams {
     BatchIndex ix;
     int32_t P, V, n_tiles_lm, n_tiles_head, mode_sh, stochastic;
+    int32_t phase;                // 0: whole round; 1: localize only (no head); 2: decide from a saved localize
+    int32_t* saved_arg;           // [R] argmax per window row kept between the two phases
+    unsigned long long* saved_mask;  // [B] candidate set S per request kept between the two phases
     float b2, tau;
     const float4* lm_part;        // [R][n_tiles_lm]
     const float* tok_logit;       // [R]
@@ -180,7 +183,11 @@ __global__ void __launch_bounds__(256) tail_kernel(const TailParams p)
 
     // ---- merge the per-tile (max, argidx, sumexp) partials of each window row
     int flag = 0;
-    for (int i = warp; i <= Kb; i += nwarps) {
+    if (p.phase == 2) {
+        // second phase: the rows were reduced by the localize call
+        for (int i = threadIdx.x; i <= Kb; i += blockDim.x) { s_arg[i] = p.saved_arg[r0 + i]; flag |= p.row_flag[r0 + i]; }
+    }
+    for (int i = warp; i <= Kb && p.phase != 2; i += nwarps) {
         const int r = r0 + i;
         RowStat st{-CUDART_INF_F, 0x7fffffff, 0.0f};
         const float4* part = p.lm_part + (size_t)r * p.n_tiles_lm;
@@ -208,6 +215,7 @@ __global__ void __launch_bounds__(256) tail_kernel(const TailParams p)
         if (lane == 0) {
             s_arg[i] = st.idx;
             s_lse[i] = l;
+            if (p.phase == 1) p.saved_arg[r] = st.idx;
             if (p.argmax) p.argmax[r] = st.idx;
             if (p.lse) p.lse[r] = l;
             if (!isfinite(l)) flag |= 4;
@@ -217,7 +225,8 @@ __global__ void __launch_bounds__(256) tail_kernel(const TailParams p)
 
     // ---- finish the decision head: s = b2 + sum of per-tile partial dot products
     int e0, e1;
-    if (p.mode_sh) { e0 = max(p.sel_off[b], 0); e1 = min(p.sel_off[b + 1], p.P); } else { e0 = k0; e1 = k0 + Kb; }
+    if (p.phase == 1) { e0 = 0; e1 = 0; }
+    else if (p.mode_sh) { e0 = max(p.sel_off[b], 0); e1 = min(p.sel_off[b + 1], p.P); } else { e0 = k0; e1 = k0 + Kb; }
     for (int e = e0 + warp; e < e1; e += nwarps) {
         float s = 0.0f;
         const float* hp = p.head_part + (size_t)e * p.n_tiles_head;
@@ -246,17 +255,21 @@ __global__ void __launch_bounds__(256) tail_kernel(const TailParams p)
             bool cand = false, rej = false;
             if (i < Kb) {
                 const int t = k0 + i;
-                const float pd = expf(p.tok_logit[r0 + i] - s_lse[i]);
-                if (p.p_draft) p.p_draft[t] = pd;
-                if (p.stochastic) {
-                    const float alpha = fminf(1.0f, pd / p.draft_q[t]);
-                    cand = !(p.uniforms[t] < alpha);
+                if (p.phase == 2) {
+                    cand = (p.saved_mask[b] >> i) & 1ull;
                 } else {
-                    cand = p.draft_tokens[t] != s_arg[i];
+                    const float pd = expf(p.tok_logit[r0 + i] - s_lse[i]);
+                    if (p.p_draft) p.p_draft[t] = pd;
+                    if (p.stochastic) {
+                        const float alpha = fminf(1.0f, pd / p.draft_q[t]);
+                        cand = !(p.uniforms[t] < alpha);
+                    } else {
+                        cand = p.draft_tokens[t] != s_arg[i];
+                    }
                 }
                 const bool has = s_has[i] != 0;
-                rej = cand && (!has || s_prob[i] >= p.tau);
-                if (cand && !has) missing = 1;
+                rej = cand && (!has || s_prob[i] >= p.tau);      // localize phase: no uploads yet, greedy
+                if (cand && !has && p.phase != 1) missing = 1;
             }
             cand_bits[h] = __ballot_sync(0xffffffffu, cand);
             rej_bits[h] = __ballot_sync(0xffffffffu, rej);
@@ -266,8 +279,9 @@ __global__ void __launch_bounds__(256) tail_kernel(const TailParams p)
             const unsigned long long rej = (unsigned long long)rej_bits[0] | ((unsigned long long)rej_bits[1] << 32);
             const unsigned long long cnd = (unsigned long long)cand_bits[0] | ((unsigned long long)cand_bits[1] << 32);
             const int A = rej ? (__ffsll((long long)rej) - 1) : Kb;
-            p.accept_len[b] = A;
-            p.correction[b] = s_arg[A];
+            if (p.accept_len) p.accept_len[b] = A;
+            if (p.correction) p.correction[b] = s_arg[A];
+            if (p.phase == 1) p.saved_mask[b] = cnd;
             if (p.mismatch_mask) p.mismatch_mask[b] = cnd;
             if (p.n_mismatch) p.n_mismatch[b] = __popcll(cnd);
             if (p.status) p.status[b] = s_flag | (missing ? 1 : 0);

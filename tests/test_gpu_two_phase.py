@@ -1,0 +1,89 @@
+"""The selective-hidden protocol in two calls (localize, then decide) against the one-call round and the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import gen
+from paper_2604_17701_b200 import WisvError, cases
+from parity import compare, oracle_ref_argmax, run_oracle
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _cfg(**kw):
+    base = dict(B=12, K=6, H=256, H_d=128, d_c=2, d_J=128, V=4096, match_rate=0.5, seed=31)
+    base.update(kw)
+    return gen.VerifyConfig("tp", **base)
+
+
+@pytest.mark.parametrize("kw", [dict(), dict(K=0, K_lo=1, K_hi=10, B=40), dict(match_rate=1.0), dict(match_rate=0.0),
+                                dict(B=1, K=8), dict(stochastic=True)],
+                         ids=["uniform", "ragged", "emptyS", "fullS", "single", "stochastic"])
+def test_localize_then_decide_equals_one_call(kw):
+    cfg = _cfg(**kw)
+    case = cases.make_case(cfg, oracle_ref_argmax)          # full-hidden traffic: dense draft hidden states
+    if cfg.stochastic:
+        base = run_oracle(case)
+        case["draft_q"] = (base["p_draft"] * np.random.default_rng(2).uniform(0.5, 4.0, size=case["T"])).astype(np.float32)
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d)
+    one = cases.run(v, d)
+    torch.cuda.synchronize()
+
+    kw_geo = dict(B=cfg.B, K=cfg.K if cfg.K_hi == 0 else 0, k_off=d["k_off_dev"], T=case["T"])
+    loc = v.localize(d["target_hidden"], d["draft_tokens"], draft_q=d["draft_q"], uniforms=d["uniforms"], **kw_geo)
+    torch.cuda.synchronize()
+    assert torch.equal(loc.mismatch_mask, one.mismatch_mask) and torch.equal(loc.n_mismatch, one.n_mismatch)
+    assert torch.equal(loc.argmax, one.argmax) and torch.equal(loc.lse, one.lse) and torch.equal(loc.p_draft, one.p_draft)
+    # greedy result while no hidden state has arrived: first candidate position
+    mask = loc.mismatch_mask.cpu().numpy().astype(np.uint64)
+    first = np.array([next((i for i in range(case["k_len"][b]) if (int(mask[b]) >> i) & 1), case["k_len"][b])
+                      for b in range(cfg.B)])
+    assert np.array_equal(loc.accept_len.cpu().numpy(), first)
+
+    # the device uploads exactly the hidden states the edge asked for (Algorithm 1: RequestHidden(S))
+    sel = np.zeros(case["T"], bool)
+    for b in range(cfg.B):
+        for i in range(case["k_len"][b]):
+            sel[case["k_off"][b] + i] = (int(mask[b]) >> i) & 1
+    packed, sel_off, sel_pos = gen.pack_selective(case["draft_hidden"], case["k_len"], sel)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+    dec = v.decide(d["target_hidden"], dev(packed), d["csi"], sel_off=dev(sel_off), sel_pos=dev(sel_pos), **kw_geo)
+    torch.cuda.synchronize()
+    assert v.device_error() == 0
+    assert torch.equal(dec.accept_len, one.accept_len) and torch.equal(dec.correction_token, one.correction_token)
+    assert torch.equal(dec.n_mismatch, one.n_mismatch)
+    hp_one = one.head_prob.cpu().numpy()[sel]
+    assert np.allclose(dec.head_prob.cpu().numpy(), hp_one, atol=1e-6)
+
+    # and against the oracle on the selective-hidden traffic
+    sh_case = dict(case, draft_hidden=packed, sel_off=sel_off, sel_pos=sel_pos)
+    ref = run_oracle(sh_case)
+    full = type("O", (), {})()
+    for k in ("argmax", "lse", "p_draft"):
+        setattr(full, k, getattr(loc, k))
+    for k in ("accept_len", "correction_token", "head_prob", "n_mismatch", "mismatch_mask", "status"):
+        setattr(full, k, getattr(dec, k))
+    compare(sh_case, ref, full, cfg.tau)
+    v.close()
+
+
+def test_decide_needs_a_matching_localize():
+    cfg = _cfg(B=4, K=4)
+    case = cases.make_case(cfg, oracle_ref_argmax)
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d)
+    with pytest.raises(WisvError) as e:                     # nothing pending
+        v.decide(d["target_hidden"], d["draft_hidden"], d["csi"], B=4, K=4, T=16)
+    assert e.value.code == -1
+    v.localize(d["target_hidden"], d["draft_tokens"], B=4, K=4)
+    with pytest.raises(WisvError) as e:                     # different geometry
+        v.decide(d["target_hidden"], d["draft_hidden"], d["csi"], B=2, K=4, T=8)
+    assert e.value.code == -2
+    out = v.decide(d["target_hidden"], d["draft_hidden"], d["csi"], B=4, K=4, T=16)     # dense upload also works
+    ref = cases.run(v, d)
+    assert torch.equal(out.accept_len, ref.accept_len)
+    with pytest.raises(WisvError):                          # consumed by the verify above
+        v.decide(d["target_hidden"], d["draft_hidden"], d["csi"], B=4, K=4, T=16)
+    v.close()
