@@ -228,6 +228,34 @@ int wisv_plan(const wisv_ctx* ctx, int32_t R, int32_t P, int32_t* lm_tile_n, int
               int32_t* lm_ctas, int32_t* head_tile_n, int32_t* head_tiles, int32_t* head_ctas);
 
 /*
+ * Link model of Section IV-A (host arithmetic only).  For one round with K_r draft
+ * tokens of which m_r were requested, computes the payloads in bits - B_hid (Eq. 3),
+ * B_fb (Eq. 4), B_u^FH (Eq. 5), B_u1^SH (Eq. 7), B_req (Eq. 8), B_u2^SH (Eq. 9) with
+ * b_id = ceil(log2 V) - and the communication latencies T_comm^FH (Eq. 6) and
+ * T_comm^SH (Eq. 10) in seconds.  m_r is the n_mismatch the verifier reports.
+ * Rates are in bit/s, PER in [0, 1), the round-trip time in seconds.
+ */
+typedef struct {
+    double rate_up_bps, rate_down_bps;   /* R_u(c), R_d(c) */
+    double per_up, per_down;             /* PER_u(c), PER_d(c) */
+    double rtt_s;                        /* tau_RTT */
+    double hdr_up_bits, hdr_down_bits;   /* B_hdr,u, B_hdr,d */
+    int32_t d_h, b_h;                    /* drafter hidden size and bits per element */
+    int32_t b_pos;                       /* bits per position index */
+} wisv_link;
+
+typedef struct {
+    int32_t b_id;
+    double B_hid, B_fb, B_u_FH, B_u1_SH, B_req, B_u2_SH;
+    double T_comm_FH, T_comm_SH;
+} wisv_link_cost;
+
+int wisv_link_cost_round(const wisv_link* link, int32_t V, int32_t K_r, int32_t m_r, wisv_link_cost* out);
+
+/* Protocol rule reported with the testbed (Section VII): WISV_MODE_FH if rtt_s > 10 ms, else WISV_MODE_SH. */
+int wisv_choose_protocol(double rtt_s);
+
+/*
  * Bring-up / test hook: the raw fp32 logits L = bf16(target_hidden) . lm_head^T
  * of R rows (Algorithm 1, Verify), written to logits_out (dev fp32 [R, V]) by the
  * same TMA + tcgen05 main loop with a store epilogue.  target_hidden: dev fp32

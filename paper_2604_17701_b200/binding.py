@@ -53,6 +53,29 @@ class _Tuning(C.Structure):
                 ("head_stages", C.c_int32)]
 
 
+class LinkParams(C.Structure):
+    _fields_ = [("rate_up_bps", C.c_double), ("rate_down_bps", C.c_double), ("per_up", C.c_double),
+                ("per_down", C.c_double), ("rtt_s", C.c_double), ("hdr_up_bits", C.c_double),
+                ("hdr_down_bits", C.c_double), ("d_h", C.c_int32), ("b_h", C.c_int32), ("b_pos", C.c_int32)]
+
+
+class LinkCost(C.Structure):
+    _fields_ = [("b_id", C.c_int32), ("B_hid", C.c_double), ("B_fb", C.c_double), ("B_u_FH", C.c_double),
+                ("B_u1_SH", C.c_double), ("B_req", C.c_double), ("B_u2_SH", C.c_double),
+                ("T_comm_FH", C.c_double), ("T_comm_SH", C.c_double)]
+
+
+def link_cost_round(link: "LinkParams", V: int, K_r: int, m_r: int) -> dict:
+    """wisv_link_cost_round: payloads (bits) and communication latencies (s) of one round."""
+    out = LinkCost()
+    _check(load_library().wisv_link_cost_round(C.byref(link), V, K_r, m_r, C.byref(out)), "wisv_link_cost_round")
+    return {n: getattr(out, n) for n, _ in LinkCost._fields_}
+
+
+def choose_protocol(rtt_s: float) -> int:
+    return int(load_library().wisv_choose_protocol(float(rtt_s)))
+
+
 def exported_symbols() -> List[str]:
     """Function names declared in include/wisv.h."""
     text = open(_HEADER).read()
@@ -96,6 +119,10 @@ def load_library(build_if_missing: bool = False):
     lib.wisv_plan.argtypes = [P, C.c_int32, C.c_int32] + [C.POINTER(C.c_int32)] * 6
     lib.wisv_debug_logits.restype = C.c_int
     lib.wisv_debug_logits.argtypes = [P, P, C.c_int32, P, P]
+    lib.wisv_link_cost_round.restype = C.c_int
+    lib.wisv_link_cost_round.argtypes = [C.POINTER(LinkParams), C.c_int32, C.c_int32, C.c_int32, C.POINTER(LinkCost)]
+    lib.wisv_choose_protocol.restype = C.c_int
+    lib.wisv_choose_protocol.argtypes = [C.c_double]
     lib.wisv_set_tuning.restype = C.c_int
     lib.wisv_set_tuning.argtypes = [P, C.POINTER(_Tuning)]
     lib.wisv_lm_head_reduce_static.restype = C.c_int
