@@ -55,6 +55,9 @@ class VerifyConfig:
 # one 8B-shaped model (LM head + decision head) serves every 8B workload
 _8B = dict(H=4096, H_d=2048, d_c=2, d_J=1024, V=128256, weight_seed=1000)
 
+# second model pair of the paper's testbed (Section VII): Qwen2.5-0.5B drafter -> Qwen2.5-7B target
+_QWEN = dict(H=3584, H_d=896, d_c=2, d_J=1024, V=152064, weight_seed=2000)
+
 CONFIGS: Dict[str, VerifyConfig] = {
     "tiny": VerifyConfig("tiny", B=8, K=4, H=256, H_d=128, d_c=2, d_J=128, V=4096,
                          match_rate=0.5, seed=0),
@@ -65,6 +68,8 @@ CONFIGS: Dict[str, VerifyConfig] = {
     "8b_sh256": VerifyConfig("8b_sh256", B=256, K=0, K_lo=4, K_hi=16, match_rate=0.65,
                              mode="SH", seed=5, **_8B),
     "8b_b512": VerifyConfig("8b_b512", B=512, K=16, match_rate=0.7, seed=6, **_8B),
+    "qwen7b_b1": VerifyConfig("qwen7b_b1", B=1, K=8, match_rate=0.7, seed=11, **_QWEN),
+    "qwen7b_b8_k64": VerifyConfig("qwen7b_b8_k64", B=8, K=64, match_rate=0.9, seed=12, **_QWEN),
     "8b_b512_stoch": VerifyConfig("8b_b512_stoch", B=512, K=16, match_rate=0.7, seed=7,
                                   stochastic=True, **_8B),
 }

@@ -338,6 +338,17 @@ def test_8b_selective_hidden_sampled():
     assert stats["tainted_requests"] < stats["requests"]
 
 
+def test_qwen_shapes_batch1_full_oracle():
+    # H = 3584 (56 K blocks), V = 152064, H_d = 896: the second model pair of the paper's testbed
+    _sampled_parity("qwen7b_b1", 1)
+
+
+def test_qwen_shapes_longest_window_sampled():
+    # K = 64, the largest draft length of Table I; 520 window rows over 5 row tiles
+    case, out, A, stats = _sampled_parity("qwen7b_b8_k64", 2)
+    assert stats["tainted_requests"] <= stats["requests"]
+
+
 @pytest.mark.parametrize("name", ["8b_b512", "8b_b512_stoch"])
 def test_8b_batch512_sampled(name):
     case, out, A, stats = _sampled_parity(name, 10)
