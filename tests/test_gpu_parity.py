@@ -329,12 +329,12 @@ def test_8b_batch1_full_oracle():
 
 @pytest.mark.parametrize("name", ["8b_b64_m30", "8b_b64", "8b_b64_m95"])
 def test_8b_batch64_sampled(name):
-    case, out, A, stats = _sampled_parity(name, 6)
+    case, out, A, stats = _sampled_parity(name, 16)
     assert stats["tainted_requests"] < stats["requests"]
 
 
 def test_8b_selective_hidden_sampled():
-    case, out, A, stats = _sampled_parity("8b_sh256", 12)
+    case, out, A, stats = _sampled_parity("8b_sh256", 24)
     assert stats["tainted_requests"] < stats["requests"]
 
 
@@ -351,7 +351,7 @@ def test_qwen_shapes_longest_window_sampled():
 
 @pytest.mark.parametrize("name", ["8b_b512", "8b_b512_stoch"])
 def test_8b_batch512_sampled(name):
-    case, out, A, stats = _sampled_parity(name, 10)
+    case, out, A, stats = _sampled_parity(name, 20)
     if name == "8b_b512":
         # i.i.d. per-position accept probability a = r' + (1 - r') P(p < tau): closed-form mean
         k = 16
