@@ -213,7 +213,10 @@ int wisv_profile_read(wisv_ctx* ctx, int32_t stage, float* ms, int32_t cap, int3
  * NULL restores the automatic plan.  The partial buffers are sized for any legal
  * setting; results do not depend on the plan beyond fp32 summation order.
  */
-typedef struct { int32_t lm_tile_n, lm_stages, head_tile_n, head_stages; } wisv_tuning;
+typedef struct {
+    int32_t lm_tile_n, lm_stages, head_tile_n, head_stages;
+    int32_t lm_single_cta;   /* 1: never use the CTA-pair LM-head kernel (batches with more than 128 window rows) */
+} wisv_tuning;
 int wisv_set_tuning(wisv_ctx* ctx, const wisv_tuning* tuning);
 
 /* Number of kernels this context has launched so far. */

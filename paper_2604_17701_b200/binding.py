@@ -50,7 +50,7 @@ class _Result(C.Structure):
 
 class _Tuning(C.Structure):
     _fields_ = [("lm_tile_n", C.c_int32), ("lm_stages", C.c_int32), ("head_tile_n", C.c_int32),
-                ("head_stages", C.c_int32)]
+                ("head_stages", C.c_int32), ("lm_single_cta", C.c_int32)]
 
 
 class LinkParams(C.Structure):
@@ -334,8 +334,9 @@ class Verifier:
         keys = ("lm_tile_n", "lm_tiles", "lm_ctas", "head_tile_n", "head_tiles", "head_ctas")
         return dict(zip(keys, (x.value for x in v)))
 
-    def set_tuning(self, lm_tile_n: int = 0, lm_stages: int = 0, head_tile_n: int = 0, head_stages: int = 0):
-        t = _Tuning(lm_tile_n, lm_stages, head_tile_n, head_stages)
+    def set_tuning(self, lm_tile_n: int = 0, lm_stages: int = 0, head_tile_n: int = 0, head_stages: int = 0,
+                   lm_single_cta: int = 0):
+        t = _Tuning(lm_tile_n, lm_stages, head_tile_n, head_stages, lm_single_cta)
         _check(self.lib.wisv_set_tuning(self._h, C.byref(t)), "wisv_set_tuning")
 
     def launch_count(self) -> int:

@@ -16,6 +16,7 @@
 #include "../../include/wisv.h"
 #include "wisv_aux.cuh"
 #include "wisv_gemm.cuh"
+#include "wisv_gemm2.cuh"
 
 using namespace wisv;
 
@@ -35,6 +36,7 @@ struct Plan {
     int a_rows;      // activation rows loaded per tile (8..128)
     int carry;       // one partial per (row, CTA) instead of per (row, N-tile)
     int parts;       // partials per row
+    int pair;        // LM head on CTA pairs (256 x 256 tiles): m_tiles then counts tiles of 256 rows
     int k_splits;    // work items per (m, n) tile along K (decision head with one row tile)
     int kb_per_split;
     size_t smem;
@@ -73,6 +75,7 @@ struct wisv_ctx {
     float* splitk_buf = nullptr;      // [sm_count][128][kSplitTileN] raw partial head tiles
     int32_t* splitk_count = nullptr;  // per (m, n) tile arrival counters, zero between calls
     int splitk_tiles = 0;
+    int max_pairs = 0;                // CTA pairs that can be resident at once
     int32_t* row_tok = nullptr; int32_t* row_flag = nullptr; float* tok_logit = nullptr;
     int32_t* pos_req = nullptr; int32_t* pos_i = nullptr;
     int32_t* err = nullptr;
@@ -90,7 +93,7 @@ struct wisv_ctx {
     long long prof_calls = 0;
     cudaEvent_t* prof_ev = nullptr;   // [prof_n][kStages + 1]
     long long launches = 0;
-    wisv_tuning tune = {0, 0, 0, 0};
+    wisv_tuning tune = {0, 0, 0, 0, 0};
     HostStaging hs;
 };
 
@@ -154,6 +157,30 @@ Plan plan_lm(const wisv_ctx* c, int R)
     Plan p{};
     const int V = c->cfg.V;
     p.m_tiles = (R + kTileM - 1) / kTileM;
+    // More than one row tile: CTA pairs on 256 x 256 tiles, each weight tile fetched once per pair.  A pair
+    // always computes 256 rows, so with an odd number of 128-row tiles its last tile is half padding:
+    // worth it with two row tiles (the launch is HBM-bound and the pair halves the weight fetches) and
+    // when the padding is a few per cent, not in between.
+    const bool pair_fits = p.m_tiles % 2 == 0 || p.m_tiles >= 33;
+    if (p.m_tiles >= 2 && pair_fits && c->max_pairs > 0 && !c->tune.lm_single_cta && !c->tune.lm_tile_n) {
+        p.pair = 1;
+        p.m_tiles = (R + kPairTileM - 1) / kPairTileM;
+        p.tile_n = kPairTileN;
+        p.n_tiles = (V + kPairTileN - 1) / kPairTileN;
+        p.a_rows = kTileM;
+        p.k_splits = 1;
+        p.kb_per_split = (c->cfg.H + kBlockK - 1) / kBlockK;
+        int s = (int)(((size_t)c->max_smem - pair_fixed_bytes()) / kPairStageBytes);
+        if (s > kMaxStages) s = kMaxStages;
+        if (c->tune.lm_stages >= 2 && c->tune.lm_stages < s) s = c->tune.lm_stages;
+        p.stages = s;
+        p.smem = pair_fixed_bytes() + (size_t)s * kPairStageBytes;
+        const long long tiles = (long long)p.m_tiles * p.n_tiles;
+        p.ctas = 2 * (int)(tiles < c->max_pairs ? tiles : c->max_pairs);
+        p.carry = 0;
+        p.parts = p.n_tiles;
+        return p;
+    }
     int best = 0;
     if (c->tune.lm_tile_n >= 16 && c->tune.lm_tile_n <= kMaxTileN && c->tune.lm_tile_n % 16 == 0) {
         best = c->tune.lm_tile_n;
@@ -377,6 +404,8 @@ int wisv_create(const wisv_config* cfg, const wisv_weights* w, wisv_ctx** out)
                                    (int)prop.sharedMemPerBlockOptin));
     WISV_CUDA(cudaFuncSetAttribute(gemm_rowreduce_kernel<EPI_RAW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)prop.sharedMemPerBlockOptin));
+    WISV_CUDA(cudaFuncSetAttribute(lmhead_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)prop.sharedMemPerBlockOptin));
 
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -391,10 +420,24 @@ int wisv_create(const wisv_config* cfg, const wisv_weights* w, wisv_ctx** out)
     c->device = dev;
     c->sm_count = prop.multiProcessorCount;
     c->max_smem = (int)prop.sharedMemPerBlockOptin;
+    {
+        // how many CTA pairs of the pair kernel fit on the device at once (sizes its persistent grid)
+        cudaLaunchConfig_t qc;
+        memset(&qc, 0, sizeof qc);
+        qc.gridDim = dim3(2 * prop.multiProcessorCount); qc.blockDim = dim3(kGemmThreads);
+        qc.dynamicSmemBytes = (size_t)prop.sharedMemPerBlockOptin;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, lmhead_pair_kernel, &qc) == cudaSuccess && n > 0) {
+            c->max_pairs = n < prop.multiProcessorCount / 2 ? n : prop.multiProcessorCount / 2;
+        } else {
+            (void)cudaGetLastError();
+            c->max_pairs = 0;          // pairs unavailable: the single-CTA kernel serves every size
+        }
+    }
     const int max_T = cfg->max_rows - 1;
     c->max_pos = cfg->max_sel > 0 ? (cfg->max_sel > max_T ? cfg->max_sel : max_T) : max_T;
     if (c->max_pos < 1) c->max_pos = 1;
-    c->rows_alloc = round_up(cfg->max_rows, kTileM);
+    c->rows_alloc = round_up(cfg->max_rows, kPairTileM);
     c->pos_alloc = round_up(c->max_pos, kTileM);
     const int hd_h = cfg->H_d + cfg->H;
 
@@ -489,7 +532,7 @@ int64_t wisv_launch_count(const wisv_ctx* c) { return c ? c->launches : 0; }
 int wisv_set_tuning(wisv_ctx* c, const wisv_tuning* t)
 {
     if (!c) return WISV_EINVAL;
-    if (!t) { c->tune = wisv_tuning{0, 0, 0, 0}; return WISV_OK; }
+    if (!t) { c->tune = wisv_tuning{0, 0, 0, 0, 0}; return WISV_OK; }
     const int32_t tn[2] = {t->lm_tile_n, t->head_tile_n};
     for (int i = 0; i < 2; ++i)
         if (tn[i] != 0 && (tn[i] < 16 || tn[i] > kMaxTileN || tn[i] % 16)) return WISV_ESHAPE;
@@ -546,7 +589,17 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
     if (ev) WISV_CUDA(cudaEventRecord(ev[1], st));
     const Plan pl = plan_lm(c, R);
     if ((size_t)R * pl.parts > c->lm_part_elems) return WISV_ECAPACITY;
-    if (phase != PHASE_DECIDE) {
+    if (phase != PHASE_DECIDE && pl.pair) {
+        PairParams qp;
+        memset(&qp, 0, sizeof qp);
+        qp.rows = R; qp.n_total = cf.V; qp.k_blocks = (cf.H + kBlockK - 1) / kBlockK; qp.mp_tiles = pl.m_tiles;
+        qp.n_tiles = pl.n_tiles; qp.stages = pl.stages; qp.part_stride = pl.parts; qp.err = c->err;
+        qp.lm_part = c->lm_part; qp.row_tok = c->row_tok; qp.tok_logit = c->tok_logit;
+        const int rc = launch_pdl(lmhead_pair_kernel, dim3(pl.ctas), dim3(kGemmThreads), pl.smem, st,
+                                  c->tmX[kNumRowVariants - 1], c->tmW[kTileM / 16 - 1], qp);
+        if (rc != WISV_OK) return rc;
+        c->launches++;
+    } else if (phase != PHASE_DECIDE) {
         GemmParams gp = base_params(c, pl, R, cf.V, cf.H);
         gp.lm_part = c->lm_part; gp.row_tok = c->row_tok; gp.tok_logit = c->tok_logit;
         const int rc = launch_gemm<EPI_LMHEAD>(c, c->tmX[pl.a_rows / 8 - 1], c->tmW[pl.tile_n / 16 - 1], gp, pl, st);

@@ -93,6 +93,36 @@ __device__ __forceinline__ float act_apply(float x, int act) {
     return 0.5f * x * (1.0f + erff(x * 0.70710678118654752440f));
 }
 
+// Online update of one row's (max, lowest argidx, sum exp) with 16 consecutive logits starting at
+// column col0 (columns >= n_total are padding), and capture of the logit at the row's draft token.
+__device__ __forceinline__ void lm_update_chunk(const uint32_t (&v)[16], int col0, int n_total, int tok,
+                                                float& mx, int& arg, float& sum, float* tok_logit_row)
+{
+    float f[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) f[j] = (col0 + j < n_total) ? __uint_as_float(v[j]) : -CUDART_INF_F;
+    float cm = f[0];
+    int ci = 0;
+#pragma unroll
+    for (int j = 1; j < 16; ++j) { if (f[j] > cm) { cm = f[j]; ci = j; } }
+    if (cm > mx) {                           // strict: earlier (lower) index wins ties
+        sum *= exp2f((mx - cm) * 1.4426950408889634f);
+        mx = cm;
+        arg = col0 + ci;
+    }
+    const float base = mx * 1.4426950408889634f;
+    float acc = 0.0f;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) acc += exp2f(fmaf(f[j], 1.4426950408889634f, -base));
+    sum += acc;
+    if (static_cast<unsigned>(tok - col0) < 16u) {
+        float tl = 0.0f;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) tl = (tok - col0 == j) ? f[j] : tl;
+        *tok_logit_row = tl;
+    }
+}
+
 template <int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -295,29 +325,7 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 if (!valid) continue;
                 const int col0 = n0 + c0;
                 if (EPI == EPI_LMHEAD) {
-                    float f[16];
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) f[j] = (col0 + j < p.n_total) ? __uint_as_float(v[j]) : -CUDART_INF_F;
-                    float cm = f[0];
-                    int ci = 0;
-#pragma unroll
-                    for (int j = 1; j < 16; ++j) { if (f[j] > cm) { cm = f[j]; ci = j; } }
-                    if (cm > mx) {                           // strict: earlier (lower) index wins ties
-                        sum *= exp2f((mx - cm) * 1.4426950408889634f);
-                        mx = cm;
-                        arg = col0 + ci;
-                    }
-                    const float base = mx * 1.4426950408889634f;
-                    float acc = 0.0f;
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) acc += exp2f(fmaf(f[j], 1.4426950408889634f, -base));
-                    sum += acc;
-                    if (static_cast<unsigned>(tok - col0) < 16u) {
-                        float tl = 0.0f;
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) tl = (tok - col0 == j) ? f[j] : tl;
-                        p.tok_logit[row] = tl;
-                    }
+                    lm_update_chunk(v, col0, p.n_total, tok, mx, arg, sum, p.tok_logit + row);
                 } else if (EPI == EPI_HEAD && p.k_splits > 1) {
                     // split K: park the raw partial tile; the last item of this (m, n) tile finishes it
                     float4* dst = reinterpret_cast<float4*>(

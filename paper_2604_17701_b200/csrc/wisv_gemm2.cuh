@@ -1,0 +1,200 @@
+// LM-head GEMM + row reduction on CTA pairs (tcgen05 cta_group::2), used when the batch has more
+// than one row tile.  Two CTAs of a cluster share one 256 x 256 output tile: CTA r holds rows
+// r*128 .. r*128+127 of the tile in its own TMEM and loads, per K block, its own 128 activation rows
+// and its half (128 rows) of the 256 weight rows - so every weight tile enters shared memory once
+// per pair instead of once per CTA, which is what limits the single-CTA kernel (shared-memory fill
+// and L2 -> SM traffic, and with it power).  One thread of the even CTA issues the MMAs for both.
+//
+// Barriers: full[s] lives in the leader and counts the bytes of both CTAs' loads; empty[s] and
+// acc_full[a] exist in both CTAs and are signalled by a multicast tcgen05.commit; acc_empty[a] lives in
+// the leader and is arrived on by the epilogue warps of both CTAs.  No load uses multicast.  Every
+// wait is bounded; both CTAs meet at a cluster barrier before TMEM is released.
+#pragma once
+
+#include "wisv_gemm.cuh"
+
+namespace wisv {
+
+constexpr int kPairTileM = 256;
+constexpr int kPairTileN = 256;
+constexpr uint32_t kPairStageBytes = 2u * kTileM * kBlockK * 2u;   // 128 activation rows + 128 weight rows
+
+struct PairParams {
+    int32_t rows;        // valid window rows
+    int32_t n_total;     // vocabulary size
+    int32_t k_blocks;
+    int32_t mp_tiles;    // row tiles of 256
+    int32_t n_tiles;     // vocabulary tiles of 256
+    int32_t stages;
+    int32_t part_stride; // partials per row (= n_tiles)
+    int32_t* err;
+    float4* lm_part;
+    const int32_t* row_tok;
+    float* tok_logit;
+};
+
+__host__ __device__ inline uint32_t pair_fixed_bytes() { return 1024u + 1024u; }   // alignment slack + barriers
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                   const PairParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;
+    uint8_t* smem = smem_raw + pad;
+    const uint32_t smem_base = raw_addr + pad;
+
+    const uint32_t rank = cluster_ctarank();
+    const bool leader = rank == 0;
+    const int pair_id = blockIdx.x >> 1;
+    const int n_pairs = gridDim.x >> 1;
+    const uint32_t half_bytes = kTileM * kBlockK * 2;                 // 16 KB
+    const uint32_t ring_bytes = kPairStageBytes * static_cast<uint32_t>(p.stages);
+
+    const uint32_t bar_base = smem_base + ring_bytes;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (kMaxStages + s); };
+    auto acc_full_bar = [&](int s) { return bar_base + 8u * (2 * kMaxStages + s); };
+    auto acc_empty_bar = [&](int s) { return bar_base + 8u * (2 * kMaxStages + 2 + s); };
+    const uint32_t drain_bar = bar_base + 8u * (2 * kMaxStages + 4);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + ring_bytes + 8 * (2 * kMaxStages + 5));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [0] abort, [1] drain scratch
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int total_tiles = p.mp_tiles * p.n_tiles;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(acc_full_bar(s), 1); mbar_init(acc_empty_bar(s), 8); }
+        mbar_init(drain_bar, 1);
+        abort_flag[0] = 0;
+        abort_flag[1] = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(smem_u32(tmem_slot), kTmemCols);
+        tmem_relinquish_pair();
+    }
+    // both CTAs' barriers and TMEM must exist before either touches the other's
+    tc_fence_before();
+    __syncwarp();
+    cluster_arrive();
+    cluster_wait();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    griddep_wait();                    // the pack kernel wrote the bf16 rows this kernel loads
+    griddep_launch_dependents();
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer (each CTA)
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            long long issued = 0;
+            bool ok = true;
+            for (int t = pair_id; t < total_tiles && ok; t += n_pairs) {
+                const int mp = t % p.mp_tiles, n = t / p.mp_tiles;
+                const int row0 = mp * kPairTileM + static_cast<int>(rank) * kTileM;
+                const int col0 = n * kPairTileN + static_cast<int>(rank) * kTileM;
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, kWaitLimitNs)) { ok = false; break; }
+                    const uint32_t a_dst = smem_base + kPairStageBytes * s;
+                    if (leader) mbar_expect_tx(full_bar(s), 2u * kPairStageBytes);   // both CTAs' bytes
+                    tma_load_2d_pair(a_dst, &tmA, kb * kBlockK, row0, full_bar(s));
+                    tma_load_2d_pair(a_dst + half_bytes, &tmB, kb * kBlockK, col0, full_bar(s));
+                    ++issued;
+                    if (++s == p.stages) { s = 0; ph ^= 1u; }
+                }
+            }
+            (void)issued;
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (lane == 0 && leader) {
+            const uint32_t idesc = idesc_bf16_f32(kPairTileM, kPairTileN);
+            int s = 0;
+            uint32_t ph = 0;
+            int local = 0;
+            bool ok = true;
+            for (int t = pair_id; t < total_tiles && ok; t += n_pairs, ++local) {
+                const int as = local & 1;
+                const uint32_t aph = (local >> 1) & 1u;
+                if (!mbar_wait_bounded(acc_empty_bar(as), aph ^ 1u, abort_flag, kWaitLimitNs)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(as * kAccCols);
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!mbar_wait_bounded(full_bar(s), ph, abort_flag, kWaitLimitNs)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_base + kPairStageBytes * s;
+                    const uint64_t a_desc = smem_desc_k128(a_addr);
+                    const uint64_t b_desc = smem_desc_k128(a_addr + half_bytes);
+#pragma unroll
+                    for (int k = 0; k < kBlockK / kUmmaK; ++k)
+                        umma_bf16_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    umma_commit_pair(empty_bar(s));          // frees the stage in both CTAs
+                    if (++s == p.stages) { s = 0; ph ^= 1u; }
+                }
+                if (ok) umma_commit_pair(acc_full_bar(as));  // accumulator ready in both CTAs
+            }
+            if (!ok) {
+                umma_commit_pair(drain_bar);
+                mbar_wait_bounded(drain_bar, 0, abort_flag + 1, kWaitLimitNs);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..5 of each CTA)
+        const int q = warp & 3;
+        int local = 0;
+        bool ok = true;
+        const uint32_t leader_acc_empty0 = mapa_u32(acc_empty_bar(0), 0);
+        const uint32_t leader_acc_empty1 = mapa_u32(acc_empty_bar(1), 0);
+        for (int t = pair_id; t < total_tiles && ok; t += n_pairs, ++local) {
+            const int mp = t % p.mp_tiles, n = t / p.mp_tiles;
+            const int as = local & 1;
+            const uint32_t aph = (local >> 1) & 1u;
+            const int row = mp * kPairTileM + static_cast<int>(rank) * kTileM + q * 32 + lane;
+            const bool valid = row < p.rows;
+            const int n0 = n * kPairTileN;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(as * kAccCols);
+
+            bool got = mbar_wait_bounded(acc_full_bar(as), aph, abort_flag, kWaitLimitNs);
+            got = __all_sync(0xffffffffu, got);
+            if (!got) { ok = false; break; }
+            tc_fence_after();
+
+            float mx = -CUDART_INF_F, sum = 0.0f;
+            int arg = 0;
+            const int tok = valid ? p.row_tok[row] : -1;
+            for (int c0 = 0; c0 < kPairTileN; c0 += 16) {
+                uint32_t v[16];
+                __syncwarp();
+                tmem_ld16(taddr + static_cast<uint32_t>(c0), v);
+                tmem_wait_ld();
+                if (!valid) continue;
+                lm_update_chunk(v, n0 + c0, p.n_total, tok, mx, arg, sum, p.tok_logit + row);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(as ? leader_acc_empty1 : leader_acc_empty0);
+            if (valid) p.lm_part[(size_t)row * p.part_stride + n] = make_float4(mx, __int_as_float(arg), sum, 0.0f);
+        }
+    }
+
+    // neither CTA may retire (or release TMEM) while its partner can still signal or read it
+    tc_fence_before();
+    __syncwarp();
+    cluster_arrive();
+    cluster_wait();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, kTmemCols);
+    }
+    if (threadIdx.x == 0 && abort_flag[0] != 0) atomicOr(p.err, 1);
+}
+
+}  // namespace wisv

@@ -70,6 +70,7 @@ def test_tiny_config(act, shift):
     dict(B=3, K=64, V=777),                    # longest window
     dict(B=40, K=4),                           # R = 200: two row tiles, ragged second tile
     dict(B=70, K=3, V=600, d_J=200),           # R = 280: three row tiles, head width not a tile multiple
+    dict(B=100, K=4, V=700),                   # R = 500: two pair tiles of 256 rows, the last one ragged
     dict(B=16, K=0, K_lo=1, K_hi=9),           # ragged windows
     dict(match_rate=1.0),                      # full-match windows accept K
     dict(match_rate=0.0),                      # every position a candidate
@@ -100,6 +101,23 @@ def test_split_k_head_matches_single_pass_head(kw):
     v.set_tuning()
     o3 = cases.run(v, d)
     assert torch.equal(o3.head_prob, out.head_prob)      # deterministic from call to call
+    v.close()
+
+
+def test_cta_pair_kernel_matches_single_cta_kernel():
+    """More than 128 window rows: the LM head runs on CTA pairs; the tuning switch forces the single-CTA kernel."""
+    cfg = _small(B=50, K=4, V=1000, seed=23)               # 250 rows: one pair tile, second CTA ragged
+    case, ref, out, _ = _run(cfg)
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d)
+    assert v.plan(case["R"], case["T"])["lm_tiles"] == 4    # ceil(1000 / 256) tiles of 256 x 256
+    v.set_tuning(lm_single_cta=1)
+    assert v.plan(case["R"], case["T"])["lm_tiles"] == 8
+    o2 = cases.run(v, d)
+    torch.cuda.synchronize()
+    assert v.device_error() == 0
+    assert torch.equal(o2.argmax, out.argmax) and torch.equal(o2.accept_len, out.accept_len)
+    assert float((o2.lse - out.lse).abs().max()) < 1e-5
     v.close()
 
 
