@@ -593,6 +593,14 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
         PairParams qp;
         memset(&qp, 0, sizeof qp);
         qp.rows = R; qp.n_total = cf.V; qp.k_blocks = (cf.H + kBlockK - 1) / kBlockK; qp.mp_tiles = pl.m_tiles;
+        {
+            // raster groups: keep a group's bf16 rows (256 x H x 2 bytes per row tile) within 32 MB of L2
+            const long long tile_bytes = (long long)kPairTileM * cf.H * 2;
+            int mg_max = (int)((32ll << 20) / tile_bytes);
+            if (mg_max < 1) mg_max = 1;
+            const int groups = (pl.m_tiles + mg_max - 1) / mg_max;
+            qp.m_group = (pl.m_tiles + groups - 1) / groups;
+        }
         qp.n_tiles = pl.n_tiles; qp.stages = pl.stages; qp.part_stride = pl.parts; qp.err = c->err;
         qp.lm_part = c->lm_part; qp.row_tok = c->row_tok; qp.tok_logit = c->tok_logit;
         const int rc = launch_pdl(lmhead_pair_kernel, dim3(pl.ctas), dim3(kGemmThreads), pl.smem, st,

@@ -24,6 +24,9 @@ struct PairParams {
     int32_t n_total;     // vocabulary size
     int32_t k_blocks;
     int32_t mp_tiles;    // row tiles of 256
+    int32_t m_group;     // row tiles per raster group: tiles run group by group (all vocabulary tiles of a
+                         // group of row tiles before the next group) so that the activation rows of a group
+                         // stay resident in L2 while the weights stream past them
     int32_t n_tiles;     // vocabulary tiles of 256
     int32_t stages;
     int32_t part_stride; // partials per row (= n_tiles)
@@ -64,6 +67,16 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int total_tiles = p.mp_tiles * p.n_tiles;
+    // tile t -> (row tile mp, vocabulary tile n): groups of m_group row tiles, row tile fastest inside a group
+    auto tile_mp_n = [&](int t, int* mp, int* n) {
+        const int per_group = p.m_group * p.n_tiles;
+        const int g = t / per_group;
+        const int mp0 = g * p.m_group;
+        const int gsize = min(p.m_group, p.mp_tiles - mp0);
+        const int idx = t - g * per_group;
+        *n = idx / gsize;
+        *mp = mp0 + idx % gsize;
+    };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -98,7 +111,8 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             long long issued = 0;
             bool ok = true;
             for (int t = pair_id; t < total_tiles && ok; t += n_pairs) {
-                const int mp = t % p.mp_tiles, n = t / p.mp_tiles;
+                int mp, n;
+                tile_mp_n(t, &mp, &n);
                 const int row0 = mp * kPairTileM + static_cast<int>(rank) * kTileM;
                 const int col0 = n * kPairTileN + static_cast<int>(rank) * kTileM;
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
@@ -154,7 +168,8 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         const uint32_t leader_acc_empty0 = mapa_u32(acc_empty_bar(0), 0);
         const uint32_t leader_acc_empty1 = mapa_u32(acc_empty_bar(1), 0);
         for (int t = pair_id; t < total_tiles && ok; t += n_pairs, ++local) {
-            const int mp = t % p.mp_tiles, n = t / p.mp_tiles;
+            int mp, n;
+            tile_mp_n(t, &mp, &n);
             const int as = local & 1;
             const uint32_t aph = (local >> 1) & 1u;
             const int row = mp * kPairTileM + static_cast<int>(rank) * kTileM + q * 32 + lane;
