@@ -300,6 +300,14 @@ int wisv_debug_logits(wisv_ctx* ctx, const float* target_hidden, int32_t R, floa
 int wisv_lm_head_reduce_static(const void* lm_head, int32_t V, int32_t H, const float* target_hidden, int32_t R,
                                int32_t* argmax, float* lse, void* cuda_stream);
 
+/*
+ * Test hook for the failure path (no counterpart in the paper): launches one small kernel that waits,
+ * with the bounded wait all pipeline waits in this library use, on a barrier nothing arrives on.  After
+ * limit_cycles SM clocks (<= 2e9) the wait gives up and sets bit 1 of the device error word, which
+ * wisv_device_error then reports and clears; the context stays usable.
+ */
+int wisv_debug_wait_probe(wisv_ctx* ctx, uint64_t limit_cycles, void* cuda_stream);
+
 const char* wisv_strerror(int code);
 int wisv_version(void);
 

@@ -117,6 +117,8 @@ def load_library(build_if_missing: bool = False):
     lib.wisv_launch_count.argtypes = [P]
     lib.wisv_plan.restype = C.c_int
     lib.wisv_plan.argtypes = [P, C.c_int32, C.c_int32] + [C.POINTER(C.c_int32)] * 6
+    lib.wisv_debug_wait_probe.restype = C.c_int
+    lib.wisv_debug_wait_probe.argtypes = [P, C.c_uint64, P]
     lib.wisv_debug_logits.restype = C.c_int
     lib.wisv_debug_logits.argtypes = [P, P, C.c_int32, P, P]
     lib.wisv_link_cost_round.restype = C.c_int
@@ -321,6 +323,11 @@ class Verifier:
         _check(self.lib.wisv_debug_logits(self._h, target_hidden.data_ptr(), R, out.data_ptr(),
                                           C.c_void_p(st.cuda_stream)), "wisv_debug_logits")
         return out
+
+    def wait_probe(self, limit_cycles: int):
+        st = self._torch.cuda.current_stream(self.device)
+        _check(self.lib.wisv_debug_wait_probe(self._h, limit_cycles, C.c_void_p(st.cuda_stream)),
+               "wisv_debug_wait_probe")
 
     def device_error(self) -> int:
         st = self._torch.cuda.current_stream(self.device)

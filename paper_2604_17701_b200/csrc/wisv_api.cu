@@ -545,6 +545,24 @@ int wisv_set_tuning(wisv_ctx* c, const wisv_tuning* t)
 
 namespace {
 
+// A barrier that nothing ever arrives on, waited for with the same bounded wait the GEMM kernels use:
+// the wait must give up after limit_cycles and report through the error word, leaving the context usable.
+__global__ void wait_probe_kernel(int32_t* err, unsigned long long limit_cycles)
+{
+    __shared__ uint64_t bar;
+    __shared__ int flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        flag = 0;
+        fence_barrier_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const bool ok = mbar_wait_bounded(smem_u32(&bar), 0, &flag, limit_cycles);
+        if (!ok) atomicOr(err, 2);
+    }
+}
+
 // One verification round, or one of its two phases (localize: pack rows + LM head + merge;
 // decide: pack positions + decision head + scan on the candidate sets the localize call saved).
 int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda_stream, int phase)
@@ -692,6 +710,15 @@ int wisv_debug_logits(wisv_ctx* c, const float* target_hidden, int32_t R, float*
     GemmParams gp = base_params(c, pl, R, c->cfg.V, c->cfg.H);
     gp.raw_out = logits_out;
     return launch_gemm<EPI_RAW>(c, c->tmX[pl.a_rows / 8 - 1], c->tmW[pl.tile_n / 16 - 1], gp, pl, st);
+}
+
+int wisv_debug_wait_probe(wisv_ctx* c, uint64_t limit_cycles, void* cuda_stream)
+{
+    if (!c || limit_cycles == 0 || limit_cycles > 2000000000ull) return WISV_EINVAL;
+    wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(c->err, limit_cycles);
+    WISV_CUDA(cudaGetLastError());
+    c->launches++;
+    return WISV_OK;
 }
 
 int wisv_device_error(wisv_ctx* c, void* cuda_stream, int32_t* flags)

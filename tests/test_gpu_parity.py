@@ -229,6 +229,22 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     v.close()
 
 
+def test_bounded_wait_gives_up_and_the_context_stays_usable():
+    cfg = _small(B=4, K=4, seed=29)
+    case = cases.make_case(cfg, oracle_ref_argmax)
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d)
+    ref = cases.run(v, d)
+    assert v.device_error() == 0
+    v.wait_probe(2_000_000)                       # about 1 ms: a barrier nobody arrives on
+    assert v.device_error() == 2                  # reported ...
+    assert v.device_error() == 0                  # ... and cleared
+    out = cases.run(v, d)                         # the context still works
+    torch.cuda.synchronize()
+    assert torch.equal(out.accept_len, ref.accept_len) and v.device_error() == 0
+    v.close()
+
+
 def test_capacity_and_argument_errors():
     cfg = _small(B=4, K=4)
     case = cases.make_case(cfg, oracle_ref_argmax)
