@@ -285,6 +285,9 @@ def run_ours(args, rank, world, local_rank):
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the verifier has no CPU path")
+    if local_rank == 0:
+        from paper_2604_17701_b200 import build as cuda_build
+        cuda_build.build()          # compiles the in-tree library only if it is missing or stale
     torch.cuda.set_device(local_rank)
     dev = "cuda:%d" % local_rank
     ranks = Ranks(world, "nccl", dev)

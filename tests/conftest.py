@@ -24,3 +24,12 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_libraries():
+    """Compile the CUDA library (nvcc) and the C oracle (gcc) if their in-tree binaries are missing or stale."""
+    from paper_2604_17701_b200 import build as cuda_build
+    import oracle
+    cuda_build.build()
+    oracle.build()
