@@ -291,6 +291,7 @@ def run_ours(args, rank, world, local_rank):
     torch.cuda.set_device(local_rank)
     dev = "cuda:%d" % local_rank
     ranks = Ranks(world, "nccl", dev)
+    ranks.barrier()                 # the other ranks load the library only after rank 0 has it in place
 
     cfg = workload_config(args.workload, rank)
     case = cases.make_case(cfg, lambda w, h: cases.library_ref_argmax(w, h, device=dev))
