@@ -186,7 +186,10 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     // pack output, which is complete by the time it can be scheduled (the LM-head kernel releases its
     // dependents only after its own wait); it waits at its end instead, so that "head kernel complete"
     // implies "LM-head kernel complete" for the merge/scan kernel that follows.
-    if (EPI != EPI_HEAD) griddep_wait();
+    // The producer thread of those kernels waits a little later: weight tiles do not depend on the
+    // pack kernel, so it first puts one ring-full of them in flight.
+    const bool producer_thread = warp == 0 && lane == 0;
+    if (EPI != EPI_HEAD && !producer_thread) griddep_wait();
     griddep_launch_dependents();
 
     if (warp == 0) {
@@ -196,15 +199,33 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             uint32_t ph = 0;
             long long issued = 0;
             bool ok = true;
+            long long pre = 0;                 // stages whose weight tile was requested before the wait
+            if (EPI != EPI_HEAD) {
+                for (int t = blockIdx.x; t < total_tiles && pre < p.stages; t += gridDim.x) {
+                    const int n = item_n(t);
+                    const int kb1 = item_kb1(t);
+                    for (int kb = item_kb0(t); kb < kb1 && pre < p.stages; ++kb, ++pre) {
+                        const uint32_t a_dst = smem_base + stage_bytes * static_cast<uint32_t>(pre);
+                        mbar_expect_tx(full_bar(static_cast<int>(pre)), stage_bytes);
+                        tma_load_2d(a_dst + a_bytes, &tmB, kb * kBlockK, n * p.tile_n, full_bar(static_cast<int>(pre)));
+                    }
+                }
+                griddep_wait();                // from here on the activation rows may be read
+            }
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
                 const int m = item_m(t), n = item_n(t);
                 const int kb1 = item_kb1(t);
                 for (int kb = item_kb0(t); kb < kb1; ++kb) {
-                    if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, kWaitLimitNs)) { ok = false; break; }
                     const uint32_t a_dst = smem_base + stage_bytes * s;
-                    mbar_expect_tx(full_bar(s), stage_bytes);
-                    tma_load_2d(a_dst, &tmA, kb * kBlockK, m * kTileM, full_bar(s));
-                    tma_load_2d(a_dst + a_bytes, &tmB, kb * kBlockK, n * p.tile_n, full_bar(s));
+                    if (issued < pre) {
+                        // first pass over the ring: the stage is free and its weight tile is already on its way
+                        tma_load_2d(a_dst, &tmA, kb * kBlockK, m * kTileM, full_bar(s));
+                    } else {
+                        if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, kWaitLimitNs)) { ok = false; break; }
+                        mbar_expect_tx(full_bar(s), stage_bytes);
+                        tma_load_2d(a_dst, &tmA, kb * kBlockK, m * kTileM, full_bar(s));
+                        tma_load_2d(a_dst + a_bytes, &tmB, kb * kBlockK, n * p.tile_n, full_bar(s));
+                    }
                     ++issued;
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
