@@ -97,6 +97,15 @@ class Ranks:
         self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
         return float(t.item())
 
+    def all_gather(self, gathered, part):
+        """gathered[g] = rank g's part (gathered: [world, ...] contiguous)."""
+        if self.dist is None:
+            gathered[0].copy_(part)
+        elif self.dist.get_backend() == "nccl":
+            self.dist.all_gather_into_tensor(gathered, part)
+        else:
+            self.dist.all_gather(list(gathered.unbind(0)), part)
+
     def close(self):
         if self.dist is not None:
             self.dist.destroy_process_group()
@@ -428,6 +437,105 @@ def run_ours(args, rank, world, local_rank):
     ranks.close()
 
 
+def shard_bounds(V, world):
+    """Vocabulary rows [lo, hi) of every rank: equal slices rounded to 16 rows."""
+    per = -(-V // world)
+    per = -(-per // 16) * 16
+    return [(min(V, r * per), min(V, (r + 1) * per)) for r in range(world)]
+
+
+def run_sharded(args, rank, world, local_rank):
+    """The same batch on every GPU, the LM head split by vocabulary: shard rows -> all-gather -> merge (strong scaling)."""
+    import torch
+    from paper_2604_17701_b200 import cases
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the verifier has no CPU path")
+    if local_rank == 0:
+        from paper_2604_17701_b200 import build as cuda_build
+        cuda_build.build()
+    torch.cuda.set_device(local_rank)
+    dev = "cuda:%d" % local_rank
+    ranks = Ranks(world, "nccl", dev)
+    ranks.barrier()
+    cfg = workload_config(args.workload)                   # one batch, seen by every rank
+    case = cases.make_case(cfg, lambda w, h: cases.library_ref_argmax(w, h, device=dev))
+    d = cases.to_device(case, dev)
+    lo, hi = shard_bounds(cfg.V, world)[rank]
+    if hi <= lo:
+        raise SystemExit("more GPUs than 16-row slices of the vocabulary")
+    v = cases.make_verifier(d, vocab_slice=(lo, hi))
+    T, R = case["T"], case["R"]
+    geo = dict(B=cfg.B, K=cfg.K if cfg.K_hi == 0 else 0, k_off=d["k_off_dev"], T=T)
+    part = torch.empty((R, 4), dtype=torch.float32, device=dev)
+    gathered = torch.empty((world, R, 4), dtype=torch.float32, device=dev)
+    res = None
+
+    def step():
+        nonlocal res
+        v.shard_rows(d["target_hidden"], d["draft_tokens"], out=part, **geo)
+        ranks.all_gather(gathered, part)                            # R * 16 bytes per GPU over NVLink
+        res = v.verify_gathered(gathered, d["target_hidden"], d["draft_tokens"], d["draft_hidden"], d["csi"],
+                                sel_off=d["sel_off"], sel_pos=d["sel_pos"], draft_q=d["draft_q"],
+                                uniforms=d["uniforms"], out=res, **geo)
+
+    stream = torch.cuda.current_stream()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize(); ranks.barrier(); torch.cuda.synchronize()
+    n0 = v.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize(); ranks.barrier(); torch.cuda.synchronize()
+    ms_step = ranks.max(e0.elapsed_time(e1) / args.steps)
+    launches = v.launch_count() - n0
+    # end to end: inputs from pinned host memory every step, accepted lengths read back
+    pin = lambda t: None if t is None else t.cpu().pin_memory()
+    host = {k: pin(d[k]) for k in ("target_hidden", "draft_tokens", "draft_hidden", "csi")}
+    e2e_steps = max(3, min(args.steps, 200))
+    back = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
+    torch.cuda.synchronize(); ranks.barrier()
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        for k, t in host.items():
+            d[k].copy_(t, non_blocking=True)
+        step()
+        back.copy_(res.accept_len, non_blocking=True)
+        torch.cuda.synchronize()
+    e1.record(stream)
+    torch.cuda.synchronize(); ranks.barrier()
+    e2e_ms = ranks.max(e0.elapsed_time(e1) / e2e_steps)
+    h2d = sum(int(t.numel() * t.element_size()) for t in host.values())
+    clocks = sampler.stop() if rank == 0 else None
+    if rank == 0:
+        peaks, peak_kind = load_peaks()
+        shard_bytes = (hi - lo) * cfg.H * 2
+        line = {"metric": METRIC, "value": T / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "strong",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": config_block(cfg, case, {"parallelism": "LM head sharded by vocabulary over %d GPU(s), "
+                                                                  "row partials all-gathered" % world,
+                                                   "vocab_rows_per_gpu": hi - lo}),
+                "clocks": clocks, "gpu_launches": int(launches),
+                "e2e": {"value": T / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                        "d2h_bytes_per_step": 4 * cfg.B, "ms_per_step": e2e_ms, "steps": e2e_steps},
+                "roofline": {"bound": "hbm", "achieved": None, "peak": float(peaks["hbm_gbs"]), "unit": "GB/s",
+                             "frac": None, "traffic": None, "peak_source": peak_kind,
+                             "algorithmic_bytes": shard_bytes,
+                             "note": "whole-step floor per GPU = shard bytes / peak = %.1f us" %
+                                     (shard_bytes / float(peaks["hbm_gbs"]) / 1e3)},
+                "mean_accept_len": float(res.accept_len.float().mean().item())}
+        print(json.dumps(line), flush=True)
+    v.close()
+    ranks.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -435,6 +543,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="8b_b1", choices=sorted(gen.CONFIGS))
+    ap.add_argument("--shard", default="requests", choices=["requests", "vocab"],
+                    help="multi-GPU split: independent batches per GPU (default), or one batch with the LM head "
+                         "sharded by vocabulary")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--oracle-seconds", type=float, default=10.0,
                     help="CPU-baseline leg: repeat the oracle round until this much time has passed")
@@ -457,7 +568,10 @@ def main():
         args.warmup = (5 if big else 50) if args.warmup is None else args.warmup
         args.warmup = max(3, args.warmup)
         args.oracle_rows = 800 if args.oracle_rows is None else args.oracle_rows
-        run_ours(args, rank, world, local_rank)
+        if args.shard == "vocab":
+            run_sharded(args, rank, world, local_rank)
+        else:
+            run_ours(args, rank, world, local_rank)
 
 
 if __name__ == "__main__":

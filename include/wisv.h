@@ -96,6 +96,8 @@ typedef struct {
     int32_t max_requests;   /* capacity: B */
     int32_t max_rows;       /* capacity: R = T + B */
     int32_t max_sel;        /* capacity: M_sel (SH); 0 = max_rows */
+    int32_t vocab_base;     /* vocabulary sharding: lm_head holds tokens [vocab_base, vocab_base + V) ... */
+    int32_t vocab_total;    /* ... of a vocabulary of vocab_total tokens; 0 = not sharded (vocab_base must be 0) */
 } wisv_config;
 
 typedef struct {
@@ -177,6 +179,30 @@ int wisv_verify(wisv_ctx* ctx, const wisv_batch* batch, const wisv_result* resul
  */
 int wisv_localize(wisv_ctx* ctx, const wisv_batch* batch, const wisv_result* result, void* cuda_stream);
 int wisv_decide(wisv_ctx* ctx, const wisv_batch* batch, const wisv_result* result, void* cuda_stream);
+
+/*
+ * The LM head sharded by vocabulary over several GPUs (each window is verified independently,
+ * Section II-A, and the logits of a row reduce associatively over the vocabulary): every GPU creates
+ * a context on its slice of the LM head (wisv_config.vocab_base / vocab_total) and on the whole
+ * decision head.
+ *
+ * wisv_shard_rows reduces this shard's logits of the R window rows to one 16-byte partial per row
+ * (out: dev [R]); it needs the same batch fields as wisv_localize.  The caller gathers the partials of
+ * all G shards into one dev array [G][R] (an all-gather of R * 16 bytes per GPU; any order of shards)
+ * and passes it to wisv_verify_gathered on the same context, which needs the batch fields of
+ * wisv_verify and completes the round: same outputs as wisv_verify on the unsharded LM head, argmax
+ * bit-identical outside exact ties between shards, log-sum-exp up to fp32 summation order.
+ */
+typedef struct {
+    float   max;        /* largest logit of the row in this shard */
+    int32_t argidx;     /* its global token id (lowest on ties) */
+    float   sumexp;     /* sum of exp(logit - max) over the shard */
+    float   tok_logit;  /* logit of the row's draft token if this shard owns it, else -inf */
+} wisv_row_partial;
+
+int wisv_shard_rows(wisv_ctx* ctx, const wisv_batch* batch, wisv_row_partial* out, void* cuda_stream);
+int wisv_verify_gathered(wisv_ctx* ctx, const wisv_batch* batch, const wisv_row_partial* gathered, int32_t n_shards,
+                         const wisv_result* result, void* cuda_stream);
 
 /*
  * Same round with HOST buffers: every pointer in `batch` and `result` is host

@@ -27,7 +27,8 @@ class WisvError(RuntimeError):
 class _Config(C.Structure):
     _fields_ = [("H", C.c_int32), ("V", C.c_int32), ("H_d", C.c_int32), ("d_c", C.c_int32), ("d_J", C.c_int32),
                 ("act", C.c_int32), ("head_row_shift", C.c_int32), ("tau", C.c_float),
-                ("max_requests", C.c_int32), ("max_rows", C.c_int32), ("max_sel", C.c_int32)]
+                ("max_requests", C.c_int32), ("max_rows", C.c_int32), ("max_sel", C.c_int32),
+                ("vocab_base", C.c_int32), ("vocab_total", C.c_int32)]
 
 
 class _Weights(C.Structure):
@@ -107,6 +108,10 @@ def load_library(build_if_missing: bool = False):
         f = getattr(lib, name)
         f.restype = C.c_int
         f.argtypes = [P, C.POINTER(_Batch), C.POINTER(_Result), P]
+    lib.wisv_shard_rows.restype = C.c_int
+    lib.wisv_shard_rows.argtypes = [P, C.POINTER(_Batch), P, P]
+    lib.wisv_verify_gathered.restype = C.c_int
+    lib.wisv_verify_gathered.argtypes = [P, C.POINTER(_Batch), P, C.c_int32, C.POINTER(_Result), P]
     lib.wisv_device_error.restype = C.c_int
     lib.wisv_device_error.argtypes = [P, P, C.POINTER(C.c_int32)]
     lib.wisv_profile_enable.restype = C.c_int
@@ -170,7 +175,8 @@ class Verifier:
     """
 
     def __init__(self, lm_head, W1, b1, w2, b2: float, *, H_d: int, d_c: int, act: int = ACT_GELU,
-                 tau: float = 0.5, head_row_shift: int = 0, max_requests: int, max_rows: int, max_sel: int = 0):
+                 tau: float = 0.5, head_row_shift: int = 0, max_requests: int, max_rows: int, max_sel: int = 0,
+                 vocab_base: int = 0, vocab_total: int = 0):
         import torch
         self._torch = torch
         self.lib = load_library()
@@ -184,7 +190,8 @@ class Verifier:
         self.H, self.V, self.H_d, self.d_c, self.d_J = H, V, H_d, d_c, d_J
         self._keep = (lm_head, W1, b1, w2)
         self.device = lm_head.device
-        cfg = _Config(H, V, H_d, d_c, d_J, act, head_row_shift, tau, max_requests, max_rows, max_sel)
+        cfg = _Config(H, V, H_d, d_c, d_J, act, head_row_shift, tau, max_requests, max_rows, max_sel,
+                      vocab_base, vocab_total)
         w = _Weights(lm_head.data_ptr(), W1.data_ptr(), b1.data_ptr(), w2.data_ptr(), float(b2))
         h = C.c_void_p()
         with torch.cuda.device(self.device):
@@ -291,6 +298,44 @@ class Verifier:
         r = self._result(out)
         st = stream if stream is not None else torch.cuda.current_stream(self.device)
         _check(self.lib.wisv_decide(self._h, C.byref(b), C.byref(r), C.c_void_p(st.cuda_stream)), "wisv_decide")
+        return out
+
+    def shard_rows(self, target_hidden, draft_tokens, *, B: int, K: int = 0, k_off=None, T: Optional[int] = None,
+                   out=None, stream=None):
+        """wisv_shard_rows: this vocabulary shard's per-row partials, a float32 tensor [R, 4] (16 bytes per row)."""
+        torch = self._torch
+        if T is None:
+            T = B * K if k_off is None else int(draft_tokens.shape[0])
+        if out is None:
+            out = torch.empty((T + B, 4), dtype=torch.float32, device=self.device)
+        b = self._batch(B=B, K=K, k_off=k_off, T=T, target_hidden=target_hidden, draft_tokens=draft_tokens,
+                        draft_hidden=None, csi=None, sel_off=None, sel_pos=None, draft_q=None, uniforms=None,
+                        tau=None)
+        st = stream if stream is not None else torch.cuda.current_stream(self.device)
+        _check(self.lib.wisv_shard_rows(self._h, C.byref(b), out.data_ptr(), C.c_void_p(st.cuda_stream)),
+               "wisv_shard_rows")
+        return out
+
+    def verify_gathered(self, gathered, target_hidden, draft_tokens, draft_hidden, csi, *, B: int, K: int = 0,
+                        k_off=None, T: Optional[int] = None, sel_off=None, sel_pos=None, draft_q=None,
+                        uniforms=None, tau: Optional[float] = None, out: Optional[VerifyOutput] = None,
+                        stream=None) -> VerifyOutput:
+        """wisv_verify_gathered: gathered is float32 [G, R, 4], the partials of all G vocabulary shards."""
+        torch = self._torch
+        if T is None:
+            T = B * K if k_off is None else int(draft_tokens.shape[0])
+        R = T + B
+        P = int(sel_pos.shape[0]) if sel_pos is not None else T
+        G = int(gathered.shape[0])
+        if out is None:
+            out = self._outputs(B, R, T, P, self.device, True)
+        b = self._batch(B=B, K=K, k_off=k_off, T=T, target_hidden=target_hidden, draft_tokens=draft_tokens,
+                        draft_hidden=draft_hidden, csi=csi, sel_off=sel_off, sel_pos=sel_pos, draft_q=draft_q,
+                        uniforms=uniforms, tau=tau)
+        r = self._result(out)
+        st = stream if stream is not None else torch.cuda.current_stream(self.device)
+        _check(self.lib.wisv_verify_gathered(self._h, C.byref(b), gathered.data_ptr(), G, C.byref(r),
+                                             C.c_void_p(st.cuda_stream)), "wisv_verify_gathered")
         return out
 
     def verify_host(self, target_hidden, draft_tokens, draft_hidden, csi, *, B: int, K: int = 0, k_off=None,

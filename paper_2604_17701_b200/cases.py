@@ -91,8 +91,16 @@ def to_device(case: Dict[str, object], device="cuda:0") -> Dict[str, object]:
 
 def make_verifier(dcase: Dict[str, object], *, act: Optional[str] = None, tau: Optional[float] = None,
                   head_row_shift: int = 0, max_requests: Optional[int] = None, max_rows: Optional[int] = None,
-                  max_sel: int = 0) -> binding.Verifier:
+                  max_sel: int = 0, vocab_slice=None) -> binding.Verifier:
     cfg = dcase["cfg"]
+    if vocab_slice is not None:
+        # a context on rows [lo, hi) of the LM head (one vocabulary shard)
+        lo, hi = vocab_slice
+        return binding.Verifier(dcase["lm_head"][lo:hi], dcase["W1"], dcase["b1"], dcase["w2"], float(dcase["b2"]),
+                                H_d=cfg.H_d, d_c=cfg.d_c, act=ACT[act or cfg.act],
+                                tau=cfg.tau if tau is None else tau, head_row_shift=head_row_shift,
+                                max_requests=max_requests or cfg.B, max_rows=max_rows or dcase["R"],
+                                max_sel=max_sel, vocab_base=lo, vocab_total=cfg.V)
     return binding.Verifier(dcase["lm_head"], dcase["W1"], dcase["b1"], dcase["w2"], float(dcase["b2"]),
                             H_d=cfg.H_d, d_c=cfg.d_c, act=ACT[act or cfg.act],
                             tau=cfg.tau if tau is None else tau, head_row_shift=head_row_shift,

@@ -274,12 +274,12 @@ int dev_alloc(T** p, size_t n)
     return WISV_OK;
 }
 
-enum { PHASE_FULL = 0, PHASE_LOCALIZE = 1, PHASE_DECIDE = 2 };
+enum { PHASE_FULL = 0, PHASE_LOCALIZE = 1, PHASE_DECIDE = 2, PHASE_GATHERED = 3, PHASE_SHARD = 4 };
 
 int validate_batch(const wisv_ctx* c, const wisv_batch* b, const wisv_result* r, int* T_out, int* R_out, int* P_out,
                    int phase = PHASE_FULL)
 {
-    if (!c || !b || !r) return WISV_EINVAL;
+    if (!c || !b || (!r && phase != PHASE_SHARD)) return WISV_EINVAL;
     if (b->B < 0 || b->K < 0) return WISV_ESHAPE;
     if (b->mode & ~3u) return WISV_EINVAL;
     const bool sh = (b->mode & WISV_MODE_SH) != 0;
@@ -293,7 +293,7 @@ int validate_batch(const wisv_ctx* c, const wisv_batch* b, const wisv_result* r,
     const long long R = T + b->B;
     if (b->B > c->cfg.max_requests || R > c->cfg.max_rows) return WISV_ECAPACITY;
     long long P = T;
-    if (phase == PHASE_LOCALIZE) {
+    if (phase == PHASE_LOCALIZE || phase == PHASE_SHARD) {
         P = 0;
     } else if (sh) {
         if (b->M_sel < 0) return WISV_ESHAPE;
@@ -305,10 +305,12 @@ int validate_batch(const wisv_ctx* c, const wisv_batch* b, const wisv_result* r,
     if (P > c->max_pos) return WISV_ECAPACITY;
     if (b->B > 0) {
         if (!b->target_hidden) return WISV_EINVAL;
-        if (phase != PHASE_LOCALIZE && (!r->accept_len || !r->correction_token)) return WISV_EINVAL;
+        if (phase != PHASE_LOCALIZE && phase != PHASE_SHARD && (!r || !r->accept_len || !r->correction_token))
+            return WISV_EINVAL;
         if (phase != PHASE_DECIDE && T > 0 && !b->draft_tokens) return WISV_EINVAL;
         if (P > 0 && (!b->draft_hidden || (c->cfg.d_c > 0 && !b->csi))) return WISV_EINVAL;
-        if (phase != PHASE_DECIDE && stoch && T > 0 && (!b->draft_q || !b->uniforms)) return WISV_EINVAL;
+        if (phase != PHASE_DECIDE && phase != PHASE_SHARD && stoch && T > 0 && (!b->draft_q || !b->uniforms))
+            return WISV_EINVAL;
         if (!aligned16(b->target_hidden) || (P > 0 && !aligned16(b->draft_hidden))) return WISV_EALIGN;
     }
     if (!(b->tau != b->tau) && b->tau < 0.0f) return WISV_EINVAL;
@@ -387,6 +389,9 @@ int wisv_create(const wisv_config* cfg, const wisv_weights* w, wisv_ctx** out)
     if (!(cfg->tau >= 0.0f)) return WISV_EINVAL;
     if (cfg->H < 64 || cfg->H % 8 || cfg->H_d < 8 || cfg->H_d % 8 || cfg->V < 1 || cfg->d_J < 1) return WISV_ESHAPE;
     if (cfg->d_c < 0 || cfg->d_c > WISV_MAX_DC) return WISV_ESHAPE;
+    if (cfg->vocab_base < 0 || cfg->vocab_total < 0) return WISV_ESHAPE;
+    if (cfg->vocab_total > 0 && (long long)cfg->vocab_base + cfg->V > cfg->vocab_total) return WISV_ESHAPE;
+    if (cfg->vocab_total == 0 && cfg->vocab_base != 0) return WISV_ESHAPE;
     if (cfg->max_requests < 1 || cfg->max_rows < cfg->max_requests || cfg->max_sel < 0) return WISV_ESHAPE;
     if ((long long)cfg->max_rows > (long long)(WISV_MAX_K + 1) * cfg->max_requests) return WISV_ESHAPE;
     if (!aligned16(w->lm_head)) return WISV_EALIGN;
@@ -565,12 +570,13 @@ __global__ void wait_probe_kernel(int32_t* err, unsigned long long limit_cycles)
 
 // One verification round, or one of its two phases (localize: pack rows + LM head + merge;
 // decide: pack positions + decision head + scan on the candidate sets the localize call saved).
-int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda_stream, int phase)
+int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda_stream, int phase,
+              float4* shard_out = nullptr, const float4* gathered = nullptr, int n_shards = 0)
 {
     int T = 0, R = 0, P = 0;
     const int vrc = validate_batch(c, b, r, &T, &R, &P, phase);
     if (vrc != WISV_OK) return vrc;
-    if (phase == PHASE_DECIDE) {
+    if (phase == PHASE_DECIDE || phase == PHASE_GATHERED) {
         if (!c->loc_valid) return WISV_EINVAL;
         if (b->B != c->loc_B || T != c->loc_T || (b->k_off ? 0 : b->K) != c->loc_K || b->k_off != c->loc_k_off)
             return WISV_ESHAPE;
@@ -590,7 +596,9 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
     if (ev) WISV_CUDA(cudaEventRecord(ev[0], st));
     PackParams pp;
     memset(&pp, 0, sizeof pp);
-    const int pack_rows = phase == PHASE_DECIDE ? 0 : R;
+    const bool rows_done = phase == PHASE_DECIDE || phase == PHASE_GATHERED;   // reduced by an earlier call
+    const int pack_rows = rows_done ? 0 : R;
+    pp.vocab_base = cf.vocab_base; pp.vocab_total = cf.vocab_total > 0 ? cf.vocab_total : cf.V;
     pp.ix = ix; pp.R = pack_rows; pp.P = P; pp.H = cf.H; pp.H_d = cf.H_d; pp.V = cf.V; pp.shift = cf.head_row_shift;
     pp.mode_sh = sh ? 1 : 0;
     pp.target_hidden = b->target_hidden; pp.draft_hidden = b->draft_hidden; pp.draft_tokens = b->draft_tokens;
@@ -607,7 +615,7 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
     if (ev) WISV_CUDA(cudaEventRecord(ev[1], st));
     const Plan pl = plan_lm(c, R);
     if ((size_t)R * pl.parts > c->lm_part_elems) return WISV_ECAPACITY;
-    if (phase != PHASE_DECIDE && pl.pair) {
+    if (!rows_done && pl.pair) {
         PairParams qp;
         memset(&qp, 0, sizeof qp);
         qp.rows = R; qp.n_total = cf.V; qp.k_blocks = (cf.H + kBlockK - 1) / kBlockK; qp.mp_tiles = pl.m_tiles;
@@ -625,11 +633,22 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
                                   c->tmX[kNumRowVariants - 1], c->tmW[kTileM / 16 - 1], qp);
         if (rc != WISV_OK) return rc;
         c->launches++;
-    } else if (phase != PHASE_DECIDE) {
+    } else if (!rows_done) {
         GemmParams gp = base_params(c, pl, R, cf.V, cf.H);
         gp.lm_part = c->lm_part; gp.row_tok = c->row_tok; gp.tok_logit = c->tok_logit;
         const int rc = launch_gemm<EPI_LMHEAD>(c, c->tmX[pl.a_rows / 8 - 1], c->tmW[pl.tile_n / 16 - 1], gp, pl, st);
         if (rc != WISV_OK) return rc;
+    }
+
+    if (phase == PHASE_SHARD) {
+        // this shard's rows reduced to one partial each; the caller gathers them across shards
+        const int rc = launch_pdl(shard_rows_kernel, dim3((R + 3) / 4), dim3(128), 0, st,
+                                  (const float4*)c->lm_part, pl.parts, R, (int)cf.vocab_base,
+                                  (const int32_t*)c->row_tok, (const float*)c->tok_logit, shard_out);
+        if (rc != WISV_OK) return rc;
+        c->launches++;
+        c->loc_valid = true; c->loc_B = b->B; c->loc_T = T; c->loc_K = b->k_off ? 0 : b->K; c->loc_k_off = b->k_off;
+        return WISV_OK;
     }
 
     // ---- 3. decision head on the evaluated positions
@@ -651,8 +670,13 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
     memset(&tp, 0, sizeof tp);
     tp.ix = ix; tp.P = P; tp.V = cf.V; tp.n_tiles_lm = pl.parts; tp.n_tiles_head = ph.parts; tp.mode_sh = sh ? 1 : 0;
     tp.phase = phase; tp.saved_arg = c->saved_arg; tp.saved_mask = c->saved_mask;
+    tp.vocab_base = cf.vocab_base; tp.part_rstride = pl.parts; tp.part_nstride = 1;
     tp.stochastic = stoch ? 1 : 0; tp.b2 = c->w.b2; tp.tau = (b->tau != b->tau) ? cf.tau : b->tau;
-    tp.lm_part = c->lm_part; tp.tok_logit = c->tok_logit; tp.row_flag = c->row_flag; tp.draft_tokens = b->draft_tokens;
+    tp.lm_part = c->lm_part;
+    if (phase == PHASE_GATHERED) {
+        tp.lm_part = gathered; tp.n_tiles_lm = n_shards; tp.part_rstride = 1; tp.part_nstride = R;
+    }
+    tp.tok_logit = c->tok_logit; tp.row_flag = c->row_flag; tp.draft_tokens = b->draft_tokens;
     tp.head_part = c->head_part; tp.pos_i = c->pos_i; tp.sel_off = b->sel_off; tp.draft_q = b->draft_q;
     tp.uniforms = b->uniforms;
     tp.accept_len = r->accept_len; tp.correction = r->correction_token; tp.argmax = r->argmax; tp.lse = r->lse;
@@ -690,6 +714,20 @@ int wisv_localize(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* 
 int wisv_decide(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda_stream)
 {
     return run_round(c, b, r, cuda_stream, PHASE_DECIDE);
+}
+
+int wisv_shard_rows(wisv_ctx* c, const wisv_batch* b, wisv_row_partial* out, void* cuda_stream)
+{
+    if (!out) return WISV_EINVAL;
+    return run_round(c, b, nullptr, cuda_stream, PHASE_SHARD, reinterpret_cast<float4*>(out));
+}
+
+int wisv_verify_gathered(wisv_ctx* c, const wisv_batch* b, const wisv_row_partial* gathered, int32_t n_shards,
+                         const wisv_result* r, void* cuda_stream)
+{
+    if (!gathered || n_shards < 1 || n_shards > 1024) return WISV_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(gathered) & 15u) != 0) return WISV_EALIGN;
+    return run_round(c, b, r, cuda_stream, PHASE_GATHERED, nullptr, reinterpret_cast<const float4*>(gathered), n_shards);
 }
 
 int wisv_debug_logits(wisv_ctx* c, const float* target_hidden, int32_t R, float* logits_out, void* cuda_stream)

@@ -39,6 +39,7 @@ struct BatchIndex {
 struct PackParams {
     BatchIndex ix;
     int32_t R, P, H, H_d, V, shift, mode_sh;
+    int32_t vocab_base, vocab_total;   // this context's LM-head rows are tokens [vocab_base, vocab_base + V) of vocab_total
     const float* target_hidden;   // [R, H]
     const float* draft_hidden;    // [P, H_d]
     const int32_t* draft_tokens;  // [T]
@@ -83,7 +84,9 @@ __global__ void __launch_bounds__(256) pack_kernel(const PackParams p)
             int tok = -1, flag = 0;
             if (i < Kb) {
                 tok = p.draft_tokens[p.ix.koff(b) + i];
-                if (tok < 0 || tok >= p.V) { flag = 2; tok = tok < 0 ? 0 : p.V - 1; }
+                if (tok < 0 || tok >= p.vocab_total) { flag = 2; tok = tok < 0 ? 0 : p.vocab_total - 1; }
+                tok -= p.vocab_base;                       // row index in this context's LM head
+                if (tok < 0 || tok >= p.V) tok = -1;       // another shard owns the token
             }
             p.row_tok[r] = tok;
             p.row_flag[r] = flag;
@@ -129,7 +132,10 @@ __global__ void split_w1_kernel(const __nv_bfloat16* __restrict__ W1, __nv_bfloa
 struct TailParams {
     BatchIndex ix;
     int32_t P, V, n_tiles_lm, n_tiles_head, mode_sh, stochastic;
-    int32_t phase;                // 0: whole round; 1: localize only (no head); 2: decide from a saved localize
+    int32_t phase;                // 0: whole round; 1: localize only (no head); 2: decide from a saved localize;
+                                  // 3: whole round on per-shard row partials gathered from G vocabulary shards
+    int32_t vocab_base;           // added to the argidx of per-tile partials (phases 0 and 1)
+    int32_t part_rstride, part_nstride;   // partial of (row r, part n) is lm_part[r * part_rstride + n * part_nstride]
     int32_t* saved_arg;           // [R] argmax per window row kept between the two phases
     unsigned long long* saved_mask;  // [B] candidate set S per request kept between the two phases
     float b2, tau;
@@ -164,6 +170,7 @@ __global__ void __launch_bounds__(256) tail_kernel(const TailParams p)
     constexpr int kMaxK = 64;
     __shared__ int s_arg[kMaxK + 1];
     __shared__ float s_lse[kMaxK + 1];
+    __shared__ float s_tl[kMaxK + 1];            // logit of the draft token (gathered flow: from the owning shard)
     __shared__ float s_prob[kMaxK];
     __shared__ int s_has[kMaxK];
     __shared__ int s_flag;
@@ -190,9 +197,20 @@ __global__ void __launch_bounds__(256) tail_kernel(const TailParams p)
     for (int i = warp; i <= Kb && p.phase != 2; i += nwarps) {
         const int r = r0 + i;
         RowStat st{-CUDART_INF_F, 0x7fffffff, 0.0f};
+        float tl = -CUDART_INF_F;
+        if (p.phase == 3) {
+            // one partial per vocabulary shard: {max, global argidx, sumexp, draft-token logit or -inf}
+            for (int n = lane; n < p.n_tiles_lm; n += 32) {
+                const float4 v = p.lm_part[(size_t)r * p.part_rstride + (size_t)n * p.part_nstride];
+                merge_stat(st, v.x, __float_as_int(v.y), v.z);
+                tl = fmaxf(tl, v.w);
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) tl = fmaxf(tl, __shfl_xor_sync(0xffffffffu, tl, off));
+        }
         const float4* part = p.lm_part + (size_t)r * p.n_tiles_lm;
         // four independent loads in flight per lane before the dependent merges
-        int n = lane;
+        int n = p.phase == 3 ? p.n_tiles_lm : lane;
         for (; n + 96 < p.n_tiles_lm; n += 128) {
             const float4 v0 = part[n], v1 = part[n + 32], v2 = part[n + 64], v3 = part[n + 96];
             merge_stat(st, v0.x, __float_as_int(v0.y), v0.z);
@@ -212,9 +230,11 @@ __global__ void __launch_bounds__(256) tail_kernel(const TailParams p)
             merge_stat(st, omx, oidx, osum);
         }
         const float l = st.mx + logf(st.sum);
+        if (p.phase != 3) st.idx += p.vocab_base;
         if (lane == 0) {
             s_arg[i] = st.idx;
             s_lse[i] = l;
+            s_tl[i] = p.phase == 3 ? tl : p.tok_logit[r];
             if (p.phase == 1) p.saved_arg[r] = st.idx;
             if (p.argmax) p.argmax[r] = st.idx;
             if (p.lse) p.lse[r] = l;
@@ -258,7 +278,7 @@ __global__ void __launch_bounds__(256) tail_kernel(const TailParams p)
                 if (p.phase == 2) {
                     cand = (p.saved_mask[b] >> i) & 1ull;
                 } else {
-                    const float pd = expf(p.tok_logit[r0 + i] - s_lse[i]);
+                    const float pd = expf(s_tl[i] - s_lse[i]);
                     if (p.p_draft) p.p_draft[t] = pd;
                     if (p.stochastic) {
                         const float alpha = fminf(1.0f, pd / p.draft_q[t]);
@@ -287,6 +307,38 @@ __global__ void __launch_bounds__(256) tail_kernel(const TailParams p)
             if (p.status) p.status[b] = s_flag | (missing ? 1 : 0);
         }
     }
+}
+
+}  // namespace wisv
+
+namespace wisv {
+
+// Vocabulary-sharded LM head: reduce the per-tile partials of this shard to one partial per window row,
+// {max, global argidx, sumexp, logit of the draft token if this shard owns it else -inf}.
+__global__ void __launch_bounds__(128) shard_rows_kernel(const float4* __restrict__ lm_part, int n_parts, int R,
+                                                         int vocab_base, const int32_t* __restrict__ row_tok,
+                                                         const float* __restrict__ tok_logit, float4* __restrict__ out)
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (r >= R) return;
+    RowStat st{-CUDART_INF_F, 0x7fffffff, 0.0f};
+    for (int n = lane; n < n_parts; n += 32) {
+        const float4 v = lm_part[(size_t)r * n_parts + n];
+        merge_stat(st, v.x, __float_as_int(v.y), v.z);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const float omx = __shfl_xor_sync(0xffffffffu, st.mx, off);
+        const int oidx = __shfl_xor_sync(0xffffffffu, st.idx, off);
+        const float osum = __shfl_xor_sync(0xffffffffu, st.sum, off);
+        merge_stat(st, omx, oidx, osum);
+    }
+    if (lane == 0)
+        out[r] = make_float4(st.mx, __int_as_float(st.idx + vocab_base), st.sum,
+                             row_tok[r] >= 0 ? tok_logit[r] : -CUDART_INF_F);
 }
 
 }  // namespace wisv

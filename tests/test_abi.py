@@ -40,7 +40,7 @@ def test_version_and_error_strings(lib):
 
 def test_struct_layouts_match_the_header():
     # field order and types mirror include/wisv.h; sizes follow the C ABI on x86-64
-    assert C.sizeof(binding._Config) == 11 * 4
+    assert C.sizeof(binding._Config) == 13 * 4
     assert C.sizeof(binding._Weights) == 4 * 8 + 8
     assert C.sizeof(binding._Result) == 9 * 8
     assert binding._Batch.k_off.offset == 8 and binding._Batch.target_hidden.offset == 24
@@ -61,7 +61,7 @@ def test_argument_errors_need_no_device(lib):
     assert lib.wisv_destroy(None) == -1
     assert lib.wisv_verify(None, None, None, None) == -1
     assert lib.wisv_launch_count(None) == 0
-    cfg = binding._Config(4096, 128256, 2048, 2, 1024, 7, 0, 0.5, 1, 9, 0)     # bad activation enum
+    cfg = binding._Config(4096, 128256, 2048, 2, 1024, 7, 0, 0.5, 1, 9, 0, 0, 0)     # bad activation enum
     w = binding._Weights(16, 16, 16, 16, 0.0)
     assert lib.wisv_create(C.byref(cfg), C.byref(w), C.byref(h)) == -1
     cfg.act = 1

@@ -58,3 +58,35 @@ def test_reference_arm_prints_one_line_from_rank_zero_only():
     assert rec["cpu_baseline"]["kind"] == "oracle" and rec["cpu_baseline"]["value"] == rec["value"]
     assert rec["e2e"]["h2d_bytes_per_step"] == 0 and rec["e2e"]["value"] == rec["value"]
     assert rec["config"]["workload"] == "tiny" and rec["vs_baseline"] is None
+
+
+def test_vocabulary_shard_bounds_cover_the_vocabulary_once():
+    import bench
+    for V, G in ((128256, 1), (128256, 2), (128256, 8), (152064, 4), (4099, 3), (100, 8)):
+        b = bench.shard_bounds(V, G)
+        assert len(b) == G and b[0][0] == 0 and b[-1][1] == V
+        assert all(lo <= hi for lo, hi in b) and all(b[i][1] == b[i + 1][0] for i in range(G - 1))
+        assert all(lo % 16 == 0 for lo, hi in b if hi > lo)          # non-empty slices start on a 16-row boundary
+
+
+def test_row_partials_are_gathered_rank_major_with_two_gloo_ranks(tmp_path):
+    script = tmp_path / "gather.py"
+    script.write_text(textwrap.dedent("""
+        import json, os, sys
+        sys.path.insert(0, %r)
+        import torch, bench
+        rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+        r = bench.Ranks(world, backend="gloo")
+        R = 5
+        part = torch.full((R, 4), float(rank)) + torch.arange(R).float()[:, None] * 10     # [R, 4] per rank
+        gathered = torch.empty((world, R, 4))
+        r.all_gather(gathered, part)                           # the layout wisv_verify_gathered expects: [G][R]
+        ok = all(bool((gathered[g] == torch.full((R, 4), float(g)) + torch.arange(R).float()[:, None] * 10).all())
+                 for g in range(world))
+        print(json.dumps({"rank": rank, "ok": ok, "shape": list(gathered.shape)}), flush=True)
+        r.close()
+    """ % ROOT))
+    out = _torchrun(2, [str(script)])
+    assert out.returncode == 0, out.stderr[-2000:]
+    recs = [json.loads(l) for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(recs) == 2 and all(r["ok"] and r["shape"] == [2, 5, 4] for r in recs)
