@@ -206,8 +206,8 @@ def pack_selective(draft_hidden: np.ndarray, k_len: np.ndarray, select: np.ndarr
     select = np.asarray(select, dtype=bool)
     idx = np.nonzero(select)[0]
     sel_off = np.zeros(len(k_len) + 1, dtype=np.int32)
-    counts = np.add.reduceat(select.astype(np.int64), k_off[:-1]) if select.size else np.zeros(len(k_len))
-    counts = np.where(np.asarray(k_len) > 0, counts, 0)
+    req_all = np.repeat(np.arange(len(k_len)), np.asarray(k_len, dtype=np.int64))
+    counts = np.bincount(req_all, weights=select.astype(np.float64), minlength=len(k_len)).astype(np.int64)
     sel_off[1:] = np.cumsum(counts)
     req = np.searchsorted(k_off[1:], idx, side="right")
     sel_pos = (idx - k_off[req]).astype(np.int32)

@@ -191,8 +191,7 @@ def verify(*, lm_head_bits, W1_bits, b1, w2, b2, act, tau, k_len, target_hidden,
     prob[eval_t] = hd["prob"]
 
     A, corr = scan(k_off, cand.astype(np.uint8), has_prob, prob, tau, lm["argmax"])
-    n_mismatch = np.add.reduceat(cand.astype(np.int32), k_off[:-1]) if T else np.zeros(B, np.int32)
-    n_mismatch = np.where(k_len > 0, n_mismatch, 0).astype(np.int32)
+    n_mismatch = np.bincount(req_of_t, weights=cand.astype(np.float64), minlength=B).astype(np.int32)   # |S| per request
     return dict(accept_len=A, correction_token=corr, argmax=lm["argmax"], lse=lm["lse"],
                 top2_gap=lm["top2_gap"], p_draft=p_draft, cand=cand, n_mismatch=n_mismatch,
                 head_prob=hd["prob"], head_logit=hd["logit"], eval_t=eval_t, has_prob=has_prob,

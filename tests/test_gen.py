@@ -64,3 +64,12 @@ def test_pack_selective_layout():
     assert np.array_equal(packed, hd[[0, 2, 6, 7]])
     packed, sel_off, sel_pos = gen.pack_selective(hd, k, np.zeros(9, bool))
     assert packed.shape == (0, 2) and sel_off.tolist() == [0, 0, 0, 0, 0]
+
+
+def test_pack_selective_with_empty_windows_at_the_end():
+    k = np.array([2, 0, 3, 0, 0], np.int32)
+    hd = np.arange(5 * 2, dtype=np.float32).reshape(5, 2)
+    sel = np.array([0, 1, 1, 0, 1], bool)
+    packed, sel_off, sel_pos = gen.pack_selective(hd, k, sel)
+    assert sel_off.tolist() == [0, 1, 1, 3, 3, 3] and sel_pos.tolist() == [1, 0, 2]
+    assert np.array_equal(packed, hd[[1, 2, 4]])

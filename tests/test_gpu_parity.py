@@ -245,6 +245,52 @@ def test_bounded_wait_gives_up_and_the_context_stays_usable():
     v.close()
 
 
+def test_empty_windows_and_empty_batch():
+    """K_b = 0 for some or all requests: nothing to accept, the correction is the bonus-row argmax."""
+    cfg = _small(B=6, K=0, K_lo=0, K_hi=2, seed=37)
+    case = cases.make_case(cfg, oracle_ref_argmax)
+    assert (case["k_len"] == 0).any()
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d)
+    out = cases.run(v, d)
+    torch.cuda.synchronize()
+    compare(case, run_oracle(case), out, cfg.tau)
+    # every window empty: T = 0, only the B bonus rows go through the LM head
+    k_off0 = torch.zeros(cfg.B + 1, dtype=torch.int32, device=DEV)
+    rows = d["target_hidden"][:cfg.B].contiguous()
+    o = v.verify(rows, d["draft_tokens"][:0], d["draft_hidden"][:0], d["csi"], B=cfg.B, k_off=k_off0, T=0)
+    torch.cuda.synchronize()
+    import oracle
+    ref = oracle.lm_head(case["lm_head"], case["target_hidden"][:cfg.B])
+    assert np.array_equal(o.accept_len.cpu().numpy(), np.zeros(cfg.B, np.int32))
+    gap_ok = ref["top2_gap"] >= 1e-2
+    assert np.array_equal(o.correction_token.cpu().numpy()[gap_ok], ref["argmax"][gap_ok])
+    # no requests at all: accepted, nothing launched
+    n = v.launch_count()
+    v.verify(rows, d["draft_tokens"][:0], d["draft_hidden"][:0], d["csi"], B=0, K=4, T=0)
+    assert v.launch_count() == n and v.device_error() == 0
+    v.close()
+
+
+def test_host_entry_point_with_selective_upload_and_sampling_test():
+    cfg = _small(B=7, K=0, K_lo=2, K_hi=6, mode="SH", stochastic=True, seed=39)
+    case = cases.make_case(cfg, oracle_ref_argmax)
+    base = run_oracle(case)
+    case["draft_q"] = (base["p_draft"] * np.random.default_rng(5).uniform(0.5, 4.0, size=case["T"])).astype(np.float32)
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d)
+    out = cases.run(v, d)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    ho = v.verify_host(pin(case["target_hidden"]), pin(case["draft_tokens"]), pin(case["draft_hidden"]),
+                       pin(case["csi"]), B=cfg.B, k_off=pin(case["k_off"]), T=case["T"], sel_off=pin(case["sel_off"]),
+                       sel_pos=pin(case["sel_pos"]), draft_q=pin(case["draft_q"]), uniforms=pin(case["uniforms"]),
+                       extras=True)
+    for k in ("accept_len", "correction_token", "argmax", "lse", "p_draft", "head_prob", "n_mismatch", "status"):
+        assert torch.equal(getattr(ho, k), getattr(out, k).cpu()), k
+    compare(case, run_oracle(case), out, cfg.tau)
+    v.close()
+
+
 def test_capacity_and_argument_errors():
     cfg = _small(B=4, K=4)
     case = cases.make_case(cfg, oracle_ref_argmax)

@@ -365,3 +365,18 @@ def test_whole_round_against_pure_python_brute_force():
         assert out["correction_token"][b] == amax[A]
         row += k[b] + 1
         t += k[b]
+
+
+def test_candidate_counts_with_empty_windows():
+    cfg = gen.VerifyConfig("e", B=5, K=0, K_lo=0, K_hi=2, H=24, H_d=16, d_c=2, d_J=8, V=97, match_rate=0.0, seed=2)
+    k = np.array([2, 0, 1, 0, 0], np.int32)
+    w = gen.make_weights(cfg)
+    h = gen.make_hidden(cfg, k)
+    ref = oracle.lm_head(w["lm_head"], h["target_hidden"])["argmax"]
+    toks = (ref[[0, 1, 4]] + 1) % cfg.V                         # every draft token mismatches
+    out = oracle.verify(lm_head_bits=w["lm_head"], W1_bits=w["W1"], b1=w["b1"], w2=w["w2"], b2=w["b2"],
+                        act=oracle.ACT_RELU, tau=0.0, k_len=k, target_hidden=h["target_hidden"],
+                        draft_tokens=toks.astype(np.int32), draft_hidden=h["draft_hidden"], csi=h["csi"])
+    assert out["n_mismatch"].tolist() == [2, 0, 1, 0, 0]
+    assert out["accept_len"].tolist() == [0, 0, 0, 0, 0]
+    assert np.array_equal(out["correction_token"], ref[[0, 3, 4, 6, 7]])     # first row of every window
