@@ -226,6 +226,18 @@ def test_host_buffer_entry_point_matches_device_entry_point():
                        pin(case["csi"]), B=cfg.B, K=cfg.K, extras=True)
     for k in ("accept_len", "correction_token", "argmax", "lse", "p_draft", "head_prob", "n_mismatch", "status"):
         assert torch.equal(getattr(ho, k), getattr(out, k).cpu()), k
+    # pageable host memory works too (the copies are then synchronous staging copies)
+    from paper_2604_17701_b200 import VerifyOutput
+    page = lambda a: torch.from_numpy(np.ascontiguousarray(a).copy())
+    po = VerifyOutput(torch.empty(cfg.B, dtype=torch.int32), torch.empty(cfg.B, dtype=torch.int32))
+    po.argmax, po.lse = torch.empty(case["R"], dtype=torch.int32), torch.empty(case["R"], dtype=torch.float32)
+    po.p_draft, po.head_prob = torch.empty(case["T"]), torch.empty(case["T"])
+    po.mismatch_mask = torch.empty(cfg.B, dtype=torch.int64)
+    po.n_mismatch, po.status = torch.empty(cfg.B, dtype=torch.int32), torch.empty(cfg.B, dtype=torch.int32)
+    v.verify_host(page(case["target_hidden"]), page(case["draft_tokens"]), page(case["draft_hidden"]),
+                  page(case["csi"]), B=cfg.B, K=cfg.K, extras=True, out=po)
+    for k in ("accept_len", "correction_token", "argmax", "lse", "p_draft", "head_prob", "n_mismatch", "status"):
+        assert torch.equal(getattr(po, k), getattr(out, k).cpu()), k
     v.close()
 
 
