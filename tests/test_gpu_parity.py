@@ -182,6 +182,39 @@ def test_selective_hidden_missing_upload_is_rejected_and_flagged():
     v.close()
 
 
+def test_selective_hidden_out_of_range_position_is_ignored_and_flagged():
+    cfg = _small(mode="SH", B=6, K=5, seed=8, match_rate=0.3)
+    case = cases.make_case(cfg, oracle_ref_argmax)
+    b = next(i for i in range(cfg.B) if case["sel_off"][i + 1] - case["sel_off"][i] >= 2)
+    j = int(case["sel_off"][b])                       # first uploaded entry of request b
+    bad = dict(case)
+    bad["sel_pos"] = case["sel_pos"].copy()
+    bad["sel_pos"][j] = cfg.K + 3                     # not a window position
+    d = cases.to_device(bad, DEV)
+    v = cases.make_verifier(d)
+    out = cases.run(v, d)
+    torch.cuda.synchronize()
+    st = out.status.cpu().numpy()
+    assert st[b] & 8 and all(not (st[i] & 8) for i in range(cfg.B) if i != b)
+    # same decisions as if that upload had never arrived
+    keep = np.ones(case["sel_pos"].shape[0], bool)
+    keep[j] = False
+    less = dict(case)
+    cnt = np.diff(case["sel_off"]).copy()
+    cnt[b] -= 1
+    less["sel_off"] = np.concatenate([[0], np.cumsum(cnt)]).astype(np.int32)
+    less["sel_pos"] = case["sel_pos"][keep]
+    less["draft_hidden"] = case["draft_hidden"][keep]
+    ref = run_oracle(less)
+    A, Ao = out.accept_len.cpu().numpy(), ref["accept_len"]
+    tie = np.zeros(cfg.B, bool)
+    for i in range(cfg.B):
+        rows = slice(ref["row_off"][i], ref["row_off"][i + 1])
+        tie[i] = (ref["top2_gap"][rows] < 1e-2).any() or (np.abs(ref["prob_t"][ref["k_off"][i]:ref["k_off"][i + 1]] - cfg.tau) < 2e-3).any()
+    assert np.array_equal(A[~tie], Ao[~tie])
+    v.close()
+
+
 def test_stochastic_acceptance():
     cfg = _small(B=32, K=6, seed=9, stochastic=True)
     case = cases.make_case(cfg, oracle_ref_argmax)
