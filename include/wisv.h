@@ -206,10 +206,15 @@ int wisv_verify_gathered(wisv_ctx* ctx, const wisv_batch* batch, const wisv_row_
 
 /*
  * Same round with HOST buffers: every pointer in `batch` and `result` is host
- * memory (pinned memory makes the copies asynchronous).  Inputs are copied to
- * staging buffers owned by the context (allocated on first use), the round is
- * run, the requested results are copied back and the stream is synchronised
- * before returning.  Returns WISV_EDEVICE if a kernel reported a time-out.
+ * memory, pinned or pageable, with no alignment requirement.  A hidden-state
+ * array of at most 1 MiB in pinned, 16-byte aligned memory is read in place by
+ * the first kernel; otherwise it is copied to a staging buffer owned by the
+ * context (allocated on first use).  All other inputs are packed into one
+ * pinned block and travel in one copy.  The last kernel writes the requested
+ * results into a device-mapped pinned block, from which they are written to
+ * the caller's arrays once the stream has been synchronised, before returning.
+ * One call at a time per context: the staging memory is reused by the next
+ * call.  Returns WISV_EDEVICE if a kernel reported a time-out.
  */
 int wisv_verify_host(wisv_ctx* ctx, const wisv_batch* batch, const wisv_result* result, void* cuda_stream);
 

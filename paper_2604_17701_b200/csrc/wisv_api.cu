@@ -42,13 +42,16 @@ struct Plan {
     size_t smem;
 };
 
+// Device and pinned-host staging of the host-buffer entry point. The two hidden-state arrays are copied straight from
+// the caller's memory; every small input travels in one packed block (one copy), and every output plus the device
+// error word comes back in one packed block (one copy), because at small batches a round is a few hundred
+// microseconds and each separate copy costs several of them in submission and DMA latency.
 struct HostStaging {
-    float* target_hidden = nullptr; int32_t* draft_tokens = nullptr; float* draft_hidden = nullptr;
-    int32_t* k_off = nullptr; int32_t* sel_off = nullptr; int32_t* sel_pos = nullptr; float* csi = nullptr;
-    float* draft_q = nullptr; float* uniforms = nullptr;
-    int32_t* accept_len = nullptr; int32_t* correction = nullptr; int32_t* argmax = nullptr; float* lse = nullptr;
-    float* p_draft = nullptr; float* head_prob = nullptr; unsigned long long* mask = nullptr;
-    int32_t* n_mismatch = nullptr; int32_t* status = nullptr;
+    float* target_hidden = nullptr; float* draft_hidden = nullptr;
+    uint8_t* dev_in = nullptr;        // packed small inputs, layout chosen per call
+    uint8_t* pin = nullptr;           // pinned, device-mapped host: [in_cap | out_cap]
+    uint8_t* pin_dev = nullptr;       // the same block as the device sees it
+    size_t in_cap = 0, out_cap = 0;
     bool ready = false;
 };
 
@@ -79,6 +82,7 @@ struct wisv_ctx {
     int32_t* row_tok = nullptr; int32_t* row_flag = nullptr; float* tok_logit = nullptr;
     int32_t* pos_req = nullptr; int32_t* pos_i = nullptr;
     int32_t* err = nullptr;
+    int32_t* err_copy_next = nullptr;           // where the next round's tail kernel mirrors the error word
     int32_t* saved_arg = nullptr;               // [rows_alloc] argmax per row, localize -> decide
     unsigned long long* saved_mask = nullptr;   // [max_requests] candidate sets, localize -> decide
     bool loc_valid = false;                     // a localize call is waiting for its decide
@@ -257,10 +261,8 @@ void free_ctx(wisv_ctx* c)
         free(c->prof_ev);
     }
     HostStaging& h = c->hs;
-    cudaFree(h.target_hidden); cudaFree(h.draft_tokens); cudaFree(h.draft_hidden); cudaFree(h.k_off);
-    cudaFree(h.sel_off); cudaFree(h.sel_pos); cudaFree(h.csi); cudaFree(h.draft_q); cudaFree(h.uniforms);
-    cudaFree(h.accept_len); cudaFree(h.correction); cudaFree(h.argmax); cudaFree(h.lse); cudaFree(h.p_draft);
-    cudaFree(h.head_prob); cudaFree(h.mask); cudaFree(h.n_mismatch); cudaFree(h.status);
+    cudaFree(h.target_hidden); cudaFree(h.draft_hidden); cudaFree(h.dev_in);
+    if (h.pin) cudaFreeHost(h.pin);
     (void)cudaGetLastError();
     delete c;
 }
@@ -272,6 +274,45 @@ int dev_alloc(T** p, size_t n)
     if (cudaMalloc(&q, (n ? n : 1) * sizeof(T)) != cudaSuccess) { (void)cudaGetLastError(); return WISV_ENOMEM; }
     *p = static_cast<T*>(q);
     return WISV_OK;
+}
+
+// Device address of a pinned host array if the kernels can read it in place (registered with CUDA, 16-byte aligned,
+// at most kZeroCopyBytes), else `staged`.
+constexpr size_t kZeroCopyBytes = 1u << 20;
+const float* mapped_or(const float* host, size_t bytes, const float* staged)
+{
+    if (!host || bytes == 0 || bytes > kZeroCopyBytes) return staged;
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, host) != cudaSuccess) { (void)cudaGetLastError(); return staged; }
+    if (at.type != cudaMemoryTypeHost || !at.devicePointer) return staged;
+    if (reinterpret_cast<uintptr_t>(at.devicePointer) & 15u) return staged;
+    return static_cast<const float*>(at.devicePointer);
+}
+
+inline size_t pad16(size_t n) { return (n + 15) & ~size_t(15); }
+
+// Offsets (past the 16 bytes that hold the mirrored error word) of the packed outputs for B requests, R rows, T drafted tokens and
+// P evaluated positions; returns the bytes used. Order: accept_len, correction, argmax, lse, p_draft, head_prob,
+// mismatch_mask, n_mismatch, status.
+enum { OUT_ACCEPT = 0, OUT_CORR, OUT_ARGMAX, OUT_LSE, OUT_PDRAFT, OUT_HEADP, OUT_MASK, OUT_NMIS, OUT_STATUS, OUT_FIELDS };
+size_t out_arena_layout(int B, int R, int T, int P, size_t* off)
+{
+    const size_t sz[OUT_FIELDS] = {4u * (size_t)B, 4u * (size_t)B, 4u * (size_t)R, 4u * (size_t)R, 4u * (size_t)T,
+                                   4u * (size_t)P, 8u * (size_t)B, 4u * (size_t)B, 4u * (size_t)B};
+    size_t at = 0;
+    for (int i = 0; i < OUT_FIELDS; ++i) { if (off) off[i] = at; at += pad16(sz[i]); }
+    return at;
+}
+
+// The same for the small inputs: k_off, draft_tokens, sel_off, sel_pos, csi, draft_q, uniforms.
+enum { IN_KOFF = 0, IN_TOK, IN_SELOFF, IN_SELPOS, IN_CSI, IN_Q, IN_U, IN_FIELDS };
+size_t in_arena_layout(int B, int T, int P, int d_c, size_t* off, size_t* bytes)
+{
+    const size_t sz[IN_FIELDS] = {4u * ((size_t)B + 1), 4u * (size_t)T, 4u * ((size_t)B + 1), 4u * (size_t)P,
+                                  4u * (size_t)B * (size_t)d_c, 4u * (size_t)T, 4u * (size_t)T};
+    size_t at = 0;
+    for (int i = 0; i < IN_FIELDS; ++i) { if (off) off[i] = at; if (bytes) bytes[i] = sz[i]; at += pad16(sz[i]); }
+    return at;
 }
 
 enum { PHASE_FULL = 0, PHASE_LOCALIZE = 1, PHASE_DECIDE = 2, PHASE_GATHERED = 3, PHASE_SHARD = 4 };
@@ -683,6 +724,8 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
     tp.p_draft = r->p_draft; tp.head_prob = r->head_prob;
     tp.mismatch_mask = reinterpret_cast<unsigned long long*>(r->mismatch_mask); tp.n_mismatch = r->n_mismatch;
     tp.status = r->status;
+    tp.err_src = c->err; tp.err_copy = c->err_copy_next;
+    c->err_copy_next = nullptr;
     {
         const int rc = launch_pdl(tail_kernel, dim3(b->B), dim3(256), 0, st, tp);
         if (rc != WISV_OK) return rc;
@@ -818,95 +861,103 @@ int wisv_verify_host(wisv_ctx* c, const wisv_batch* hb, const wisv_result* hr, v
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     HostStaging& h = c->hs;
     const wisv_config& cf = c->cfg;
-    const int maxB = cf.max_requests, maxR = cf.max_rows, maxT = cf.max_rows - 1 > 0 ? cf.max_rows - 1 : 1;
+    const int maxB = cf.max_requests, maxR = cf.max_rows;
     if (!h.ready) {
         int rc = WISV_OK;
         do {
             if ((rc = dev_alloc(&h.target_hidden, (size_t)maxR * cf.H))) break;
-            if ((rc = dev_alloc(&h.draft_tokens, (size_t)maxT))) break;
             if ((rc = dev_alloc(&h.draft_hidden, (size_t)c->max_pos * cf.H_d))) break;
-            if ((rc = dev_alloc(&h.k_off, (size_t)maxB + 1))) break;
-            if ((rc = dev_alloc(&h.sel_off, (size_t)maxB + 1))) break;
-            if ((rc = dev_alloc(&h.sel_pos, (size_t)c->max_pos))) break;
-            if ((rc = dev_alloc(&h.csi, (size_t)maxB * (cf.d_c > 0 ? cf.d_c : 1)))) break;
-            if ((rc = dev_alloc(&h.draft_q, (size_t)maxT))) break;
-            if ((rc = dev_alloc(&h.uniforms, (size_t)maxT))) break;
-            if ((rc = dev_alloc(&h.accept_len, (size_t)maxB))) break;
-            if ((rc = dev_alloc(&h.correction, (size_t)maxB))) break;
-            if ((rc = dev_alloc(&h.argmax, (size_t)maxR))) break;
-            if ((rc = dev_alloc(&h.lse, (size_t)maxR))) break;
-            if ((rc = dev_alloc(&h.p_draft, (size_t)maxT))) break;
-            if ((rc = dev_alloc(&h.head_prob, (size_t)c->max_pos))) break;
-            if ((rc = dev_alloc(&h.mask, (size_t)maxB))) break;
-            if ((rc = dev_alloc(&h.n_mismatch, (size_t)maxB))) break;
-            if ((rc = dev_alloc(&h.status, (size_t)maxB))) break;
+            h.in_cap = in_arena_layout(maxB, maxR, c->max_pos, cf.d_c, nullptr, nullptr);
+            h.out_cap = 16 + out_arena_layout(maxB, maxR, maxR, c->max_pos, nullptr);
+            if ((rc = dev_alloc(&h.dev_in, h.in_cap))) break;
+            if (cudaHostAlloc(reinterpret_cast<void**>(&h.pin), h.in_cap + h.out_cap, cudaHostAllocMapped) != cudaSuccess ||
+                cudaHostGetDevicePointer(reinterpret_cast<void**>(&h.pin_dev), h.pin, 0) != cudaSuccess) {
+                (void)cudaGetLastError();
+                if (h.pin) cudaFreeHost(h.pin);
+                h.pin = nullptr;
+                rc = WISV_ENOMEM;
+                break;
+            }
         } while (0);
         if (rc != WISV_OK) return rc;
         h.ready = true;
     }
+    // sizes of this call as the batch states them; out-of-range ones are left for validate_batch to name
+    const int B = hb->B;
+    const bool sh = (hb->mode & WISV_MODE_SH) != 0;
+    const bool stoch = (hb->mode & WISV_ACCEPT_STOCHASTIC) != 0;
+    const long long T_ll = hb->k_off ? (long long)hb->T_total : (long long)hb->B * hb->K;
+    const long long P_ll = sh ? (long long)hb->M_sel : T_ll;
+    const bool fits = B >= 0 && B <= maxB && T_ll >= 0 && T_ll + B <= maxR && P_ll >= 0 && P_ll <= c->max_pos;
+    const int T = fits ? (int)T_ll : 0, P = fits ? (int)P_ll : 0, R = fits ? T + B : 0;
+    size_t ioff[IN_FIELDS], ibytes[IN_FIELDS], ooff[OUT_FIELDS];
+    const size_t in_used = in_arena_layout(fits ? B : 0, T, P, cf.d_c, ioff, ibytes);
+    const size_t out_used = 16 + out_arena_layout(fits ? B : 0, R, T, P, ooff);
+    if (in_used > h.in_cap || out_used > h.out_cap) return WISV_ECAPACITY;
+    uint8_t* pin_in = h.pin;
+    uint8_t* pin_out = h.pin + h.in_cap;
+    uint8_t* dev_out = h.pin_dev + h.in_cap + 16;   // the tail kernel writes the results straight to host memory
     // the device-side view of the batch, validated before any copy
     wisv_batch db = *hb;
     wisv_result dr;
     memset(&dr, 0, sizeof dr);
-    db.k_off = hb->k_off ? h.k_off : nullptr;
-    db.target_hidden = hb->target_hidden ? h.target_hidden : nullptr;
-    db.draft_tokens = hb->draft_tokens ? h.draft_tokens : nullptr;
-    db.draft_hidden = hb->draft_hidden ? h.draft_hidden : nullptr;
-    db.sel_off = hb->sel_off ? h.sel_off : nullptr;
-    db.sel_pos = hb->sel_pos ? h.sel_pos : nullptr;
-    db.csi = hb->csi ? h.csi : nullptr;
-    db.draft_q = hb->draft_q ? h.draft_q : nullptr;
-    db.uniforms = hb->uniforms ? h.uniforms : nullptr;
-    dr.accept_len = hr->accept_len ? h.accept_len : nullptr;
-    dr.correction_token = hr->correction_token ? h.correction : nullptr;
-    dr.argmax = hr->argmax ? h.argmax : nullptr;
-    dr.lse = hr->lse ? h.lse : nullptr;
-    dr.p_draft = hr->p_draft ? h.p_draft : nullptr;
-    dr.head_prob = hr->head_prob ? h.head_prob : nullptr;
-    dr.mismatch_mask = hr->mismatch_mask ? reinterpret_cast<uint64_t*>(h.mask) : nullptr;
-    dr.n_mismatch = hr->n_mismatch ? h.n_mismatch : nullptr;
-    dr.status = hr->status ? h.status : nullptr;
-    int T = 0, R = 0, P = 0;
-    const int vrc = validate_batch(c, &db, &dr, &T, &R, &P);
+    const void* src[IN_FIELDS] = {hb->k_off, hb->draft_tokens, sh ? hb->sel_off : nullptr, sh ? hb->sel_pos : nullptr,
+                                  hb->csi, stoch ? hb->draft_q : nullptr, stoch ? hb->uniforms : nullptr};
+    db.k_off = hb->k_off ? reinterpret_cast<int32_t*>(h.dev_in + ioff[IN_KOFF]) : nullptr;
+    // a small hidden-state array in pinned memory is read in place by the pack kernel (one pass over PCIe, no
+    // separate copy to wait for); a large or pageable one goes through the copy engine
+    const size_t th_bytes = sizeof(float) * (size_t)R * cf.H, dh_bytes = sizeof(float) * (size_t)P * cf.H_d;
+    const float* th_dev = mapped_or(hb->target_hidden, th_bytes, h.target_hidden);
+    const float* dh_dev = mapped_or(hb->draft_hidden, dh_bytes, h.draft_hidden);
+    db.target_hidden = hb->target_hidden ? th_dev : nullptr;
+    db.draft_tokens = hb->draft_tokens ? reinterpret_cast<int32_t*>(h.dev_in + ioff[IN_TOK]) : nullptr;
+    db.draft_hidden = hb->draft_hidden ? dh_dev : nullptr;
+    db.sel_off = hb->sel_off ? reinterpret_cast<int32_t*>(h.dev_in + ioff[IN_SELOFF]) : nullptr;
+    db.sel_pos = hb->sel_pos ? reinterpret_cast<int32_t*>(h.dev_in + ioff[IN_SELPOS]) : nullptr;
+    db.csi = hb->csi ? reinterpret_cast<float*>(h.dev_in + ioff[IN_CSI]) : nullptr;
+    db.draft_q = hb->draft_q ? reinterpret_cast<float*>(h.dev_in + ioff[IN_Q]) : nullptr;
+    db.uniforms = hb->uniforms ? reinterpret_cast<float*>(h.dev_in + ioff[IN_U]) : nullptr;
+    dr.accept_len = hr->accept_len ? reinterpret_cast<int32_t*>(dev_out + ooff[OUT_ACCEPT]) : nullptr;
+    dr.correction_token = hr->correction_token ? reinterpret_cast<int32_t*>(dev_out + ooff[OUT_CORR]) : nullptr;
+    dr.argmax = hr->argmax ? reinterpret_cast<int32_t*>(dev_out + ooff[OUT_ARGMAX]) : nullptr;
+    dr.lse = hr->lse ? reinterpret_cast<float*>(dev_out + ooff[OUT_LSE]) : nullptr;
+    dr.p_draft = hr->p_draft ? reinterpret_cast<float*>(dev_out + ooff[OUT_PDRAFT]) : nullptr;
+    dr.head_prob = hr->head_prob ? reinterpret_cast<float*>(dev_out + ooff[OUT_HEADP]) : nullptr;
+    dr.mismatch_mask = hr->mismatch_mask ? reinterpret_cast<uint64_t*>(dev_out + ooff[OUT_MASK]) : nullptr;
+    dr.n_mismatch = hr->n_mismatch ? reinterpret_cast<int32_t*>(dev_out + ooff[OUT_NMIS]) : nullptr;
+    dr.status = hr->status ? reinterpret_cast<int32_t*>(dev_out + ooff[OUT_STATUS]) : nullptr;
+    int Tv = 0, Rv = 0, Pv = 0;
+    const int vrc = validate_batch(c, &db, &dr, &Tv, &Rv, &Pv);
     if (vrc != WISV_OK) return vrc;
-    if (hb->B == 0) return WISV_OK;
-    const int B = hb->B;
-    const bool sh = (hb->mode & WISV_MODE_SH) != 0;
-    const bool stoch = (hb->mode & WISV_ACCEPT_STOCHASTIC) != 0;
-#define H2D(dst, src, n) \
-    do { if ((src) && (n) > 0) WISV_CUDA(cudaMemcpyAsync((dst), (src), (size_t)(n), cudaMemcpyHostToDevice, st)); } while (0)
-#define D2H(dst, src, n) \
-    do { if ((dst) && (n) > 0) WISV_CUDA(cudaMemcpyAsync((dst), (src), (size_t)(n), cudaMemcpyDeviceToHost, st)); } while (0)
-    H2D(h.k_off, hb->k_off, sizeof(int32_t) * (B + 1));
-    H2D(h.target_hidden, hb->target_hidden, sizeof(float) * (size_t)R * cf.H);
-    H2D(h.draft_tokens, hb->draft_tokens, sizeof(int32_t) * (size_t)T);
-    H2D(h.draft_hidden, hb->draft_hidden, sizeof(float) * (size_t)P * cf.H_d);
-    if (sh) {
-        H2D(h.sel_off, hb->sel_off, sizeof(int32_t) * (B + 1));
-        H2D(h.sel_pos, hb->sel_pos, sizeof(int32_t) * (size_t)P);
-    }
-    H2D(h.csi, hb->csi, sizeof(float) * (size_t)B * cf.d_c);
-    if (stoch) {
-        H2D(h.draft_q, hb->draft_q, sizeof(float) * (size_t)T);
-        H2D(h.uniforms, hb->uniforms, sizeof(float) * (size_t)T);
-    }
+    if (!fits) return WISV_ESHAPE;
+    if (B == 0) return WISV_OK;
+    for (int i = 0; i < IN_FIELDS; ++i)
+        if (src[i] && ibytes[i] > 0) memcpy(pin_in + ioff[i], src[i], ibytes[i]);
+    WISV_CUDA(cudaMemcpyAsync(h.dev_in, pin_in, in_used, cudaMemcpyHostToDevice, st));
+    if (th_dev != h.target_hidden)
+        ;   // the pack kernel reads the caller's pinned array in place
+    else if (hb->target_hidden)
+        WISV_CUDA(cudaMemcpyAsync(h.target_hidden, hb->target_hidden, th_bytes, cudaMemcpyHostToDevice, st));
+    if (dh_dev != h.draft_hidden)
+        ;
+    else if (hb->draft_hidden && P > 0)
+        WISV_CUDA(cudaMemcpyAsync(h.draft_hidden, hb->draft_hidden, dh_bytes, cudaMemcpyHostToDevice, st));
+    memset(pin_out, 0, 4);
+    c->err_copy_next = reinterpret_cast<int32_t*>(h.pin_dev + h.in_cap);
     const int rc = wisv_verify(c, &db, &dr, cuda_stream);
+    c->err_copy_next = nullptr;
     if (rc != WISV_OK) return rc;
-    D2H(hr->accept_len, h.accept_len, sizeof(int32_t) * B);
-    D2H(hr->correction_token, h.correction, sizeof(int32_t) * B);
-    D2H(hr->argmax, h.argmax, sizeof(int32_t) * (size_t)R);
-    D2H(hr->lse, h.lse, sizeof(float) * (size_t)R);
-    D2H(hr->p_draft, h.p_draft, sizeof(float) * (size_t)T);
-    D2H(hr->head_prob, h.head_prob, sizeof(float) * (size_t)P);
-    D2H(hr->mismatch_mask, h.mask, sizeof(uint64_t) * B);
-    D2H(hr->n_mismatch, h.n_mismatch, sizeof(int32_t) * B);
-    D2H(hr->status, h.status, sizeof(int32_t) * B);
-#undef H2D
-#undef D2H
-    int32_t dev_err = 0;
-    WISV_CUDA(cudaMemcpyAsync(&dev_err, c->err, sizeof dev_err, cudaMemcpyDeviceToHost, st));
     WISV_CUDA(cudaStreamSynchronize(st));
+    int32_t dev_err = 0;
+    memcpy(&dev_err, pin_out, sizeof dev_err);
     if (dev_err != 0) { (void)cudaMemset(c->err, 0, sizeof dev_err); return WISV_EDEVICE; }
+    const uint8_t* po = pin_out + 16;
+    void* dst[OUT_FIELDS] = {hr->accept_len, hr->correction_token, hr->argmax, hr->lse, hr->p_draft,
+                             hr->head_prob, hr->mismatch_mask, hr->n_mismatch, hr->status};
+    const size_t obytes[OUT_FIELDS] = {4u * (size_t)B, 4u * (size_t)B, 4u * (size_t)R, 4u * (size_t)R, 4u * (size_t)T,
+                                       4u * (size_t)P, 8u * (size_t)B, 4u * (size_t)B, 4u * (size_t)B};
+    for (int i = 0; i < OUT_FIELDS; ++i)
+        if (dst[i] && obytes[i] > 0) memcpy(dst[i], po + ooff[i], obytes[i]);
     return WISV_OK;
 }
 

@@ -150,6 +150,8 @@ struct TailParams {
     const float* uniforms;        // [T] (stochastic)
     int32_t* accept_len; int32_t* correction; int32_t* argmax; float* lse; float* p_draft; float* head_prob;
     unsigned long long* mismatch_mask; int32_t* n_mismatch; int32_t* status;
+    const int32_t* err_src;       // device error word of the earlier kernels of this round
+    int32_t* err_copy;            // if set, receives *err_src (lets a host caller read it with the results)
 };
 
 struct RowStat { float mx; int idx; float sum; };
@@ -187,6 +189,8 @@ __global__ void __launch_bounds__(256) tail_kernel(const TailParams p)
     // partials of the LM-head and decision-head kernels must be complete and visible
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    if (p.err_copy && b == 0 && threadIdx.x == 0) *p.err_copy = *p.err_src;
 
     // ---- merge the per-tile (max, argidx, sumexp) partials of each window row
     int flag = 0;

@@ -274,6 +274,30 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     v.close()
 
 
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_buffer_entry_point_ragged_selective_stochastic(pinned):
+    """Every optional input (row offsets, selective positions, q and u of Eq. 1) through the packed host block; the
+    target hidden states exceed the in-place limit (copy-engine path) while the draft ones stay below it."""
+    cfg = _small(B=40, K=0, K_lo=1, K_hi=8, H=2048, H_d=128, mode="SH", stochastic=True, seed=71)
+    case = cases.make_case(cfg, oracle_ref_argmax)
+    assert case["R"] * cfg.H * 4 > (1 << 20) > case["sel_pos"].shape[0] * cfg.H_d * 4
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d)
+    out = cases.run(v, d)
+    mk = (lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()) if pinned else \
+        (lambda a: torch.from_numpy(np.ascontiguousarray(a).copy()))
+    for _ in range(2):                           # the staging blocks are reused by the second call
+        ho = v.verify_host(mk(case["target_hidden"]), mk(case["draft_tokens"]), mk(case["draft_hidden"]),
+                           mk(case["csi"]), B=cfg.B, k_off=mk(case["k_off"]), T=case["T"], sel_off=mk(case["sel_off"]),
+                           sel_pos=mk(case["sel_pos"]), draft_q=mk(case["draft_q"]), uniforms=mk(case["uniforms"]),
+                           extras=True)
+        for k in ("accept_len", "correction_token", "argmax", "lse", "p_draft", "head_prob", "mismatch_mask",
+                  "n_mismatch", "status"):
+            assert torch.equal(getattr(ho, k), getattr(out, k).cpu()), k
+    assert v.device_error() == 0
+    v.close()
+
+
 def test_bounded_wait_gives_up_and_the_context_stays_usable():
     cfg = _small(B=4, K=4, seed=29)
     case = cases.make_case(cfg, oracle_ref_argmax)
