@@ -156,7 +156,7 @@ double wave_eff(long long tiles, int sms)
 // LM head: with a single row tile the kernel streams the weights once and is
 // HBM-bound, so the tile height over the vocabulary is chosen to fill the last
 // wave of CTAs; with many row tiles it is tensor-bound and takes the largest tile.
-Plan plan_lm(const wisv_ctx* c, int R)
+Plan plan_lm(const wisv_ctx* c, int R, bool single_only = false)
 {
     Plan p{};
     const int V = c->cfg.V;
@@ -166,7 +166,7 @@ Plan plan_lm(const wisv_ctx* c, int R)
     // The pair kernel keeps the tensor pipe about 10 % busier than the single-CTA kernel (95 % against
     // 86 %), so the padding pays off from 11 row tiles on.
     const bool pair_fits = p.m_tiles % 2 == 0 || p.m_tiles >= 11;
-    if (p.m_tiles >= 2 && pair_fits && c->max_pairs > 0 && !c->tune.lm_single_cta && !c->tune.lm_tile_n) {
+    if (p.m_tiles >= 2 && pair_fits && c->max_pairs > 0 && !single_only && !c->tune.lm_single_cta && !c->tune.lm_tile_n) {
         p.pair = 1;
         p.m_tiles = (R + kPairTileM - 1) / kPairTileM;
         p.tile_n = kPairTileN;
@@ -787,7 +787,7 @@ int wisv_debug_logits(wisv_ctx* c, const float* target_hidden, int32_t R, float*
     pack_kernel<<<R, 256, 0, st>>>(pp);
     WISV_CUDA(cudaGetLastError());
     c->launches++;
-    const Plan pl = plan_lm(c, R);
+    const Plan pl = plan_lm(c, R, true);            // the raw-logits epilogue exists for the single-CTA kernel only
     GemmParams gp = base_params(c, pl, R, c->cfg.V, c->cfg.H);
     gp.raw_out = logits_out;
     return launch_gemm<EPI_RAW>(c, c->tmX[pl.a_rows / 8 - 1], c->tmW[pl.tile_n / 16 - 1], gp, pl, st);

@@ -45,8 +45,9 @@ def _run(cfg, *, act=None, tau=None, shift=0, ref_fn=oracle_ref_argmax):
     return case, ref, out, stats
 
 
-def test_raw_logits_match_oracle():
-    cfg = _small(B=8, K=4)
+@pytest.mark.parametrize("B", [8, 52], ids=["R40", "R260"])     # one row tile; three row tiles, the last ragged
+def test_raw_logits_match_oracle(B):
+    cfg = _small(B=B, K=4)
     case = cases.make_case(cfg, oracle_ref_argmax)
     d = cases.to_device(case, DEV)
     v = cases.make_verifier(d)
