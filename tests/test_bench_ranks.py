@@ -34,8 +34,9 @@ def test_max_over_ranks_and_sharded_seeds_with_two_gloo_ranks(tmp_path):
         r.barrier()
         slowest = r.max(1.0 + rank)                       # every rank must learn the slowest rank's time
         cfg = bench.workload_config("8b_b1", rank)        # each rank verifies its own batch of the same model
-        print(json.dumps({"rank": rank, "max": slowest, "seed": cfg.seed, "weight_seed": cfg.weight_seed,
-                          "value": bench.aggregate(world, 8, slowest)}), flush=True)
+        rec = {"rank": rank, "max": slowest, "seed": cfg.seed, "weight_seed": cfg.weight_seed,
+               "value": bench.aggregate(world, 8, slowest)}
+        os.write(1, (json.dumps(rec) + chr(10)).encode())   # one write per line: the ranks share the pipe
         r.close()
     """ % ROOT))
     out = _torchrun(2, [str(script)])
@@ -83,7 +84,8 @@ def test_row_partials_are_gathered_rank_major_with_two_gloo_ranks(tmp_path):
         r.all_gather(gathered, part)                           # the layout wisv_verify_gathered expects: [G][R]
         ok = all(bool((gathered[g] == torch.full((R, 4), float(g)) + torch.arange(R).float()[:, None] * 10).all())
                  for g in range(world))
-        print(json.dumps({"rank": rank, "ok": ok, "shape": list(gathered.shape)}), flush=True)
+        rec = {"rank": rank, "ok": ok, "shape": list(gathered.shape)}
+        os.write(1, (json.dumps(rec) + chr(10)).encode())   # one write per line: the ranks share the pipe
         r.close()
     """ % ROOT))
     out = _torchrun(2, [str(script)])
