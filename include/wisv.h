@@ -247,6 +247,8 @@ int wisv_profile_read(wisv_ctx* ctx, int32_t stage, float* ms, int32_t cap, int3
 typedef struct {
     int32_t lm_tile_n, lm_stages, head_tile_n, head_stages;
     int32_t lm_single_cta;   /* 1: never use the CTA-pair LM-head kernel (batches with more than 128 window rows) */
+    int32_t head_ctas;       /* batches of at most 128 window rows and 128 head positions run both GEMMs in one
+                                launch: CTAs given to the decision head there (0 = default), -1 = two launches */
 } wisv_tuning;
 int wisv_set_tuning(wisv_ctx* ctx, const wisv_tuning* tuning);
 
@@ -260,6 +262,14 @@ int64_t wisv_launch_count(const wisv_ctx* ctx);
  */
 int wisv_plan(const wisv_ctx* ctx, int32_t R, int32_t P, int32_t* lm_tile_n, int32_t* lm_tiles,
               int32_t* lm_ctas, int32_t* head_tile_n, int32_t* head_tiles, int32_t* head_ctas);
+
+/*
+ * Kernels one wisv_verify round launches for such a batch: 4 (pack, LM head,
+ * decision head, merge + scan), or 3 when the batch has at most 128 window rows
+ * and 128 head positions and the two GEMMs share one launch, or when P = 0.
+ * Negative on bad arguments.
+ */
+int wisv_plan_kernels(const wisv_ctx* ctx, int32_t R, int32_t P);
 
 /*
  * Link model of Section IV-A (host arithmetic only).  For one round with K_r draft

@@ -51,7 +51,7 @@ class _Result(C.Structure):
 
 class _Tuning(C.Structure):
     _fields_ = [("lm_tile_n", C.c_int32), ("lm_stages", C.c_int32), ("head_tile_n", C.c_int32),
-                ("head_stages", C.c_int32), ("lm_single_cta", C.c_int32)]
+                ("head_stages", C.c_int32), ("lm_single_cta", C.c_int32), ("head_ctas", C.c_int32)]
 
 
 class LinkParams(C.Structure):
@@ -130,6 +130,8 @@ def load_library(build_if_missing: bool = False):
     lib.wisv_link_cost_round.argtypes = [C.POINTER(LinkParams), C.c_int32, C.c_int32, C.c_int32, C.POINTER(LinkCost)]
     lib.wisv_choose_protocol.restype = C.c_int
     lib.wisv_choose_protocol.argtypes = [C.c_double]
+    lib.wisv_plan_kernels.restype = C.c_int
+    lib.wisv_plan_kernels.argtypes = [P, C.c_int32, C.c_int32]
     lib.wisv_set_tuning.restype = C.c_int
     lib.wisv_set_tuning.argtypes = [P, C.POINTER(_Tuning)]
     lib.wisv_lm_head_reduce_static.restype = C.c_int
@@ -386,9 +388,14 @@ class Verifier:
         keys = ("lm_tile_n", "lm_tiles", "lm_ctas", "head_tile_n", "head_tiles", "head_ctas")
         return dict(zip(keys, (x.value for x in v)))
 
+    def plan_kernels(self, R: int, P: int) -> int:
+        n = self.lib.wisv_plan_kernels(self._h, R, P)
+        _check(min(n, 0), "wisv_plan_kernels")
+        return n
+
     def set_tuning(self, lm_tile_n: int = 0, lm_stages: int = 0, head_tile_n: int = 0, head_stages: int = 0,
-                   lm_single_cta: int = 0):
-        t = _Tuning(lm_tile_n, lm_stages, head_tile_n, head_stages, lm_single_cta)
+                   lm_single_cta: int = 0, head_ctas: int = 0):
+        t = _Tuning(lm_tile_n, lm_stages, head_tile_n, head_stages, lm_single_cta, head_ctas)
         _check(self.lib.wisv_set_tuning(self._h, C.byref(t)), "wisv_set_tuning")
 
     def launch_count(self) -> int:

@@ -97,7 +97,7 @@ struct wisv_ctx {
     long long prof_calls = 0;
     cudaEvent_t* prof_ev = nullptr;   // [prof_n][kStages + 1]
     long long launches = 0;
-    wisv_tuning tune = {0, 0, 0, 0, 0};
+    wisv_tuning tune = {0, 0, 0, 0, 0, 0};
     HostStaging hs;
 };
 
@@ -130,7 +130,7 @@ size_t gemm_fixed_bytes(int tile_n, int a_rows, int d_c)
 }
 
 // stage count, tile geometry -> shared memory; fills stages / smem of the plan
-void finish_plan(const wisv_ctx* c, Plan* p, int d_c, int k_blocks, int forced_stages)
+void finish_plan(const wisv_ctx* c, Plan* p, int d_c, int k_blocks, int forced_stages, int sms)
 {
     const size_t fixed = gemm_fixed_bytes(p->tile_n, p->a_rows, d_c);
     const size_t stage = gemm_stage_bytes(p->tile_n, p->a_rows);
@@ -142,7 +142,7 @@ void finish_plan(const wisv_ctx* c, Plan* p, int d_c, int k_blocks, int forced_s
     p->smem = fixed + (size_t)s * stage;
     if (p->k_splits < 1) { p->k_splits = 1; p->kb_per_split = k_blocks; }
     const long long items = (long long)p->m_tiles * p->n_tiles * p->k_splits;
-    p->ctas = (int)(items < c->sm_count ? items : c->sm_count);
+    p->ctas = (int)(items < sms ? items : sms);
     p->carry = (p->m_tiles == 1 && p->k_splits == 1) ? 1 : 0;
     p->parts = p->carry ? p->ctas : p->n_tiles;
 }
@@ -156,9 +156,10 @@ double wave_eff(long long tiles, int sms)
 // LM head: with a single row tile the kernel streams the weights once and is
 // HBM-bound, so the tile height over the vocabulary is chosen to fill the last
 // wave of CTAs; with many row tiles it is tensor-bound and takes the largest tile.
-Plan plan_lm(const wisv_ctx* c, int R, bool single_only = false)
+Plan plan_lm(const wisv_ctx* c, int R, bool single_only = false, int sms = 0)
 {
     Plan p{};
+    if (sms <= 0) sms = c->sm_count;
     const int V = c->cfg.V;
     p.m_tiles = (R + kTileM - 1) / kTileM;
     // More than one row tile: CTA pairs on 256 x 256 tiles, each weight tile fetched once per pair.  A pair
@@ -192,11 +193,11 @@ Plan plan_lm(const wisv_ctx* c, int R, bool single_only = false)
         // largest tile whose wave efficiency is within half a percent of the best
         double best_eff = -1.0;
         for (int tn = 64; tn <= kMaxTileN; tn += 16) {
-            const double e = wave_eff((V + tn - 1) / tn, c->sm_count);
+            const double e = wave_eff((V + tn - 1) / tn, sms);
             if (e > best_eff) best_eff = e;
         }
         for (int tn = 64; tn <= kMaxTileN; tn += 16)
-            if (wave_eff((V + tn - 1) / tn, c->sm_count) >= best_eff - 0.005) best = tn;
+            if (wave_eff((V + tn - 1) / tn, sms) >= best_eff - 0.005) best = tn;
     } else {
         best = kMaxTileN;
     }
@@ -204,7 +205,7 @@ Plan plan_lm(const wisv_ctx* c, int R, bool single_only = false)
     p.tile_n = best;
     p.n_tiles = (V + best - 1) / best;
     p.a_rows = p.m_tiles == 1 ? round_up(R, 8) : kTileM;
-    finish_plan(c, &p, 0, (c->cfg.H + kBlockK - 1) / kBlockK, c->tune.lm_stages);
+    finish_plan(c, &p, 0, (c->cfg.H + kBlockK - 1) / kBlockK, c->tune.lm_stages, sms);
     return p;
 }
 
@@ -243,8 +244,33 @@ Plan plan_head(const wisv_ctx* c, int P)
     p.tile_n = best;
     p.n_tiles = (N + best - 1) / best;
     p.a_rows = p.m_tiles == 1 ? round_up(P, 8) : kTileM;
-    finish_plan(c, &p, c->cfg.d_c, k_blocks, c->tune.head_stages);
+    finish_plan(c, &p, c->cfg.d_c, k_blocks, c->tune.head_stages, c->sm_count);
     return p;
+}
+
+// Small batches (one row tile of window rows, one of head positions): the two GEMMs share one launch.
+// The decision head gets a few CTAs of its own - enough to finish well inside the time the LM head needs
+// to stream its weights - and the LM head is planned for the SMs that remain.
+constexpr int kFusedHeadCtas = 8;
+bool plan_fused(const wisv_ctx* c, int R, int P, Plan* lm, Plan* hd)
+{
+    if (c->tune.head_ctas < 0 || R < 1 || P < 1 || R > kTileM || P > kTileM) return false;
+    int want = c->tune.head_ctas > 0 ? c->tune.head_ctas : kFusedHeadCtas;
+    if (want > c->sm_count / 2) want = c->sm_count / 2;
+    if (want < 1) return false;
+    Plan h{};
+    const int N = c->cfg.d_J;
+    int tn = kSplitTileN;
+    if (c->tune.head_tile_n >= 16 && c->tune.head_tile_n <= kMaxTileN && c->tune.head_tile_n % 16 == 0) tn = c->tune.head_tile_n;
+    if (tn > round_up(N, 16)) tn = round_up(N, 16);
+    h.m_tiles = 1; h.tile_n = tn; h.n_tiles = (N + tn - 1) / tn;
+    h.a_rows = round_up(P, 8);
+    h.k_splits = 1;
+    h.kb_per_split = (c->cfg.H_d + c->cfg.H + kBlockK - 1) / kBlockK;
+    finish_plan(c, &h, c->cfg.d_c, h.kb_per_split, c->tune.head_stages, want);
+    *hd = h;
+    *lm = plan_lm(c, R, true, c->sm_count - h.ctas);
+    return true;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -452,6 +478,8 @@ int wisv_create(const wisv_config* cfg, const wisv_weights* w, wisv_ctx** out)
                                    (int)prop.sharedMemPerBlockOptin));
     WISV_CUDA(cudaFuncSetAttribute(lmhead_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)prop.sharedMemPerBlockOptin));
+    WISV_CUDA(cudaFuncSetAttribute(round_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)prop.sharedMemPerBlockOptin));
 
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -562,15 +590,26 @@ int wisv_plan(const wisv_ctx* c, int32_t R, int32_t P, int32_t* lm_tile_n, int32
               int32_t* head_tile_n, int32_t* head_tiles, int32_t* head_ctas)
 {
     if (!c || R < 1 || P < 0) return WISV_EINVAL;
-    const Plan a = plan_lm(c, R);
+    Plan a, h;
+    if (!plan_fused(c, R, P, &a, &h)) {
+        a = plan_lm(c, R);
+        h = plan_head(c, P > 0 ? P : 1);
+    }
     if (lm_tile_n) *lm_tile_n = a.tile_n;
     if (lm_tiles) *lm_tiles = a.m_tiles * a.n_tiles;
     if (lm_ctas) *lm_ctas = a.ctas;
-    const Plan h = plan_head(c, P > 0 ? P : 1);
     if (head_tile_n) *head_tile_n = h.tile_n;
     if (head_tiles) *head_tiles = P > 0 ? h.m_tiles * h.n_tiles : 0;
     if (head_ctas) *head_ctas = P > 0 ? h.ctas : 0;
     return WISV_OK;
+}
+
+int wisv_plan_kernels(const wisv_ctx* c, int32_t R, int32_t P)
+{
+    if (!c || R < 1 || P < 0) return WISV_EINVAL;
+    Plan a, h;
+    if (plan_fused(c, R, P, &a, &h)) return 3;        // pack, LM head + decision head, merge/scan
+    return P > 0 ? 4 : 3;
 }
 
 int64_t wisv_launch_count(const wisv_ctx* c) { return c ? c->launches : 0; }
@@ -578,7 +617,7 @@ int64_t wisv_launch_count(const wisv_ctx* c) { return c ? c->launches : 0; }
 int wisv_set_tuning(wisv_ctx* c, const wisv_tuning* t)
 {
     if (!c) return WISV_EINVAL;
-    if (!t) { c->tune = wisv_tuning{0, 0, 0, 0, 0}; return WISV_OK; }
+    if (!t) { c->tune = wisv_tuning{0, 0, 0, 0, 0, 0}; return WISV_OK; }
     const int32_t tn[2] = {t->lm_tile_n, t->head_tile_n};
     for (int i = 0; i < 2; ++i)
         if (tn[i] != 0 && (tn[i] < 16 || tn[i] > kMaxTileN || tn[i] % 16)) return WISV_ESHAPE;
@@ -654,9 +693,25 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
 
     // ---- 2. LM head: logits reduced on the fly
     if (ev) WISV_CUDA(cudaEventRecord(ev[1], st));
-    const Plan pl = plan_lm(c, R);
+    Plan pl{}, ph{};
+    const bool fused = phase == PHASE_FULL && plan_fused(c, R, P, &pl, &ph);
+    if (!fused) pl = plan_lm(c, R);
     if ((size_t)R * pl.parts > c->lm_part_elems) return WISV_ECAPACITY;
-    if (!rows_done && pl.pair) {
+    if (fused) {
+        // both GEMMs in one launch: LM-head CTAs and decision-head CTAs side by side
+        if ((size_t)P * ph.parts > c->head_part_elems) return WISV_ECAPACITY;
+        GemmParams gl = base_params(c, pl, R, cf.V, cf.H);
+        gl.lm_part = c->lm_part; gl.row_tok = c->row_tok; gl.tok_logit = c->tok_logit;
+        GemmParams gh = base_params(c, ph, P, cf.d_J, cf.H_d + cf.H);
+        gh.head_part = c->head_part; gh.b1 = c->w.b1; gh.w2 = c->w.w2; gh.w1c = c->W1c; gh.csi = b->csi;
+        gh.pos_req = c->pos_req; gh.d_c = cf.d_c; gh.act = cf.act;
+        const size_t smem = pl.smem > ph.smem ? pl.smem : ph.smem;
+        const int rc = launch_pdl(round_small_kernel, dim3(pl.ctas + ph.ctas), dim3(kGemmThreads), smem, st,
+                                  c->tmX[pl.a_rows / 8 - 1], c->tmW[pl.tile_n / 16 - 1], c->tmZ[ph.a_rows / 8 - 1],
+                                  c->tmW1[ph.tile_n / 16 - 1], gl, gh, pl.ctas);
+        if (rc != WISV_OK) return rc;
+        c->launches++;
+    } else if (!rows_done && pl.pair) {
         PairParams qp;
         memset(&qp, 0, sizeof qp);
         qp.rows = R; qp.n_total = cf.V; qp.k_blocks = (cf.H + kBlockK - 1) / kBlockK; qp.mp_tiles = pl.m_tiles;
@@ -694,8 +749,7 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
 
     // ---- 3. decision head on the evaluated positions
     if (ev) WISV_CUDA(cudaEventRecord(ev[2], st));
-    Plan ph{};
-    if (P > 0) {
+    if (P > 0 && !fused) {
         ph = plan_head(c, P);
         if ((size_t)P * ph.parts > c->head_part_elems) return WISV_ECAPACITY;
         GemmParams gp = base_params(c, ph, P, cf.d_J, cf.H_d + cf.H);

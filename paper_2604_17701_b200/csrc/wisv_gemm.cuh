@@ -123,10 +123,11 @@ __device__ __forceinline__ void lm_update_chunk(const uint32_t (&v)[16], int col
     }
 }
 
-template <int EPI>
-__global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                      const GemmParams p)
+// The work of CTA `cta` of `ncta` CTAs that share the tiles of one GEMM.  HEAD_WAITS_LAST selects where
+// the decision-head CTAs synchronise with the preceding kernels of the stream (see below).
+template <int EPI, bool HEAD_WAITS_LAST>
+__device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, const CUtensorMap& tmB,
+                                                    const GemmParams& p, const int cta, const int ncta)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
@@ -182,14 +183,17 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     const uint32_t tmem_base = *tmem_slot;
 
     // Everything above overlaps the previous kernel in the stream.  The LM-head and raw kernels read
-    // what the pack kernel wrote, so they wait for it here.  The decision-head kernel also reads only
-    // pack output, which is complete by the time it can be scheduled (the LM-head kernel releases its
-    // dependents only after its own wait); it waits at its end instead, so that "head kernel complete"
-    // implies "LM-head kernel complete" for the merge/scan kernel that follows.
-    // The producer thread of those kernels waits a little later: weight tiles do not depend on the
+    // what the pack kernel wrote, so they wait for it here.  A decision-head kernel launched after the
+    // LM-head kernel (HEAD_WAITS_LAST) also reads only pack output, which is complete by the time it can
+    // be scheduled (the LM-head kernel releases its dependents only after its own wait); it waits at its
+    // end instead, so that "head kernel complete" implies "LM-head kernel complete" for the merge/scan
+    // kernel that follows.  Decision-head CTAs that share a launch with the LM head follow the pack
+    // kernel directly and wait here like the others.
+    // The producer thread of the early waiters waits a little later: weight tiles do not depend on the
     // pack kernel, so it first puts one ring-full of them in flight.
+    constexpr bool kWaitLast = (EPI == EPI_HEAD) && HEAD_WAITS_LAST;
     const bool producer_thread = warp == 0 && lane == 0;
-    if (EPI != EPI_HEAD && !producer_thread) griddep_wait();
+    if (!kWaitLast && !producer_thread) griddep_wait();
     griddep_launch_dependents();
 
     if (warp == 0) {
@@ -200,8 +204,8 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             long long issued = 0;
             bool ok = true;
             long long pre = 0;                 // stages whose weight tile was requested before the wait
-            if (EPI != EPI_HEAD) {
-                for (int t = blockIdx.x; t < total_tiles && pre < p.stages; t += gridDim.x) {
+            if (!kWaitLast) {
+                for (int t = cta; t < total_tiles && pre < p.stages; t += ncta) {
                     const int n = item_n(t);
                     const int kb1 = item_kb1(t);
                     for (int kb = item_kb0(t); kb < kb1 && pre < p.stages; ++kb, ++pre) {
@@ -212,7 +216,7 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 }
                 griddep_wait();                // from here on the activation rows may be read
             }
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            for (int t = cta; t < total_tiles && ok; t += ncta) {
                 const int m = item_m(t), n = item_n(t);
                 const int kb1 = item_kb1(t);
                 for (int kb = item_kb0(t); kb < kb1; ++kb) {
@@ -249,7 +253,7 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             uint32_t ph = 0;
             int local = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++local) {
+            for (int t = cta; t < total_tiles && ok; t += ncta, ++local) {
                 const int as = local & 1;
                 const uint32_t aph = (local >> 1) & 1u;
                 if (!mbar_wait_bounded(acc_empty_bar(as), aph ^ 1u, abort_flag, kWaitLimitNs)) { ok = false; break; }
@@ -286,7 +290,7 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         bool ok = true;
         float mx = -CUDART_INF_F, sum = 0.0f, hs = 0.0f;   // running row state (per tile, or per CTA when carry)
         int arg = 0;
-        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++local) {
+        for (int t = cta; t < total_tiles && ok; t += ncta, ++local) {
             const int m = item_m(t), n = item_n(t);
             const int as = local & 1;
             const uint32_t aph = (local >> 1) & 1u;
@@ -441,9 +445,9 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             const int row = q * 32 + lane;
             if (row < p.rows) {
                 if (EPI == EPI_LMHEAD)
-                    p.lm_part[(size_t)row * p.part_stride + blockIdx.x] = make_float4(mx, __int_as_float(arg), sum, 0.0f);
+                    p.lm_part[(size_t)row * p.part_stride + cta] = make_float4(mx, __int_as_float(arg), sum, 0.0f);
                 else if (EPI == EPI_HEAD)
-                    p.head_part[(size_t)row * p.part_stride + blockIdx.x] = hs;
+                    p.head_part[(size_t)row * p.part_stride + cta] = hs;
             }
         }
     }
@@ -454,8 +458,32 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         tc_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
     }
-    if (EPI == EPI_HEAD) griddep_wait();
+    if (kWaitLast) griddep_wait();
     if (threadIdx.x == 0 && (abort_flag[0] != 0)) atomicOr(p.err, 1);
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                      const GemmParams p)
+{
+    gemm_rowreduce_body<EPI, true>(tmA, tmB, p, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x));
+}
+
+// One row tile of window rows and one of head positions (small batches, where the LM head streams the
+// weights at HBM speed and the decision head is a latency-bound 12 MB side stream): both GEMMs in one
+// launch.  The first lm_ctas CTAs reduce the LM head, the others evaluate the decision head at the
+// same time, so the round no longer pays for the head after the LM head has finished.
+static __global__ void __launch_bounds__(kGemmThreads, 1)
+round_small_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
+                   const __grid_constant__ CUtensorMap tmZ, const __grid_constant__ CUtensorMap tmW1,
+                   const GemmParams lm, const GemmParams hd, const int lm_ctas)
+{
+    const int cta = static_cast<int>(blockIdx.x);
+    if (cta < lm_ctas)
+        gemm_rowreduce_body<EPI_LMHEAD, false>(tmX, tmW, lm, cta, lm_ctas);
+    else
+        gemm_rowreduce_body<EPI_HEAD, false>(tmZ, tmW1, hd, cta - lm_ctas, static_cast<int>(gridDim.x) - lm_ctas);
 }
 
 }  // namespace wisv

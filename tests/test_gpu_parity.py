@@ -86,22 +86,64 @@ def test_shapes(kw):
                                 dict(B=5, K=3, act="relu"), dict(B=20, K=5, d_J=200)],
                          ids=["P16", "P16dc3", "P3odd", "P15relu", "P100"])
 def test_split_k_head_matches_single_pass_head(kw):
-    """One row tile of positions: the head GEMM splits K over CTAs; forcing a tile height turns that off."""
+    """One row tile of positions, the head in a launch of its own: the head GEMM splits K over CTAs;
+    forcing a tile height turns that off."""
     cfg = _small(seed=17, **kw)
-    case, ref, out, _ = _run(cfg)
+    case, ref, _, _ = _run(cfg)
     d = cases.to_device(case, DEV)
     v = cases.make_verifier(d)
-    v.set_tuning(head_tile_n=16)
+    P = case["T"]
+    v.set_tuning(head_ctas=-1)
+    assert v.plan_kernels(case["R"], P) == 4
     for _ in range(2):                       # twice: the split-K tile counters must have reset themselves
-        o2 = cases.run(v, d)
+        out = cases.run(v, d)
+    torch.cuda.synchronize()
+    assert v.device_error() == 0
+    compare(case, ref, out, cfg.tau)
+    v.set_tuning(head_ctas=-1, head_tile_n=16)
+    o2 = cases.run(v, d)
     torch.cuda.synchronize()
     assert v.device_error() == 0
     compare(case, ref, o2, cfg.tau)
     assert float((o2.head_prob - out.head_prob).abs().max()) < 1e-5
     assert torch.equal(o2.accept_len, out.accept_len)
-    v.set_tuning()
+    v.set_tuning(head_ctas=-1)
     o3 = cases.run(v, d)
     assert torch.equal(o3.head_prob, out.head_prob)      # deterministic from call to call
+    v.close()
+
+
+@pytest.mark.parametrize("kw", [dict(B=2, K=8), dict(B=3, K=1, H=72, H_d=40, d_J=50), dict(B=20, K=5, d_J=200),
+                                dict(B=14, K=8, d_c=3, act="relu"), dict(B=16, K=0, K_lo=1, K_hi=7)],
+                         ids=["P16", "P3odd", "P100", "P112relu", "ragged"])
+@pytest.mark.parametrize("head_ctas", [0, 1, 3, 40])
+def test_one_launch_for_both_gemms_matches_separate_launches(kw, head_ctas):
+    """At most 128 window rows and 128 head positions: LM-head CTAs and decision-head CTAs share a launch
+    (three kernels per round); the result must not depend on how the CTAs are divided, and must equal the
+    four-kernel round up to the fp32 summation order of the head partials."""
+    cfg = _small(seed=29, **kw)
+    case = cases.make_case(cfg, oracle_ref_argmax)
+    ref = run_oracle(case)
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d)
+    v.set_tuning(head_ctas=head_ctas)
+    assert v.plan_kernels(case["R"], case["T"]) == 3
+    plan = v.plan(case["R"], case["T"])
+    assert plan["head_ctas"] >= 1 and plan["lm_ctas"] >= 1
+    n0 = v.launch_count()
+    for _ in range(2):
+        out = cases.run(v, d)
+    torch.cuda.synchronize()
+    assert v.launch_count() - n0 == 6
+    assert v.device_error() == 0
+    compare(case, ref, out, cfg.tau)
+    v.set_tuning(head_ctas=-1)
+    sep = cases.run(v, d)
+    torch.cuda.synchronize()
+    assert torch.equal(sep.argmax, out.argmax) and torch.equal(sep.accept_len, out.accept_len)
+    assert torch.equal(sep.correction_token, out.correction_token)
+    assert float((sep.lse - out.lse).abs().max()) < 1e-5
+    assert float((sep.head_prob - out.head_prob).abs().max()) < 1e-5
     v.close()
 
 
