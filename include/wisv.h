@@ -249,6 +249,7 @@ typedef struct {
     int32_t lm_single_cta;   /* 1: never use the CTA-pair LM-head kernel (batches with more than 128 window rows) */
     int32_t head_ctas;       /* batches of at most 128 window rows and 128 head positions run both GEMMs in one
                                 launch: CTAs given to the decision head there (0 = default), -1 = two launches */
+    int32_t lm_mma_m;        /* 128: never use 64-row MMAs (the default for GEMMs with at most 64 valid rows) */
 } wisv_tuning;
 int wisv_set_tuning(wisv_ctx* ctx, const wisv_tuning* tuning);
 

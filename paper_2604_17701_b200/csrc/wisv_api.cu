@@ -39,6 +39,7 @@ struct Plan {
     int pair;        // LM head on CTA pairs (256 x 256 tiles): m_tiles then counts tiles of 256 rows
     int k_splits;    // work items per (m, n) tile along K (decision head with one row tile)
     int kb_per_split;
+    int units_base, units_rem, tiles_per_cta;   // carry: contiguous ranges of 16-row units per CTA
     size_t smem;
 };
 
@@ -97,7 +98,7 @@ struct wisv_ctx {
     long long prof_calls = 0;
     cudaEvent_t* prof_ev = nullptr;   // [prof_n][kStages + 1]
     long long launches = 0;
-    wisv_tuning tune = {0, 0, 0, 0, 0, 0};
+    wisv_tuning tune = {0, 0, 0, 0, 0, 0, 0};
     HostStaging hs;
 };
 
@@ -130,8 +131,31 @@ size_t gemm_fixed_bytes(int tile_n, int a_rows, int d_c)
 }
 
 // stage count, tile geometry -> shared memory; fills stages / smem of the plan
-void finish_plan(const wisv_ctx* c, Plan* p, int d_c, int k_blocks, int forced_stages, int sms)
+// On entry tile_n is the largest tile height allowed; n_total = rows of the weight matrix.
+void finish_plan(const wisv_ctx* c, Plan* p, int d_c, int k_blocks, int forced_stages, int sms, int n_total)
 {
+    if (p->k_splits < 1) { p->k_splits = 1; p->kb_per_split = k_blocks; }
+    p->carry = (p->m_tiles == 1 && p->k_splits == 1) ? 1 : 0;
+    if (p->carry) {
+        // One row tile and no split of K: every CTA gets one contiguous range of the weight rows, in units
+        // of 16 rows, base or base + 1 units each, and cuts it into tiles of (nearly) equal height.  The CTAs
+        // then finish together whatever the number of rows and CTAs - there is no last, partly filled wave.
+        const int units = (n_total + 15) / 16;
+        const int ctas = units < sms ? units : sms;
+        p->units_base = units / ctas;
+        p->units_rem = units % ctas;
+        const int umax = p->units_base + (p->units_rem ? 1 : 0);
+        const int cap = p->tile_n / 16 > 0 ? p->tile_n / 16 : 1;
+        p->tiles_per_cta = (umax + cap - 1) / cap;
+        p->tile_n = (umax + p->tiles_per_cta - 1) / p->tiles_per_cta * 16;
+        p->ctas = ctas;
+        p->n_tiles = ctas * p->tiles_per_cta;
+        p->parts = ctas;
+    } else {
+        const long long items = (long long)p->m_tiles * p->n_tiles * p->k_splits;
+        p->ctas = (int)(items < sms ? items : sms);
+        p->parts = p->n_tiles;
+    }
     const size_t fixed = gemm_fixed_bytes(p->tile_n, p->a_rows, d_c);
     const size_t stage = gemm_stage_bytes(p->tile_n, p->a_rows);
     int s = (int)(((size_t)c->max_smem - fixed) / stage);
@@ -140,11 +164,6 @@ void finish_plan(const wisv_ctx* c, Plan* p, int d_c, int k_blocks, int forced_s
     if (forced_stages >= 2 && forced_stages < s) s = forced_stages;
     p->stages = s;
     p->smem = fixed + (size_t)s * stage;
-    if (p->k_splits < 1) { p->k_splits = 1; p->kb_per_split = k_blocks; }
-    const long long items = (long long)p->m_tiles * p->n_tiles * p->k_splits;
-    p->ctas = (int)(items < sms ? items : sms);
-    p->carry = (p->m_tiles == 1 && p->k_splits == 1) ? 1 : 0;
-    p->parts = p->carry ? p->ctas : p->n_tiles;
 }
 
 double wave_eff(long long tiles, int sms)
@@ -189,23 +208,16 @@ Plan plan_lm(const wisv_ctx* c, int R, bool single_only = false, int sms = 0)
     int best = 0;
     if (c->tune.lm_tile_n >= 16 && c->tune.lm_tile_n <= kMaxTileN && c->tune.lm_tile_n % 16 == 0) {
         best = c->tune.lm_tile_n;
-    } else if (p.m_tiles == 1) {
-        // largest tile whose wave efficiency is within half a percent of the best
-        double best_eff = -1.0;
-        for (int tn = 64; tn <= kMaxTileN; tn += 16) {
-            const double e = wave_eff((V + tn - 1) / tn, sms);
-            if (e > best_eff) best_eff = e;
-        }
-        for (int tn = 64; tn <= kMaxTileN; tn += 16)
-            if (wave_eff((V + tn - 1) / tn, sms) >= best_eff - 0.005) best = tn;
     } else {
+        // one row tile (HBM-bound): finish_plan balances the vocabulary over the CTAs, tiles as high as allowed
+        // (fewest MMA instructions per byte streamed); several row tiles (tensor-bound): the largest tile
         best = kMaxTileN;
     }
     if (best > round_up(V, 16)) best = round_up(V, 16);
     p.tile_n = best;
     p.n_tiles = (V + best - 1) / best;
     p.a_rows = p.m_tiles == 1 ? round_up(R, 8) : kTileM;
-    finish_plan(c, &p, 0, (c->cfg.H + kBlockK - 1) / kBlockK, c->tune.lm_stages, sms);
+    finish_plan(c, &p, 0, (c->cfg.H + kBlockK - 1) / kBlockK, c->tune.lm_stages, sms, V);
     return p;
 }
 
@@ -244,14 +256,14 @@ Plan plan_head(const wisv_ctx* c, int P)
     p.tile_n = best;
     p.n_tiles = (N + best - 1) / best;
     p.a_rows = p.m_tiles == 1 ? round_up(P, 8) : kTileM;
-    finish_plan(c, &p, c->cfg.d_c, k_blocks, c->tune.head_stages, c->sm_count);
+    finish_plan(c, &p, c->cfg.d_c, k_blocks, c->tune.head_stages, c->sm_count, N);
     return p;
 }
 
 // Small batches (one row tile of window rows, one of head positions): the two GEMMs share one launch.
 // The decision head gets a few CTAs of its own - enough to finish well inside the time the LM head needs
 // to stream its weights - and the LM head is planned for the SMs that remain.
-constexpr int kFusedHeadCtas = 8;
+constexpr int kFusedHeadCtas = 6;
 bool plan_fused(const wisv_ctx* c, int R, int P, Plan* lm, Plan* hd)
 {
     if (c->tune.head_ctas < 0 || R < 1 || P < 1 || R > kTileM || P > kTileM) return false;
@@ -267,7 +279,7 @@ bool plan_fused(const wisv_ctx* c, int R, int P, Plan* lm, Plan* hd)
     h.a_rows = round_up(P, 8);
     h.k_splits = 1;
     h.kb_per_split = (c->cfg.H_d + c->cfg.H + kBlockK - 1) / kBlockK;
-    finish_plan(c, &h, c->cfg.d_c, h.kb_per_split, c->tune.head_stages, want);
+    finish_plan(c, &h, c->cfg.d_c, h.kb_per_split, c->tune.head_stages, want, N);
     *hd = h;
     *lm = plan_lm(c, R, true, c->sm_count - h.ctas);
     return true;
@@ -305,6 +317,7 @@ int dev_alloc(T** p, size_t n)
 // Device address of a pinned host array if the kernels can read it in place (registered with CUDA, 16-byte aligned,
 // at most kZeroCopyBytes), else `staged`.
 constexpr size_t kZeroCopyBytes = 1u << 20;
+constexpr size_t kSmallInputsInPlace = 8u << 10;   // packed small inputs up to this size are not copied either
 const float* mapped_or(const float* host, size_t bytes, const float* staged)
 {
     if (!host || bytes == 0 || bytes > kZeroCopyBytes) return staged;
@@ -401,11 +414,17 @@ int launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cud
     return WISV_OK;
 }
 
+// index of the tensor map whose box is `tile_n` weight rows high, and of the one 16 rows lower (the second
+// tile height of a balanced plan; never used when tile_n is 16)
+inline int map_hi(const Plan& pl) { return pl.tile_n / 16 - 1; }
+inline int map_lo(const Plan& pl) { return pl.tile_n / 16 - 2 > 0 ? pl.tile_n / 16 - 2 : 0; }
+
 template <int EPI>
-int launch_gemm(wisv_ctx* c, const CUtensorMap& tA, const CUtensorMap& tB, const GemmParams& gp, const Plan& pl,
+int launch_gemm(wisv_ctx* c, const CUtensorMap& tA, const CUtensorMap* tB, const GemmParams& gp, const Plan& pl,
                 cudaStream_t st)
 {
-    const int rc = launch_pdl(gemm_rowreduce_kernel<EPI>, dim3(pl.ctas), dim3(kGemmThreads), pl.smem, st, tA, tB, gp);
+    const int rc = launch_pdl(gemm_rowreduce_kernel<EPI>, dim3(pl.ctas), dim3(kGemmThreads), pl.smem, st, tA,
+                              tB[map_hi(pl)], tB[map_lo(pl)], gp);
     if (rc != WISV_OK) return rc;
     c->launches++;
     return WISV_OK;
@@ -419,6 +438,9 @@ GemmParams base_params(const wisv_ctx* c, const Plan& pl, int rows, int n_total,
     gp.tile_n = pl.tile_n; gp.m_tiles = pl.m_tiles; gp.n_tiles = pl.n_tiles; gp.stages = pl.stages;
     gp.a_rows = pl.a_rows; gp.carry = pl.carry; gp.part_stride = pl.parts;
     gp.k_splits = pl.k_splits; gp.kb_per_split = pl.kb_per_split;
+    // one row tile with at most 64 valid rows: MMAs of 64 rows do the same job with half the tensor work
+    gp.mma_m = (pl.m_tiles == 1 && rows <= 64 && c->tune.lm_mma_m != kTileM) ? 64 : kTileM;
+    gp.units_base = pl.units_base; gp.units_rem = pl.units_rem; gp.tiles_per_cta = pl.tiles_per_cta;
     gp.splitk_buf = c->splitk_buf; gp.splitk_count = c->splitk_count;
     gp.err = c->err;
     return gp;
@@ -617,11 +639,12 @@ int64_t wisv_launch_count(const wisv_ctx* c) { return c ? c->launches : 0; }
 int wisv_set_tuning(wisv_ctx* c, const wisv_tuning* t)
 {
     if (!c) return WISV_EINVAL;
-    if (!t) { c->tune = wisv_tuning{0, 0, 0, 0, 0, 0}; return WISV_OK; }
+    if (!t) { c->tune = wisv_tuning{0, 0, 0, 0, 0, 0, 0}; return WISV_OK; }
     const int32_t tn[2] = {t->lm_tile_n, t->head_tile_n};
     for (int i = 0; i < 2; ++i)
         if (tn[i] != 0 && (tn[i] < 16 || tn[i] > kMaxTileN || tn[i] % 16)) return WISV_ESHAPE;
     if (t->lm_stages < 0 || t->head_stages < 0 || t->lm_stages == 1 || t->head_stages == 1) return WISV_ESHAPE;
+    if (t->lm_mma_m != 0 && t->lm_mma_m != 64 && t->lm_mma_m != 128) return WISV_ESHAPE;
     c->tune = *t;
     return WISV_OK;
 }
@@ -707,8 +730,8 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
         gh.pos_req = c->pos_req; gh.d_c = cf.d_c; gh.act = cf.act;
         const size_t smem = pl.smem > ph.smem ? pl.smem : ph.smem;
         const int rc = launch_pdl(round_small_kernel, dim3(pl.ctas + ph.ctas), dim3(kGemmThreads), smem, st,
-                                  c->tmX[pl.a_rows / 8 - 1], c->tmW[pl.tile_n / 16 - 1], c->tmZ[ph.a_rows / 8 - 1],
-                                  c->tmW1[ph.tile_n / 16 - 1], gl, gh, pl.ctas);
+                                  c->tmX[pl.a_rows / 8 - 1], c->tmW[map_hi(pl)], c->tmW[map_lo(pl)],
+                                  c->tmZ[ph.a_rows / 8 - 1], c->tmW1[map_hi(ph)], c->tmW1[map_lo(ph)], gl, gh, pl.ctas);
         if (rc != WISV_OK) return rc;
         c->launches++;
     } else if (!rows_done && pl.pair) {
@@ -732,7 +755,7 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
     } else if (!rows_done) {
         GemmParams gp = base_params(c, pl, R, cf.V, cf.H);
         gp.lm_part = c->lm_part; gp.row_tok = c->row_tok; gp.tok_logit = c->tok_logit;
-        const int rc = launch_gemm<EPI_LMHEAD>(c, c->tmX[pl.a_rows / 8 - 1], c->tmW[pl.tile_n / 16 - 1], gp, pl, st);
+        const int rc = launch_gemm<EPI_LMHEAD>(c, c->tmX[pl.a_rows / 8 - 1], c->tmW, gp, pl, st);
         if (rc != WISV_OK) return rc;
     }
 
@@ -755,7 +778,7 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
         GemmParams gp = base_params(c, ph, P, cf.d_J, cf.H_d + cf.H);
         gp.head_part = c->head_part; gp.b1 = c->w.b1; gp.w2 = c->w.w2; gp.w1c = c->W1c; gp.csi = b->csi;
         gp.pos_req = c->pos_req; gp.d_c = cf.d_c; gp.act = cf.act;
-        const int rc = launch_gemm<EPI_HEAD>(c, c->tmZ[ph.a_rows / 8 - 1], c->tmW1[ph.tile_n / 16 - 1], gp, ph, st);
+        const int rc = launch_gemm<EPI_HEAD>(c, c->tmZ[ph.a_rows / 8 - 1], c->tmW1, gp, ph, st);
         if (rc != WISV_OK) return rc;
     }
 
@@ -844,7 +867,7 @@ int wisv_debug_logits(wisv_ctx* c, const float* target_hidden, int32_t R, float*
     const Plan pl = plan_lm(c, R, true);            // the raw-logits epilogue exists for the single-CTA kernel only
     GemmParams gp = base_params(c, pl, R, c->cfg.V, c->cfg.H);
     gp.raw_out = logits_out;
-    return launch_gemm<EPI_RAW>(c, c->tmX[pl.a_rows / 8 - 1], c->tmW[pl.tile_n / 16 - 1], gp, pl, st);
+    return launch_gemm<EPI_RAW>(c, c->tmX[pl.a_rows / 8 - 1], c->tmW, gp, pl, st);
 }
 
 int wisv_debug_wait_probe(wisv_ctx* c, uint64_t limit_cycles, void* cuda_stream)
@@ -957,20 +980,25 @@ int wisv_verify_host(wisv_ctx* c, const wisv_batch* hb, const wisv_result* hr, v
     memset(&dr, 0, sizeof dr);
     const void* src[IN_FIELDS] = {hb->k_off, hb->draft_tokens, sh ? hb->sel_off : nullptr, sh ? hb->sel_pos : nullptr,
                                   hb->csi, stoch ? hb->draft_q : nullptr, stoch ? hb->uniforms : nullptr};
-    db.k_off = hb->k_off ? reinterpret_cast<int32_t*>(h.dev_in + ioff[IN_KOFF]) : nullptr;
+    // A few KB of small inputs are read by the kernels in place from the pinned block (each is touched once or
+    // twice per round, and a separate copy costs more in submission and DMA latency than those reads over PCIe);
+    // larger ones are copied to the device in one piece.
+    const bool small_in_place = in_used <= kSmallInputsInPlace;
+    uint8_t* in_base = small_in_place ? h.pin_dev : h.dev_in;
+    db.k_off = hb->k_off ? reinterpret_cast<int32_t*>(in_base + ioff[IN_KOFF]) : nullptr;
     // a small hidden-state array in pinned memory is read in place by the pack kernel (one pass over PCIe, no
     // separate copy to wait for); a large or pageable one goes through the copy engine
     const size_t th_bytes = sizeof(float) * (size_t)R * cf.H, dh_bytes = sizeof(float) * (size_t)P * cf.H_d;
     const float* th_dev = mapped_or(hb->target_hidden, th_bytes, h.target_hidden);
     const float* dh_dev = mapped_or(hb->draft_hidden, dh_bytes, h.draft_hidden);
     db.target_hidden = hb->target_hidden ? th_dev : nullptr;
-    db.draft_tokens = hb->draft_tokens ? reinterpret_cast<int32_t*>(h.dev_in + ioff[IN_TOK]) : nullptr;
+    db.draft_tokens = hb->draft_tokens ? reinterpret_cast<int32_t*>(in_base + ioff[IN_TOK]) : nullptr;
     db.draft_hidden = hb->draft_hidden ? dh_dev : nullptr;
-    db.sel_off = hb->sel_off ? reinterpret_cast<int32_t*>(h.dev_in + ioff[IN_SELOFF]) : nullptr;
-    db.sel_pos = hb->sel_pos ? reinterpret_cast<int32_t*>(h.dev_in + ioff[IN_SELPOS]) : nullptr;
-    db.csi = hb->csi ? reinterpret_cast<float*>(h.dev_in + ioff[IN_CSI]) : nullptr;
-    db.draft_q = hb->draft_q ? reinterpret_cast<float*>(h.dev_in + ioff[IN_Q]) : nullptr;
-    db.uniforms = hb->uniforms ? reinterpret_cast<float*>(h.dev_in + ioff[IN_U]) : nullptr;
+    db.sel_off = hb->sel_off ? reinterpret_cast<int32_t*>(in_base + ioff[IN_SELOFF]) : nullptr;
+    db.sel_pos = hb->sel_pos ? reinterpret_cast<int32_t*>(in_base + ioff[IN_SELPOS]) : nullptr;
+    db.csi = hb->csi ? reinterpret_cast<float*>(in_base + ioff[IN_CSI]) : nullptr;
+    db.draft_q = hb->draft_q ? reinterpret_cast<float*>(in_base + ioff[IN_Q]) : nullptr;
+    db.uniforms = hb->uniforms ? reinterpret_cast<float*>(in_base + ioff[IN_U]) : nullptr;
     dr.accept_len = hr->accept_len ? reinterpret_cast<int32_t*>(dev_out + ooff[OUT_ACCEPT]) : nullptr;
     dr.correction_token = hr->correction_token ? reinterpret_cast<int32_t*>(dev_out + ooff[OUT_CORR]) : nullptr;
     dr.argmax = hr->argmax ? reinterpret_cast<int32_t*>(dev_out + ooff[OUT_ARGMAX]) : nullptr;
@@ -987,7 +1015,7 @@ int wisv_verify_host(wisv_ctx* c, const wisv_batch* hb, const wisv_result* hr, v
     if (B == 0) return WISV_OK;
     for (int i = 0; i < IN_FIELDS; ++i)
         if (src[i] && ibytes[i] > 0) memcpy(pin_in + ioff[i], src[i], ibytes[i]);
-    WISV_CUDA(cudaMemcpyAsync(h.dev_in, pin_in, in_used, cudaMemcpyHostToDevice, st));
+    if (!small_in_place) WISV_CUDA(cudaMemcpyAsync(h.dev_in, pin_in, in_used, cudaMemcpyHostToDevice, st));
     if (th_dev != h.target_hidden)
         ;   // the pack kernel reads the caller's pinned array in place
     else if (hb->target_hidden)

@@ -71,9 +71,11 @@ __device__ __forceinline__ void cast_row(const float* __restrict__ src, __nv_bfl
 __global__ void __launch_bounds__(256) pack_kernel(const PackParams p)
 {
     __shared__ int s_src_row;
+    // Let the GEMM kernel that follows be scheduled at once: until its own wait it only sets up barriers and
+    // tensor memory and requests weight tiles, which depend on nothing this kernel or its predecessors write.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // the previous round's kernels still read the buffers this kernel rewrites
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int blk = blockIdx.x;
     if (blk < p.R) {
         const int r = blk;
@@ -186,9 +188,11 @@ __global__ void __launch_bounds__(256) tail_kernel(const TailParams p)
     if (threadIdx.x < kMaxK) { s_has[threadIdx.x] = 0; s_prob[threadIdx.x] = 0.0f; }
     if (threadIdx.x == 0) s_flag = 0;
     __syncthreads();
+    // The next round's pack kernel may be scheduled already; it waits for this kernel to complete before it
+    // writes anything, and in turn lets the next GEMM kernel set up and prefetch weights meanwhile.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // partials of the LM-head and decision-head kernels must be complete and visible
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (p.err_copy && b == 0 && threadIdx.x == 0) *p.err_copy = *p.err_src;
 

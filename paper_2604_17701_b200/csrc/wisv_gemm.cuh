@@ -48,8 +48,17 @@ struct GemmParams {
     int32_t a_rows;      // rows of A actually loaded per tile (multiple of 8, <= 128); the MMA still spans
                          // 128 rows, the rest of its A operand is whatever follows in shared memory and only
                          // feeds accumulator rows that are never read
+    int32_t mma_m;       // rows of one MMA: 128 (accumulator row i in TMEM lane i), or 64 when the one row tile has
+                         // at most 64 valid rows (row i in lane (i / 16) * 32 + i % 16: sixteen lanes of each
+                         // quadrant) - half the tensor work per weight byte, which the HBM-bound case turns
+                         // into lower power and higher clocks
     int32_t carry;       // 1: one row tile, each CTA keeps its running row state across its tiles and
                          //    writes one partial per (row, CTA); 0: one partial per (row, N-tile)
+    // carry only: the rows of Bw are dealt out in units of 16 as one contiguous range per CTA - CTA c gets
+    // units_base units, one more if c < units_rem - and each CTA cuts its range into tiles_per_cta tiles
+    // whose heights differ by at most one unit (tile_n is the larger height, tile_n - 16 the smaller).
+    // No CTA then has more than 16 rows more than another, whatever n_total and the number of CTAs.
+    int32_t units_base, units_rem, tiles_per_cta;
     int32_t part_stride; // partials per row (CTAs when carry, else n_tiles)
     int32_t k_splits;    // decision head only: the K range is cut into k_splits work items per (m, n) tile;
                          // each item stores its raw fp32 tile, the last one to finish adds them up in
@@ -127,7 +136,8 @@ __device__ __forceinline__ void lm_update_chunk(const uint32_t (&v)[16], int col
 // the decision-head CTAs synchronise with the preceding kernels of the stream (see below).
 template <int EPI, bool HEAD_WAITS_LAST>
 __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, const CUtensorMap& tmB,
-                                                    const GemmParams& p, const int cta, const int ncta)
+                                                    const CUtensorMap& tmB2, const GemmParams& p,
+                                                    const int cta, const int ncta)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
@@ -162,6 +172,31 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
     auto item_n = [&](int t) { return (t / p.m_tiles) / p.k_splits; };
     auto item_kb0 = [&](int t) { return item_ks(t) * p.kb_per_split; };
     auto item_kb1 = [&](int t) { const int e = (item_ks(t) + 1) * p.kb_per_split; return e < p.k_blocks ? e : p.k_blocks; };
+    // carry: this CTA's contiguous range of 16-row units and how it is cut into tiles
+    const int my_units = p.units_base + (cta < p.units_rem ? 1 : 0);
+    const int my_unit0 = cta * p.units_base + (cta < p.units_rem ? cta : p.units_rem);
+    const int my_tiles = my_units < p.tiles_per_cta ? my_units : p.tiles_per_cta;     // tiles that are not empty
+    const int my_hq = p.carry ? my_units / p.tiles_per_cta : 0;
+    const int my_hr = p.carry ? my_units % p.tiles_per_cta : 0;
+    // The i-th work item of this CTA: row tile m, first row n0 and height h of its block of Bw, column tile
+    // index n and global item number t (both used only without carry), K blocks [kb0, kb1).
+    struct Item { int t, m, n, n0, h, kb0, kb1; };
+    auto item_at = [&](int i, Item& w) -> bool {
+        if (p.carry) {
+            if (i >= my_tiles) return false;
+            w.t = i; w.m = 0; w.n = 0;
+            w.h = (my_hq + (i < my_hr ? 1 : 0)) * 16;
+            w.n0 = (my_unit0 + i * my_hq + (i < my_hr ? i : my_hr)) * 16;
+            w.kb0 = 0; w.kb1 = p.k_blocks;
+            return true;
+        }
+        const int t = cta + i * ncta;
+        if (t >= total_tiles) return false;
+        w.t = t; w.m = item_m(t); w.n = item_n(t); w.n0 = w.n * p.tile_n; w.h = p.tile_n;
+        w.kb0 = item_kb0(t); w.kb1 = item_kb1(t);
+        return true;
+    };
+    auto b_map = [&](int h) -> const CUtensorMap* { return h == p.tile_n ? &tmB : &tmB2; };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -194,7 +229,8 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
     constexpr bool kWaitLast = (EPI == EPI_HEAD) && HEAD_WAITS_LAST;
     const bool producer_thread = warp == 0 && lane == 0;
     if (!kWaitLast && !producer_thread) griddep_wait();
-    griddep_launch_dependents();
+    // no thread of an early waiter lets the next kernel start before it has passed its own wait
+    if (kWaitLast || !producer_thread) griddep_launch_dependents();
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -204,31 +240,31 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
             long long issued = 0;
             bool ok = true;
             long long pre = 0;                 // stages whose weight tile was requested before the wait
+            Item w;
             if (!kWaitLast) {
-                for (int t = cta; t < total_tiles && pre < p.stages; t += ncta) {
-                    const int n = item_n(t);
-                    const int kb1 = item_kb1(t);
-                    for (int kb = item_kb0(t); kb < kb1 && pre < p.stages; ++kb, ++pre) {
+                for (int i = 0; pre < p.stages && item_at(i, w); ++i) {
+                    const uint32_t tx = a_bytes + static_cast<uint32_t>(w.h) * kBlockK * 2;
+                    for (int kb = w.kb0; kb < w.kb1 && pre < p.stages; ++kb, ++pre) {
                         const uint32_t a_dst = smem_base + stage_bytes * static_cast<uint32_t>(pre);
-                        mbar_expect_tx(full_bar(static_cast<int>(pre)), stage_bytes);
-                        tma_load_2d(a_dst + a_bytes, &tmB, kb * kBlockK, n * p.tile_n, full_bar(static_cast<int>(pre)));
+                        mbar_expect_tx(full_bar(static_cast<int>(pre)), tx);
+                        tma_load_2d(a_dst + a_bytes, b_map(w.h), kb * kBlockK, w.n0, full_bar(static_cast<int>(pre)));
                     }
                 }
                 griddep_wait();                // from here on the activation rows may be read
+                griddep_launch_dependents();
             }
-            for (int t = cta; t < total_tiles && ok; t += ncta) {
-                const int m = item_m(t), n = item_n(t);
-                const int kb1 = item_kb1(t);
-                for (int kb = item_kb0(t); kb < kb1; ++kb) {
+            for (int i = 0; ok && item_at(i, w); ++i) {
+                const uint32_t tx = a_bytes + static_cast<uint32_t>(w.h) * kBlockK * 2;
+                for (int kb = w.kb0; kb < w.kb1; ++kb) {
                     const uint32_t a_dst = smem_base + stage_bytes * s;
                     if (issued < pre) {
                         // first pass over the ring: the stage is free and its weight tile is already on its way
-                        tma_load_2d(a_dst, &tmA, kb * kBlockK, m * kTileM, full_bar(s));
+                        tma_load_2d(a_dst, &tmA, kb * kBlockK, w.m * kTileM, full_bar(s));
                     } else {
                         if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, kWaitLimitNs)) { ok = false; break; }
-                        mbar_expect_tx(full_bar(s), stage_bytes);
-                        tma_load_2d(a_dst, &tmA, kb * kBlockK, m * kTileM, full_bar(s));
-                        tma_load_2d(a_dst + a_bytes, &tmB, kb * kBlockK, n * p.tile_n, full_bar(s));
+                        mbar_expect_tx(full_bar(s), tx);
+                        tma_load_2d(a_dst, &tmA, kb * kBlockK, w.m * kTileM, full_bar(s));
+                        tma_load_2d(a_dst + a_bytes, b_map(w.h), kb * kBlockK, w.n0, full_bar(s));
                     }
                     ++issued;
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
@@ -248,18 +284,18 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            const uint32_t idesc = idesc_bf16_f32(kTileM, static_cast<uint32_t>(p.tile_n));
             int s = 0;
             uint32_t ph = 0;
-            int local = 0;
             bool ok = true;
-            for (int t = cta; t < total_tiles && ok; t += ncta, ++local) {
+            Item w;
+            for (int local = 0; ok && item_at(local, w); ++local) {
+                const uint32_t idesc = idesc_bf16_f32(static_cast<uint32_t>(p.mma_m), static_cast<uint32_t>(w.h));
                 const int as = local & 1;
                 const uint32_t aph = (local >> 1) & 1u;
                 if (!mbar_wait_bounded(acc_empty_bar(as), aph ^ 1u, abort_flag, kWaitLimitNs)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(as * kAccCols);
-                const int kb0 = item_kb0(t), kb1 = item_kb1(t);
+                const int kb0 = w.kb0, kb1 = w.kb1;
                 for (int kb = kb0; kb < kb1; ++kb) {
                     if (!mbar_wait_bounded(full_bar(s), ph, abort_flag, kWaitLimitNs)) { ok = false; break; }
                     tc_fence_after();
@@ -286,17 +322,20 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
         // ------------------------------------------------------------ epilogue (warps 2..5)
         const int q = warp & 3;                            // TMEM lane quadrant this warp may read
         const int et = threadIdx.x - 64;                   // 0..127 among epilogue threads
-        int local = 0;
+        // row of the tile held by this thread's TMEM lane (see GemmParams::mma_m)
+        const int rit = p.mma_m == 64 ? q * 16 + (lane & 15) : q * 32 + lane;
+        const bool lane_used = p.mma_m == 64 ? lane < 16 : true;
         bool ok = true;
         float mx = -CUDART_INF_F, sum = 0.0f, hs = 0.0f;   // running row state (per tile, or per CTA when carry)
         int arg = 0;
-        for (int t = cta; t < total_tiles && ok; t += ncta, ++local) {
-            const int m = item_m(t), n = item_n(t);
+        Item w;
+        for (int local = 0; ok && item_at(local, w); ++local) {
+            const int t = w.t, m = w.m, n = w.n;
             const int as = local & 1;
             const uint32_t aph = (local >> 1) & 1u;
-            const int row = m * kTileM + q * 32 + lane;
-            const bool valid = row < p.rows;
-            const int n0 = n * p.tile_n;
+            const int row = m * kTileM + rit;
+            const bool valid = lane_used && row < p.rows;
+            const int n0 = w.n0;
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(as * kAccCols);
 
             const float* cb1 = nullptr; const float* cw2 = nullptr; const float* cwc = nullptr; const float* ccs = nullptr;
@@ -315,8 +354,9 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
                 }
                 const int rq = valid ? p.pos_req[row] : 0;
                 // indexed by row within the tile (this thread's TMEM lane), not by thread number
-                for (int c = 0; c < p.d_c; ++c)
-                    wcs[c * kEpiThreads + q * 32 + lane] = valid ? p.csi[(size_t)rq * p.d_c + c] : 0.0f;
+                if (lane_used)
+                    for (int c = 0; c < p.d_c; ++c)
+                        wcs[c * kEpiThreads + rit] = valid ? p.csi[(size_t)rq * p.d_c + c] : 0.0f;
                 cb1 = wb1; cw2 = ww2; cwc = wwc; ccs = wcs;
             }
 
@@ -342,7 +382,7 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
             if (!p.carry) { mx = -CUDART_INF_F; sum = 0.0f; hs = 0.0f; arg = 0; }
             const int tok = (EPI == EPI_LMHEAD && valid) ? p.row_tok[row] : -1;
 
-            for (int c0 = 0; c0 < p.tile_n; c0 += 16) {
+            for (int c0 = 0; c0 < w.h; c0 += 16) {
                 uint32_t v[16];
                 __syncwarp();                                // tcgen05.ld is warp-collective
                 tmem_ld16(taddr + static_cast<uint32_t>(c0), v);
@@ -354,7 +394,7 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
                 } else if (EPI == EPI_HEAD && p.k_splits > 1) {
                     // split K: park the raw partial tile; the last item of this (m, n) tile finishes it
                     float4* dst = reinterpret_cast<float4*>(
-                        p.splitk_buf + ((size_t)t * kTileM + (q * 32 + lane)) * p.tile_n + c0);
+                        p.splitk_buf + ((size_t)t * kTileM + rit) * p.tile_n + c0);
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
                         dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
@@ -364,7 +404,7 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
 #pragma unroll
                     for (int j = 0; j < 16; ++j) pre[j] = __uint_as_float(v[j]) + cb1[c0 + j];
                     for (int c = 0; c < p.d_c; ++c) {
-                        const float x = ccs[c * kEpiThreads + q * 32 + lane];
+                        const float x = ccs[c * kEpiThreads + rit];
 #pragma unroll
                         for (int j = 0; j < 16; ++j) pre[j] = fmaf(x, cwc[c * p.tile_n + c0 + j], pre[j]);
                     }
@@ -442,8 +482,8 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
         if (p.carry && ok) {
             // one row tile: tiles of this CTA ascend through the vocabulary, so the strict '>' above
             // already kept the lowest index; a CTA without tiles is never launched
-            const int row = q * 32 + lane;
-            if (row < p.rows) {
+            const int row = rit;
+            if (lane_used && row < p.rows) {
                 if (EPI == EPI_LMHEAD)
                     p.lm_part[(size_t)row * p.part_stride + cta] = make_float4(mx, __int_as_float(arg), sum, 0.0f);
                 else if (EPI == EPI_HEAD)
@@ -465,9 +505,9 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
 template <int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                      const GemmParams p)
+                      const __grid_constant__ CUtensorMap tmB2, const GemmParams p)
 {
-    gemm_rowreduce_body<EPI, true>(tmA, tmB, p, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x));
+    gemm_rowreduce_body<EPI, true>(tmA, tmB, tmB2, p, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x));
 }
 
 // One row tile of window rows and one of head positions (small batches, where the LM head streams the
@@ -476,14 +516,16 @@ gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 // same time, so the round no longer pays for the head after the LM head has finished.
 static __global__ void __launch_bounds__(kGemmThreads, 1)
 round_small_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
-                   const __grid_constant__ CUtensorMap tmZ, const __grid_constant__ CUtensorMap tmW1,
+                   const __grid_constant__ CUtensorMap tmW_2, const __grid_constant__ CUtensorMap tmZ,
+                   const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUtensorMap tmW1_2,
                    const GemmParams lm, const GemmParams hd, const int lm_ctas)
 {
     const int cta = static_cast<int>(blockIdx.x);
     if (cta < lm_ctas)
-        gemm_rowreduce_body<EPI_LMHEAD, false>(tmX, tmW, lm, cta, lm_ctas);
+        gemm_rowreduce_body<EPI_LMHEAD, false>(tmX, tmW, tmW_2, lm, cta, lm_ctas);
     else
-        gemm_rowreduce_body<EPI_HEAD, false>(tmZ, tmW1, hd, cta - lm_ctas, static_cast<int>(gridDim.x) - lm_ctas);
+        gemm_rowreduce_body<EPI_HEAD, false>(tmZ, tmW1, tmW1_2, hd, cta - lm_ctas,
+                                             static_cast<int>(gridDim.x) - lm_ctas);
 }
 
 }  // namespace wisv

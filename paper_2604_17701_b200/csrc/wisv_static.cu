@@ -207,7 +207,7 @@ extern "C" int wisv_lm_head_reduce_static(const void* lm_head, int32_t V, int32_
     GemmParams gp;
     memset(&gp, 0, sizeof gp);
     gp.rows = R; gp.n_total = V; gp.k_blocks = (H + kBlockK - 1) / kBlockK; gp.tile_n = tile_n;
-    gp.m_tiles = 1; gp.n_tiles = n_tiles; gp.a_rows = kTileM; gp.carry = 0; gp.part_stride = n_tiles;
+    gp.m_tiles = 1; gp.n_tiles = n_tiles; gp.a_rows = kTileM; gp.mma_m = kTileM; gp.carry = 0; gp.part_stride = n_tiles;
     gp.k_splits = 1; gp.kb_per_split = gp.k_blocks;
     const size_t fixed = 1024 + gemm_tail_bytes(tile_n, 0);
     int stages = (int)(((size_t)s->max_smem - fixed) / gemm_stage_bytes(tile_n));
@@ -216,7 +216,7 @@ extern "C" int wisv_lm_head_reduce_static(const void* lm_head, int32_t V, int32_
     gp.err = err; gp.lm_part = part; gp.row_tok = row_tok; gp.tok_logit = tok_logit;
     const size_t smem = fixed + (size_t)stages * gemm_stage_bytes(tile_n);
     const int ctas = n_tiles < s->sm_count ? n_tiles : s->sm_count;
-    gemm_rowreduce_kernel<EPI_LMHEAD><<<ctas, kGemmThreads, smem, st>>>(tmX, tmW, gp);
+    gemm_rowreduce_kernel<EPI_LMHEAD><<<ctas, kGemmThreads, smem, st>>>(tmX, tmW, tmW, gp);
 
     static_merge_rows_kernel<<<(R + 3) / 4, 128, 0, st>>>(part, n_tiles, R, err, argmax, lse);
     if (cudaGetLastError() != cudaSuccess) return WISV_ECUDA;

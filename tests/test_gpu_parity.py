@@ -164,6 +164,34 @@ def test_cta_pair_kernel_matches_single_cta_kernel():
     v.close()
 
 
+@pytest.mark.parametrize("B,K", [(1, 8), (4, 3), (2, 8), (8, 4), (7, 8), (8, 7), (13, 4)],
+                         ids=["R9", "R16", "R18", "R40", "R63", "R64", "R65"])
+@pytest.mark.parametrize("head_ctas", [0, -1], ids=["one_launch", "two_launches"])
+def test_mma_of_64_rows_matches_mma_of_128_rows(B, K, head_ctas):
+    """Up to 64 valid rows the GEMMs issue MMAs of 64 rows, whose accumulator rows sit in sixteen TMEM lanes of
+    each quadrant; the products are the same, so forcing 128-row MMAs must not change a bit."""
+    cfg = _small(B=B, K=K, seed=31, V=2000)
+    case = cases.make_case(cfg, oracle_ref_argmax)
+    ref = run_oracle(case)
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d)
+    v.set_tuning(head_ctas=head_ctas)
+    out = cases.run(v, d)
+    torch.cuda.synchronize()
+    assert v.device_error() == 0
+    compare(case, ref, out, cfg.tau)
+    L = v.debug_logits(d["target_hidden"])
+    v.set_tuning(head_ctas=head_ctas, lm_mma_m=128)
+    big = cases.run(v, d)
+    L128 = v.debug_logits(d["target_hidden"])
+    torch.cuda.synchronize()
+    assert v.device_error() == 0
+    assert torch.equal(L, L128)
+    for k in ("accept_len", "correction_token", "argmax", "lse", "p_draft", "head_prob", "n_mismatch", "status"):
+        assert torch.equal(getattr(big, k), getattr(out, k)), k
+    v.close()
+
+
 @pytest.mark.parametrize("tune", [dict(lm_tile_n=64), dict(lm_tile_n=256, lm_stages=2), dict(head_tile_n=64, head_stages=3)],
                          ids=lambda t: "-".join("%s%s" % kv for kv in t.items()))
 def test_results_do_not_depend_on_the_launch_plan(tune):

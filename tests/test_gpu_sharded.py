@@ -55,7 +55,9 @@ def test_gathered_round_equals_unsharded_round(kw, cuts):
     assert torch.equal(out.n_mismatch, one.n_mismatch) and torch.equal(out.mismatch_mask, one.mismatch_mask)
     assert float((out.lse - one.lse).abs().max()) < 1e-5
     assert torch.allclose(out.p_draft, one.p_draft, rtol=1e-4, atol=0)
-    assert torch.equal(out.head_prob, one.head_prob)
+    # small batches evaluate the head inside the LM-head launch in a whole round but in a launch of its own here:
+    # same products, another fp32 summation order
+    assert float((out.head_prob - one.head_prob).abs().max()) < 1e-5
     compare(case, run_oracle(case), out, cfg.tau)
     for v in shards:
         v.close()

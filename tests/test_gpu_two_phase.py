@@ -35,7 +35,11 @@ def test_localize_then_decide_equals_one_call(kw):
     loc = v.localize(d["target_hidden"], d["draft_tokens"], draft_q=d["draft_q"], uniforms=d["uniforms"], **kw_geo)
     torch.cuda.synchronize()
     assert torch.equal(loc.mismatch_mask, one.mismatch_mask) and torch.equal(loc.n_mismatch, one.n_mismatch)
-    assert torch.equal(loc.argmax, one.argmax) and torch.equal(loc.lse, one.lse) and torch.equal(loc.p_draft, one.p_draft)
+    # the one-call round of a small batch divides the vocabulary over fewer CTAs (some evaluate the decision head in
+    # the same launch): same logits, another fp32 summation order in the log-sum-exp
+    assert torch.equal(loc.argmax, one.argmax)
+    assert float((loc.lse - one.lse).abs().max()) < 1e-5
+    assert torch.allclose(loc.p_draft, one.p_draft, rtol=1e-4, atol=0)
     # greedy result while no hidden state has arrived: first candidate position
     mask = loc.mismatch_mask.cpu().numpy().astype(np.uint64)
     first = np.array([next((i for i in range(case["k_len"][b]) if (int(mask[b]) >> i) & 1), case["k_len"][b])
@@ -55,7 +59,7 @@ def test_localize_then_decide_equals_one_call(kw):
     assert torch.equal(dec.accept_len, one.accept_len) and torch.equal(dec.correction_token, one.correction_token)
     assert torch.equal(dec.n_mismatch, one.n_mismatch)
     hp_one = one.head_prob.cpu().numpy()[sel]
-    assert np.allclose(dec.head_prob.cpu().numpy(), hp_one, atol=1e-6)
+    assert np.allclose(dec.head_prob.cpu().numpy(), hp_one, atol=1e-5)      # up to the fp32 summation order
 
     # and against the oracle on the selective-hidden traffic
     sh_case = dict(case, draft_hidden=packed, sel_off=sel_off, sel_pos=sel_pos)
