@@ -804,7 +804,8 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
     tp.err_src = c->err; tp.err_copy = c->err_copy_next;
     c->err_copy_next = nullptr;
     {
-        const int rc = launch_pdl(tail_kernel, dim3(b->B), dim3(256), 0, st, tp);
+        // few requests: one warp per window row and head position, so nothing in a block runs one after the other
+        const int rc = launch_pdl(tail_kernel, dim3(b->B), dim3(b->B <= 32 ? 1024 : 256), 0, st, tp);
         if (rc != WISV_OK) return rc;
     }
     c->launches++;

@@ -55,16 +55,30 @@ struct PackParams {
 };
 
 __device__ __forceinline__ void cast_row(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, int n) {
-    // n % 8 == 0; 8 floats in, one 16-byte store out
-    for (int i = threadIdx.x * 8; i < n; i += blockDim.x * 8) {
-        const float4 a = *reinterpret_cast<const float4*>(src + i);
-        const float4 b = *reinterpret_cast<const float4*>(src + i + 4);
-        __nv_bfloat162 o[4];
-        o[0] = __floats2bfloat162_rn(a.x, a.y);
-        o[1] = __floats2bfloat162_rn(a.z, a.w);
-        o[2] = __floats2bfloat162_rn(b.x, b.y);
-        o[3] = __floats2bfloat162_rn(b.z, b.w);
-        *reinterpret_cast<uint4*>(dst + i) = *reinterpret_cast<const uint4*>(o);
+    // n % 8 == 0; 8 floats in, one 16-byte store out; the loads of four steps are issued before the first store
+    const int step = blockDim.x * 8;
+    for (int i0 = threadIdx.x * 8; i0 < n; i0 += 4 * step) {
+        float4 a[4], b[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = i0 + u * step;
+            if (i < n) {
+                a[u] = *reinterpret_cast<const float4*>(src + i);
+                b[u] = *reinterpret_cast<const float4*>(src + i + 4);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = i0 + u * step;
+            if (i < n) {
+                __nv_bfloat162 o[4];
+                o[0] = __floats2bfloat162_rn(a[u].x, a[u].y);
+                o[1] = __floats2bfloat162_rn(a[u].z, a[u].w);
+                o[2] = __floats2bfloat162_rn(b[u].x, b[u].y);
+                o[3] = __floats2bfloat162_rn(b[u].z, b[u].w);
+                *reinterpret_cast<uint4*>(dst + i) = *reinterpret_cast<const uint4*>(o);
+            }
+        }
     }
 }
 
@@ -169,7 +183,10 @@ __device__ __forceinline__ void merge_stat(RowStat& a, float mx, int idx, float 
     }
 }
 
-__global__ void __launch_bounds__(256) tail_kernel(const TailParams p)
+// Latency matters here more than throughput (at batch 1 the whole kernel is a handful of dependent global
+// loads): every warp takes one task at a time - a window row to merge or a head position to finish - and
+// issues all the loads of the task before it uses any of them; the scan warp fetches its tokens first.
+__global__ void __launch_bounds__(1024) tail_kernel(const TailParams p)
 {
     constexpr int kMaxK = 64;
     __shared__ int s_arg[kMaxK + 1];
@@ -181,9 +198,6 @@ __global__ void __launch_bounds__(256) tail_kernel(const TailParams p)
 
     const int b = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-    const int k0 = p.ix.koff(b);
-    const int Kb = min(p.ix.koff(b + 1) - k0, kMaxK);
-    const int r0 = k0 + b;
 
     if (threadIdx.x < kMaxK) { s_has[threadIdx.x] = 0; s_prob[threadIdx.x] = 0.0f; }
     if (threadIdx.x == 0) s_flag = 0;
@@ -194,80 +208,111 @@ __global__ void __launch_bounds__(256) tail_kernel(const TailParams p)
     // partials of the LM-head and decision-head kernels must be complete and visible
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
+    const int k0 = p.ix.koff(b);
+    const int Kb = min(p.ix.koff(b + 1) - k0, kMaxK);
+    const int r0 = k0 + b;
+
     if (p.err_copy && b == 0 && threadIdx.x == 0) *p.err_copy = *p.err_src;
 
-    // ---- merge the per-tile (max, argidx, sumexp) partials of each window row
+    // what the scan needs of the inputs, requested before anything else (warp 0, positions lane and lane + 32)
+    int tokv[2] = {0, 0};
+    float qv[2] = {1.0f, 1.0f}, uv[2] = {0.0f, 0.0f};
+    if (warp == 0 && p.phase != 2) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int i = lane + 32 * h;
+            if (i < Kb) {
+                if (p.stochastic) { qv[h] = p.draft_q[k0 + i]; uv[h] = p.uniforms[k0 + i]; }
+                else tokv[h] = p.draft_tokens[k0 + i];
+            }
+        }
+    }
+
     int flag = 0;
     if (p.phase == 2) {
         // second phase: the rows were reduced by the localize call
         for (int i = threadIdx.x; i <= Kb; i += blockDim.x) { s_arg[i] = p.saved_arg[r0 + i]; flag |= p.row_flag[r0 + i]; }
     }
-    for (int i = warp; i <= Kb && p.phase != 2; i += nwarps) {
-        const int r = r0 + i;
-        RowStat st{-CUDART_INF_F, 0x7fffffff, 0.0f};
-        float tl = -CUDART_INF_F;
-        if (p.phase == 3) {
-            // one partial per vocabulary shard: {max, global argidx, sumexp, draft-token logit or -inf}
-            for (int n = lane; n < p.n_tiles_lm; n += 32) {
-                const float4 v = p.lm_part[(size_t)r * p.part_rstride + (size_t)n * p.part_nstride];
-                merge_stat(st, v.x, __float_as_int(v.y), v.z);
-                tl = fmaxf(tl, v.w);
-            }
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) tl = fmaxf(tl, __shfl_xor_sync(0xffffffffu, tl, off));
-        }
-        const float4* part = p.lm_part + (size_t)r * p.n_tiles_lm;
-        // four independent loads in flight per lane before the dependent merges
-        int n = p.phase == 3 ? p.n_tiles_lm : lane;
-        for (; n + 96 < p.n_tiles_lm; n += 128) {
-            const float4 v0 = part[n], v1 = part[n + 32], v2 = part[n + 64], v3 = part[n + 96];
-            merge_stat(st, v0.x, __float_as_int(v0.y), v0.z);
-            merge_stat(st, v1.x, __float_as_int(v1.y), v1.z);
-            merge_stat(st, v2.x, __float_as_int(v2.y), v2.z);
-            merge_stat(st, v3.x, __float_as_int(v3.y), v3.z);
-        }
-        for (; n < p.n_tiles_lm; n += 32) {
-            const float4 v = part[n];
-            merge_stat(st, v.x, __float_as_int(v.y), v.z);
-        }
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            const float omx = __shfl_xor_sync(0xffffffffu, st.mx, off);
-            const int oidx = __shfl_xor_sync(0xffffffffu, st.idx, off);
-            const float osum = __shfl_xor_sync(0xffffffffu, st.sum, off);
-            merge_stat(st, omx, oidx, osum);
-        }
-        const float l = st.mx + logf(st.sum);
-        if (p.phase != 3) st.idx += p.vocab_base;
-        if (lane == 0) {
-            s_arg[i] = st.idx;
-            s_lse[i] = l;
-            s_tl[i] = p.phase == 3 ? tl : p.tok_logit[r];
-            if (p.phase == 1) p.saved_arg[r] = st.idx;
-            if (p.argmax) p.argmax[r] = st.idx;
-            if (p.lse) p.lse[r] = l;
-            if (!isfinite(l)) flag |= 4;
-            flag |= p.row_flag[r];
-        }
-    }
-
-    // ---- finish the decision head: s = b2 + sum of per-tile partial dot products
+    const int row_tasks = p.phase == 2 ? 0 : Kb + 1;
     int e0, e1;
     if (p.phase == 1) { e0 = 0; e1 = 0; }
     else if (p.mode_sh) { e0 = max(p.sel_off[b], 0); e1 = min(p.sel_off[b + 1], p.P); } else { e0 = k0; e1 = k0 + Kb; }
-    for (int e = e0 + warp; e < e1; e += nwarps) {
-        float s = 0.0f;
-        const float* hp = p.head_part + (size_t)e * p.n_tiles_head;
-        for (int n = lane; n < p.n_tiles_head; n += 32) s += hp[n];
+    const int pos_tasks = e1 > e0 ? e1 - e0 : 0;
+
+    for (int task = warp; task < row_tasks + pos_tasks; task += nwarps) {
+        if (task < row_tasks) {
+            // ---- merge the (max, argidx, sumexp) partials of one window row: one per vocabulary tile or CTA,
+            //      or per shard {max, global argidx, sumexp, draft-token logit or -inf} in the gathered flow
+            const int i = task;
+            const int r = r0 + i;
+            float tlg = 0.0f;
+            int rf = 0;
+            if (lane == 0) {
+                rf = p.row_flag[r];
+                if (p.phase != 3) tlg = p.tok_logit[r];
+            }
+            RowStat st{-CUDART_INF_F, 0x7fffffff, 0.0f};
+            float tl = -CUDART_INF_F;
+            const float4* part = p.lm_part + (size_t)r * p.part_rstride;
+            for (int base = 0; base < p.n_tiles_lm; base += 256) {
+                float4 v[8];
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
-        s += p.b2;
-        const float prob = 1.0f / (1.0f + expf(-s));
-        if (lane == 0) {
-            if (p.head_prob) p.head_prob[e] = prob;
-            const int i = p.pos_i[e];
-            if (i >= 0 && i < Kb) { s_prob[i] = prob; s_has[i] = 1; } else { flag |= 8; }
-            if (!isfinite(s)) flag |= 4;
+                for (int j = 0; j < 8; ++j) {
+                    const int n = base + j * 32 + lane;
+                    v[j] = n < p.n_tiles_lm ? part[(size_t)n * p.part_nstride]
+                                            : make_float4(-CUDART_INF_F, 0.0f, 0.0f, -CUDART_INF_F);
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    merge_stat(st, v[j].x, __float_as_int(v[j].y), v[j].z);
+                    tl = fmaxf(tl, v[j].w);
+                }
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                const float omx = __shfl_xor_sync(0xffffffffu, st.mx, off);
+                const int oidx = __shfl_xor_sync(0xffffffffu, st.idx, off);
+                const float osum = __shfl_xor_sync(0xffffffffu, st.sum, off);
+                merge_stat(st, omx, oidx, osum);
+                tl = fmaxf(tl, __shfl_xor_sync(0xffffffffu, tl, off));
+            }
+            const float l = st.mx + logf(st.sum);
+            if (p.phase != 3) st.idx += p.vocab_base;
+            if (lane == 0) {
+                s_arg[i] = st.idx;
+                s_lse[i] = l;
+                s_tl[i] = p.phase == 3 ? tl : tlg;
+                if (p.phase == 1) p.saved_arg[r] = st.idx;
+                if (p.argmax) p.argmax[r] = st.idx;
+                if (p.lse) p.lse[r] = l;
+                if (!isfinite(l)) flag |= 4;
+                flag |= rf;
+            }
+        } else {
+            // ---- finish the decision head of one position: s = b2 + sum of the partial dot products
+            const int e = e0 + (task - row_tasks);
+            int pi = 0;
+            if (lane == 0) pi = p.pos_i[e];
+            float s = 0.0f;
+            const float* hp = p.head_part + (size_t)e * p.n_tiles_head;
+            for (int base = 0; base < p.n_tiles_head; base += 128) {
+                float x[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int n = base + j * 32 + lane;
+                    x[j] = n < p.n_tiles_head ? hp[n] : 0.0f;
+                }
+                s += (x[0] + x[1]) + (x[2] + x[3]);
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+            s += p.b2;
+            const float prob = 1.0f / (1.0f + expf(-s));
+            if (lane == 0) {
+                if (p.head_prob) p.head_prob[e] = prob;
+                if (pi >= 0 && pi < Kb) { s_prob[pi] = prob; s_has[pi] = 1; } else { flag |= 8; }
+                if (!isfinite(s)) flag |= 4;
+            }
         }
     }
     if (flag) atomicOr(&s_flag, flag);
@@ -289,10 +334,10 @@ __global__ void __launch_bounds__(256) tail_kernel(const TailParams p)
                     const float pd = expf(s_tl[i] - s_lse[i]);
                     if (p.p_draft) p.p_draft[t] = pd;
                     if (p.stochastic) {
-                        const float alpha = fminf(1.0f, pd / p.draft_q[t]);
-                        cand = !(p.uniforms[t] < alpha);
+                        const float alpha = fminf(1.0f, pd / qv[h]);
+                        cand = !(uv[h] < alpha);
                     } else {
-                        cand = p.draft_tokens[t] != s_arg[i];
+                        cand = tokv[h] != s_arg[i];
                     }
                 }
                 const bool has = s_has[i] != 0;
