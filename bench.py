@@ -43,10 +43,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 SINGLE_CTA_SOURCES = ("wisv_gemm.cuh", "wisv_ptx.cuh")
 CTA_PAIR_SOURCES = ("wisv_gemm2.cuh", "wisv_gemm.cuh", "wisv_ptx.cuh")
 NCU_TRAFFIC = {
-    # single-CTA kernel, 9 window rows: 1.0513 GB read + 4.2 MB written per launch
-    "8b_b1": {"bytes": 1055500000, "files": SINGLE_CTA_SOURCES, "kernel_hash": "ee178e4ce3d4c82a"},
-    # single-CTA kernel, 576 window rows: 1.0584 GB read + 8.0 MB written per launch
-    "8b_b64": {"bytes": 1066430000, "files": SINGLE_CTA_SOURCES, "kernel_hash": "ee178e4ce3d4c82a"},
+    # LM-head and decision-head CTAs in one launch, 9 window rows: 1.0642 GB read + 4.4 MB written per launch
+    "8b_b1": {"bytes": 1068600000, "files": SINGLE_CTA_SOURCES, "kernel_hash": "246e580b4bdc4e06"},
+    # single-CTA kernel, 576 window rows: 1.0589 GB read + 8.4 MB written per launch
+    "8b_b64": {"bytes": 1067400000, "files": SINGLE_CTA_SOURCES, "kernel_hash": "246e580b4bdc4e06"},
     # CTA-pair kernel, 8704 window rows: 6.013 GB read + 102.7 MB written per launch (4.6-6.0 GB between captures)
     "8b_b512": {"bytes": 6115700000, "files": CTA_PAIR_SOURCES, "kernel_hash": "4873c99cd8dddf90"},
 }
