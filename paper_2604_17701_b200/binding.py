@@ -170,6 +170,25 @@ class VerifyOutput:
     status: "object" = None
 
 
+class BoundHostCall:
+    """One wisv_verify_host call with its arguments already marshalled (see Verifier.bind_host)."""
+
+    def __init__(self, verifier, batch, result, out, stream, keep):
+        self._v, self._b, self._r, self.out, self._keep = verifier, batch, result, out, keep
+        self._fn = verifier.lib.wisv_verify_host
+        self._args = (verifier._h, C.byref(batch), C.byref(result), C.c_void_p(stream.cuda_stream))
+        self._dev = verifier.device.index if verifier.device.index is not None else 0
+        self._current_device = verifier._torch.cuda.current_device
+
+    def __call__(self) -> "VerifyOutput":
+        if self._current_device() != self._dev:
+            with self._v._torch.cuda.device(self._dev):
+                _check(self._fn(*self._args), "wisv_verify_host")
+        else:
+            _check(self._fn(*self._args), "wisv_verify_host")
+        return self.out
+
+
 class Verifier:
     """wisv_create / wisv_verify / wisv_destroy on torch CUDA tensors.
 
@@ -362,6 +381,27 @@ class Verifier:
             _check(self.lib.wisv_verify_host(self._h, C.byref(b), C.byref(r), C.c_void_p(st.cuda_stream)),
                    "wisv_verify_host")
         return out
+
+    def bind_host(self, target_hidden, draft_tokens, draft_hidden, csi, *, B: int, K: int = 0, k_off=None,
+                  T: Optional[int] = None, sel_off=None, sel_pos=None, draft_q=None, uniforms=None,
+                  tau: Optional[float] = None, extras: bool = False, out: Optional[VerifyOutput] = None,
+                  stream=None) -> "BoundHostCall":
+        """wisv_verify_host with the argument blocks built once, for a loop that reuses the same host buffers
+        (a server refills its pinned input buffers in place and calls again): each call of the returned object
+        is one wisv_verify_host on the buffers as they are then, and returns the same VerifyOutput."""
+        torch = self._torch
+        if T is None:
+            T = B * K if k_off is None else int(draft_tokens.shape[0])
+        R = T + B
+        P = int(sel_pos.shape[0]) if sel_pos is not None else T
+        if out is None:
+            out = self._outputs(B, R, T, P, "cpu", extras, pin=True)
+        b = self._batch(B=B, K=K, k_off=k_off, T=T, target_hidden=target_hidden, draft_tokens=draft_tokens,
+                        draft_hidden=draft_hidden, csi=csi, sel_off=sel_off, sel_pos=sel_pos, draft_q=draft_q,
+                        uniforms=uniforms, tau=tau)
+        st = stream if stream is not None else torch.cuda.current_stream(self.device)
+        keep = (target_hidden, draft_tokens, draft_hidden, csi, k_off, sel_off, sel_pos, draft_q, uniforms, st)
+        return BoundHostCall(self, b, self._result(out), out, st, keep)
 
     def debug_logits(self, target_hidden):
         torch = self._torch

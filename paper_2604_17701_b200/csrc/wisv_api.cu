@@ -84,6 +84,9 @@ struct wisv_ctx {
     int32_t* pos_req = nullptr; int32_t* pos_i = nullptr;
     int32_t* err = nullptr;
     int32_t* err_copy_next = nullptr;           // where the next round's tail kernel mirrors the error word
+    volatile int32_t* done_flag_next = nullptr; // where it announces that the results are written (host-buffer calls)
+    int32_t done_seq = 0;                       // value it announces with
+    int32_t* done_count = nullptr;              // blocks of that kernel that have finished
     int32_t* saved_arg = nullptr;               // [rows_alloc] argmax per row, localize -> decide
     unsigned long long* saved_mask = nullptr;   // [max_requests] candidate sets, localize -> decide
     bool loc_valid = false;                     // a localize call is waiting for its decide
@@ -293,7 +296,7 @@ void free_ctx(wisv_ctx* c)
     cudaFree(c->X); cudaFree(c->Z); cudaFree(c->W1p); cudaFree(c->W1c); cudaFree(c->lm_part);
     cudaFree(c->head_part); cudaFree(c->row_tok); cudaFree(c->row_flag); cudaFree(c->tok_logit);
     cudaFree(c->pos_req); cudaFree(c->pos_i); cudaFree(c->err); cudaFree(c->splitk_buf); cudaFree(c->splitk_count);
-    cudaFree(c->saved_arg); cudaFree(c->saved_mask);
+    cudaFree(c->saved_arg); cudaFree(c->saved_mask); cudaFree(c->done_count);
     if (c->prof_ev) {
         for (int i = 0; i < c->prof_n * (kStages + 1); ++i) cudaEventDestroy(c->prof_ev[i]);
         free(c->prof_ev);
@@ -567,6 +570,8 @@ int wisv_create(const wisv_config* cfg, const wisv_weights* w, wisv_ctx** out)
         if ((rc = dev_alloc(&c->pos_req, (size_t)c->pos_alloc))) break;
         if ((rc = dev_alloc(&c->pos_i, (size_t)c->pos_alloc))) break;
         if ((rc = dev_alloc(&c->err, 1))) break;
+        if ((rc = dev_alloc(&c->done_count, 1))) break;
+        if (cudaMemset(c->done_count, 0, sizeof(int32_t)) != cudaSuccess) { rc = WISV_ECUDA; break; }
         if ((rc = dev_alloc(&c->saved_arg, (size_t)c->rows_alloc))) break;
         if ((rc = dev_alloc(&c->saved_mask, (size_t)cfg->max_requests))) break;
         c->splitk_tiles = (cfg->d_J + 15) / 16;
@@ -803,6 +808,8 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
     tp.status = r->status;
     tp.err_src = c->err; tp.err_copy = c->err_copy_next;
     c->err_copy_next = nullptr;
+    tp.done_flag = c->done_flag_next; tp.done_count = c->done_count; tp.done_seq = c->done_seq;
+    c->done_flag_next = nullptr;
     {
         // few requests: one warp per window row and head position, so nothing in a block runs one after the other
         const int rc = launch_pdl(tail_kernel, dim3(b->B), dim3(b->B <= 32 ? 1024 : 256), 0, st, tp);
@@ -1027,10 +1034,26 @@ int wisv_verify_host(wisv_ctx* c, const wisv_batch* hb, const wisv_result* hr, v
         WISV_CUDA(cudaMemcpyAsync(h.draft_hidden, hb->draft_hidden, dh_bytes, cudaMemcpyHostToDevice, st));
     memset(pin_out, 0, 4);
     c->err_copy_next = reinterpret_cast<int32_t*>(h.pin_dev + h.in_cap);
+    // The merge/scan kernel stores a fresh sequence number next to the results when all of them are written;
+    // watching that word costs less than a stream synchronisation at the end of a round of a few hundred
+    // microseconds.  The stream is polled now and then as well, so a failed launch or kernel ends the wait.
+    volatile int32_t* host_flag = reinterpret_cast<volatile int32_t*>(pin_out + 4);
+    c->done_seq = c->done_seq == 0x7fffffff ? 1 : c->done_seq + 1;
+    *host_flag = 0;
+    c->done_flag_next = reinterpret_cast<volatile int32_t*>(h.pin_dev + h.in_cap + 4);
     const int rc = wisv_verify(c, &db, &dr, cuda_stream);
     c->err_copy_next = nullptr;
+    c->done_flag_next = nullptr;
     if (rc != WISV_OK) return rc;
-    WISV_CUDA(cudaStreamSynchronize(st));
+    for (unsigned spins = 1; *host_flag != c->done_seq; ++spins) {
+        if ((spins & 0x3FFu) == 0) {
+            const cudaError_t q = cudaStreamQuery(st);
+            if (q == cudaErrorNotReady) continue;
+            if (q != cudaSuccess) { (void)cudaGetLastError(); return WISV_ECUDA; }
+            break;                               // stream idle: everything has been written
+        }
+    }
+    __atomic_thread_fence(__ATOMIC_ACQUIRE);
     int32_t dev_err = 0;
     memcpy(&dev_err, pin_out, sizeof dev_err);
     if (dev_err != 0) { (void)cudaMemset(c->err, 0, sizeof dev_err); return WISV_EDEVICE; }

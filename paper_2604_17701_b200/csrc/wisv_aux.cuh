@@ -168,6 +168,12 @@ struct TailParams {
     unsigned long long* mismatch_mask; int32_t* n_mismatch; int32_t* status;
     const int32_t* err_src;       // device error word of the earlier kernels of this round
     int32_t* err_copy;            // if set, receives *err_src (lets a host caller read it with the results)
+    // Host-buffer calls only: once every block has written its results (to device-mapped host memory) the last
+    // block to finish stores done_seq to *done_flag, so the host can watch for it instead of synchronising
+    // the stream.  done_count is a device counter that the last block leaves at zero.
+    volatile int32_t* done_flag;
+    int32_t* done_count;
+    int32_t done_seq;
 };
 
 struct RowStat { float mx; int idx; float sum; };
@@ -358,6 +364,18 @@ __global__ void __launch_bounds__(1024) tail_kernel(const TailParams p)
             if (p.mismatch_mask) p.mismatch_mask[b] = cnd;
             if (p.n_mismatch) p.n_mismatch[b] = __popcll(cnd);
             if (p.status) p.status[b] = s_flag | (missing ? 1 : 0);
+        }
+    }
+    if (p.done_flag) {
+        __threadfence_system();                  // this thread's results before the flag, as the host sees them
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const int old = atomicAdd(p.done_count, 1);
+            if (old == static_cast<int>(gridDim.x) - 1) {
+                *p.done_count = 0;
+                __threadfence_system();
+                *p.done_flag = p.done_seq;
+            }
         }
     }
 }

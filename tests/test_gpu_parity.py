@@ -345,6 +345,30 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     v.close()
 
 
+def test_bound_host_call_sees_buffers_refilled_in_place():
+    """Serving loop: pinned buffers bound once, refilled in place, one wisv_verify_host per step; each step must
+    equal a device-entry-point round on that step's data (also exercises the completion word, step after step)."""
+    cfgs = [_small(B=6, K=5, seed=s, weight_seed=50) for s in (51, 52, 53)]       # one model, three batches
+    built = [cases.make_case(c, oracle_ref_argmax, weights=_shared_weights(c)) for c in cfgs]
+    d0 = cases.to_device(built[0], DEV)
+    v = cases.make_verifier(d0)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    bufs = {k: pin(built[0][k]) for k in ("target_hidden", "draft_tokens", "draft_hidden", "csi")}
+    call = v.bind_host(bufs["target_hidden"], bufs["draft_tokens"], bufs["draft_hidden"], bufs["csi"],
+                       B=cfgs[0].B, K=cfgs[0].K, extras=True)
+    for case in built * 2:
+        for k, t in bufs.items():
+            t.copy_(torch.from_numpy(np.ascontiguousarray(case[k])))
+        ho = call()
+        ref = cases.run(v, cases.to_device(case, DEV))
+        torch.cuda.synchronize()
+        for k in ("accept_len", "correction_token", "argmax", "lse", "p_draft", "head_prob", "n_mismatch", "status"):
+            assert torch.equal(getattr(ho, k), getattr(ref, k).cpu()), k
+        compare(case, run_oracle(case), ho, cfgs[0].tau)
+    assert v.device_error() == 0
+    v.close()
+
+
 @pytest.mark.parametrize("pinned", [True, False])
 def test_host_buffer_entry_point_ragged_selective_stochastic(pinned):
     """Every optional input (row offsets, selective positions, q and u of Eq. 1) through the packed host block; the
