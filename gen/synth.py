@@ -62,6 +62,9 @@ CONFIGS: Dict[str, VerifyConfig] = {
     "tiny": VerifyConfig("tiny", B=8, K=4, H=256, H_d=128, d_c=2, d_J=128, V=4096,
                          match_rate=0.5, seed=0),
     "8b_b1": VerifyConfig("8b_b1", B=1, K=8, match_rate=0.7, seed=1, **_8B),
+    # between the two: 144 and 288 window rows (two and three row tiles of 128)
+    "8b_b16": VerifyConfig("8b_b16", B=16, K=8, match_rate=0.7, seed=8, **_8B),
+    "8b_b32": VerifyConfig("8b_b32", B=32, K=8, match_rate=0.7, seed=9, **_8B),
     "8b_b64": VerifyConfig("8b_b64", B=64, K=8, match_rate=0.7, seed=3, **_8B),
     "8b_b64_m30": VerifyConfig("8b_b64_m30", B=64, K=8, match_rate=0.30, seed=2, **_8B),
     "8b_b64_m95": VerifyConfig("8b_b64_m95", B=64, K=8, match_rate=0.95, seed=4, **_8B),
