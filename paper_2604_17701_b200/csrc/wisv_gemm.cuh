@@ -64,7 +64,7 @@ struct GemmParams {
                          // each item stores its raw fp32 tile, the last one to finish adds them up in
                          // split order and applies the epilogue (no CTA ever waits for another)
     int32_t kb_per_split;
-    float* splitk_buf;        // [items][128][tile_n] raw partial pre-activations
+    float* splitk_buf;        // [items][tile_n][128] raw partial pre-activations, column-major per item
     int32_t* splitk_count;    // [m_tiles * n_tiles], zero between calls (the last item resets it)
     int32_t* err;        // device error word (bit 0: a bounded wait gave up)
     // LM-head epilogue
@@ -160,7 +160,6 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + ring_bytes + 8 * (2 * kMaxStages + 5));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [0] abort, [1] drain scratch
     volatile int* last_flag = abort_flag + 2;                                    // split-K: this CTA finishes the tile
-    float* split_red = reinterpret_cast<float*>(smem + ring_bytes + 1024);     // [128][<= 8] split-K row sums
     float* epi_const = reinterpret_cast<float*>(smem + ring_bytes + 1024 + 4096);
 
     const int warp = threadIdx.x >> 5;
@@ -392,13 +391,12 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
                 if (EPI == EPI_LMHEAD) {
                     lm_update_chunk(v, col0, p.n_total, tok, mx, arg, sum, p.tok_logit + row);
                 } else if (EPI == EPI_HEAD && p.k_splits > 1) {
-                    // split K: park the raw partial tile; the last item of this (m, n) tile finishes it
-                    float4* dst = reinterpret_cast<float4*>(
-                        p.splitk_buf + ((size_t)t * kTileM + rit) * p.tile_n + c0);
+                    // split K: park the raw partial tile, column-major ([tile_n][128]: consecutive lanes hold
+                    // consecutive rows, so these stores and the finisher's loads are coalesced); the last item of
+                    // this (m, n) tile finishes it
+                    float* dst = p.splitk_buf + ((size_t)t * p.tile_n + c0) * kTileM + rit;
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
-                                             __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                    for (int j = 0; j < 16; ++j) dst[(size_t)j * kTileM] = __uint_as_float(v[j]);
                 } else if (EPI == EPI_HEAD) {
                     float pre[16];
 #pragma unroll
@@ -434,42 +432,47 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 const bool finisher = *last_flag != 0;
                 if (finisher) {
-                    // The whole epilogue group adds up the split tiles: a warp takes 32 columns of one
-                    // row at a time (coalesced reads, all split loads in flight together), applies the
-                    // head epilogue per column and reduces over the 32 columns with shuffles; the
-                    // per-(row, chunk) sums are then added in chunk order, so the result is deterministic.
+                    // Every epilogue thread finishes one row of the tile: per 16 columns it fetches the partial
+                    // sums of all splits (all loads in flight together), adds them in split order and then runs
+                    // the same 16-wide epilogue as the unsplit path, so the long dependent chain of the exact
+                    // GELU is overlapped sixteen-fold.  (A first version gave a warp 32 columns of one row at a
+                    // time and reduced with shuffles: one GELU chain per lane at a time, 60 us for a full tile.)
                     __threadfence();
-                    const int chunks = (p.tile_n + 31) / 32;
                     const int rows_here = min(kTileM, p.rows - m * kTileM);
-                    const int ew = et >> 5;
-                    for (int pair = ew; pair < rows_here * chunks; pair += kEpiThreads / 32) {
-                        const int r = pair / chunks, ch = pair - r * chunks;
-                        const int col = ch * 32 + lane;
-                        float val = 0.0f;
-                        if (col < p.tile_n) {
-                            float x[kMaxKSplits];
-#pragma unroll
-                            for (int ks = 0; ks < kMaxKSplits; ++ks) {
-                                const int it = (n * p.k_splits + ks) * p.m_tiles + m;
-                                x[ks] = ks < p.k_splits
-                                            ? __ldcg(p.splitk_buf + ((size_t)it * kTileM + r) * p.tile_n + col) : 0.0f;
-                            }
-                            float pre = 0.0f;
-#pragma unroll
-                            for (int ks = 0; ks < kMaxKSplits; ++ks) pre += x[ks];      // split order
-                            pre += cb1[col];
-                            for (int c = 0; c < p.d_c; ++c) pre = fmaf(ccs[c * kEpiThreads + r], cwc[c * p.tile_n + col], pre);
-                            val = cw2[col] * act_apply(pre, p.act);
-                        }
-#pragma unroll
-                        for (int off = 16; off > 0; off >>= 1) val += __shfl_xor_sync(0xffffffffu, val, off);
-                        if (lane == 0) split_red[r * chunks + ch] = val;
-                    }
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
-                    if (et < rows_here) {
+                    const int r = et;
+                    if (r < rows_here) {
                         float tot = 0.0f;
-                        for (int ch = 0; ch < chunks; ++ch) tot += split_red[et * chunks + ch];
-                        p.head_part[(size_t)(m * kTileM + et) * p.part_stride + n] = tot;
+                        for (int c0 = 0; c0 < p.tile_n; c0 += 16) {
+                            float pre[16];
+#pragma unroll
+                            for (int jj = 0; jj < 16; ++jj) pre[jj] = 0.0f;
+                            for (int ks0 = 0; ks0 < p.k_splits; ks0 += 4) {             // four splits' loads at a time
+                                float x[4][16];
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) {
+                                    const int ks = ks0 + u;
+                                    const int it = (n * p.k_splits + ks) * p.m_tiles + m;
+                                    const float* src = p.splitk_buf + ((size_t)it * p.tile_n + c0) * kTileM + r;
+#pragma unroll
+                                    for (int jj = 0; jj < 16; ++jj)
+                                        x[u][jj] = ks < p.k_splits ? __ldcg(src + (size_t)jj * kTileM) : 0.0f;
+                                }
+#pragma unroll
+                                for (int u = 0; u < 4; ++u)                              // split order
+#pragma unroll
+                                    for (int jj = 0; jj < 16; ++jj) pre[jj] += x[u][jj];
+                            }
+#pragma unroll
+                            for (int jj = 0; jj < 16; ++jj) pre[jj] += cb1[c0 + jj];
+                            for (int c = 0; c < p.d_c; ++c) {
+                                const float xc = ccs[c * kEpiThreads + r];
+#pragma unroll
+                                for (int jj = 0; jj < 16; ++jj) pre[jj] = fmaf(xc, cwc[c * p.tile_n + c0 + jj], pre[jj]);
+                            }
+#pragma unroll
+                            for (int jj = 0; jj < 16; ++jj) tot = fmaf(cw2[c0 + jj], act_apply(pre[jj], p.act), tot);
+                        }
+                        p.head_part[(size_t)(m * kTileM + r) * p.part_stride + n] = tot;
                     }
                 }
             } else if (valid && !p.carry) {
