@@ -178,7 +178,7 @@ double wave_eff(long long tiles, int sms)
 // LM head: with a single row tile the kernel streams the weights once and is
 // HBM-bound, so the tile height over the vocabulary is chosen to fill the last
 // wave of CTAs; with many row tiles it is tensor-bound and takes the largest tile.
-Plan plan_lm(const wisv_ctx* c, int R, bool single_only = false, int sms = 0)
+Plan plan_lm(const wisv_ctx* c, int R, bool single_only = false, int sms = 0, int reserved_pairs = 0)
 {
     Plan p{};
     if (sms <= 0) sms = c->sm_count;
@@ -202,8 +202,28 @@ Plan plan_lm(const wisv_ctx* c, int R, bool single_only = false, int sms = 0)
         if (c->tune.lm_stages >= 2 && c->tune.lm_stages < s) s = c->tune.lm_stages;
         p.stages = s;
         p.smem = pair_fixed_bytes() + (size_t)s * kPairStageBytes;
+        int pairs_free = c->max_pairs - reserved_pairs;
+        if (pairs_free < 1) pairs_free = 1;
+        if (p.m_tiles == 1) {
+            // One row tile of 256 (HBM-bound): like the single-CTA kernel with one row tile, every pair gets one
+            // contiguous range of the vocabulary, here in units of 32 rows (each CTA of a pair loads half a tile,
+            // a multiple of 16 rows), cut into tiles of nearly equal height; one partial per (row, pair).
+            const int units = (V + 31) / 32;
+            const int pairs = units < pairs_free ? units : pairs_free;
+            p.units_base = units / pairs;
+            p.units_rem = units % pairs;
+            const int umax = p.units_base + (p.units_rem ? 1 : 0);
+            const int cap = kPairTileN / 32;
+            p.tiles_per_cta = (umax + cap - 1) / cap;
+            p.tile_n = (umax + p.tiles_per_cta - 1) / p.tiles_per_cta * 32;
+            p.n_tiles = pairs * p.tiles_per_cta;
+            p.ctas = 2 * pairs;
+            p.carry = 1;
+            p.parts = pairs;
+            return p;
+        }
         const long long tiles = (long long)p.m_tiles * p.n_tiles;
-        p.ctas = 2 * (int)(tiles < c->max_pairs ? tiles : c->max_pairs);
+        p.ctas = 2 * (int)(tiles < pairs_free ? tiles : pairs_free);
         p.carry = 0;
         p.parts = p.n_tiles;
         return p;
@@ -267,24 +287,33 @@ Plan plan_head(const wisv_ctx* c, int P)
 // The decision head gets a few CTAs of its own - enough to finish well inside the time the LM head needs
 // to stream its weights - and the LM head is planned for the SMs that remain.
 constexpr int kFusedHeadCtas = 6;
+constexpr int kFusedHeadCtasTwoTiles = 8;     // head positions in two row tiles (129..255)
 bool plan_fused(const wisv_ctx* c, int R, int P, Plan* lm, Plan* hd)
 {
-    if (c->tune.head_ctas < 0 || R < 1 || P < 1 || R > kTileM || P > kTileM) return false;
-    int want = c->tune.head_ctas > 0 ? c->tune.head_ctas : kFusedHeadCtas;
+    if (c->tune.head_ctas < 0 || R < 1 || P < 1) return false;
+    const bool small = R <= kTileM && P <= kTileM;
+    // up to 256 window rows: the LM head runs on CTA pairs (one row tile of 256, still bound by HBM) and the
+    // decision head on a few clusters of the same launch
+    const bool with_pairs = !small && R <= kPairTileM && P <= kPairTileM && c->max_pairs > 2 &&
+                            !c->tune.lm_single_cta && !c->tune.lm_tile_n;
+    if (!small && !with_pairs) return false;
+    const int head_m_tiles = (P + kTileM - 1) / kTileM;
+    int want = c->tune.head_ctas > 0 ? c->tune.head_ctas : (head_m_tiles > 1 ? kFusedHeadCtasTwoTiles : kFusedHeadCtas);
     if (want > c->sm_count / 2) want = c->sm_count / 2;
     if (want < 1) return false;
     Plan h{};
     const int N = c->cfg.d_J;
-    int tn = kSplitTileN;
+    int tn = head_m_tiles > 1 ? 128 : kSplitTileN;
     if (c->tune.head_tile_n >= 16 && c->tune.head_tile_n <= kMaxTileN && c->tune.head_tile_n % 16 == 0) tn = c->tune.head_tile_n;
     if (tn > round_up(N, 16)) tn = round_up(N, 16);
-    h.m_tiles = 1; h.tile_n = tn; h.n_tiles = (N + tn - 1) / tn;
-    h.a_rows = round_up(P, 8);
+    h.m_tiles = head_m_tiles; h.tile_n = tn; h.n_tiles = (N + tn - 1) / tn;
+    h.a_rows = head_m_tiles > 1 ? kTileM : round_up(P, 8);
     h.k_splits = 1;
     h.kb_per_split = (c->cfg.H_d + c->cfg.H + kBlockK - 1) / kBlockK;
     finish_plan(c, &h, c->cfg.d_c, h.kb_per_split, c->tune.head_stages, want, N);
     *hd = h;
-    *lm = plan_lm(c, R, true, c->sm_count - h.ctas);
+    if (small) *lm = plan_lm(c, R, true, c->sm_count - h.ctas);
+    else *lm = plan_lm(c, R, false, 0, (h.ctas + 1) / 2);
     return true;
 }
 
@@ -421,6 +450,31 @@ int launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cud
 // tile height of a balanced plan; never used when tile_n is 16)
 inline int map_hi(const Plan& pl) { return pl.tile_n / 16 - 1; }
 inline int map_lo(const Plan& pl) { return pl.tile_n / 16 - 2 > 0 ? pl.tile_n / 16 - 2 : 0; }
+
+// tensor maps of the pair kernel's weight tiles: each CTA of a pair loads half of a tile's rows
+inline int pair_map_hi(const Plan& pl) { return pl.tile_n / 32 - 1; }
+inline int pair_map_lo(const Plan& pl) { return pl.tile_n / 32 - 2 > 0 ? pl.tile_n / 32 - 2 : 0; }
+
+PairParams pair_params(const wisv_ctx* c, const Plan& pl, int R)
+{
+    const wisv_config& cf = c->cfg;
+    PairParams qp;
+    memset(&qp, 0, sizeof qp);
+    qp.rows = R; qp.n_total = cf.V; qp.k_blocks = (cf.H + kBlockK - 1) / kBlockK; qp.mp_tiles = pl.m_tiles;
+    {
+        // raster groups: keep a group's bf16 rows (256 x H x 2 bytes per row tile) within 32 MB of L2
+        const long long tile_bytes = (long long)kPairTileM * cf.H * 2;
+        int mg_max = (int)((32ll << 20) / tile_bytes);
+        if (mg_max < 1) mg_max = 1;
+        const int groups = (pl.m_tiles + mg_max - 1) / mg_max;
+        qp.m_group = (pl.m_tiles + groups - 1) / groups;
+    }
+    qp.n_tiles = pl.n_tiles; qp.stages = pl.stages; qp.part_stride = pl.parts; qp.err = c->err;
+    qp.carry = pl.carry; qp.units_base = pl.units_base; qp.units_rem = pl.units_rem;
+    qp.tiles_per_pair = pl.tiles_per_cta > 0 ? pl.tiles_per_cta : 1; qp.tile_n = pl.tile_n;
+    qp.lm_part = c->lm_part; qp.row_tok = c->row_tok; qp.tok_logit = c->tok_logit;
+    return qp;
+}
 
 template <int EPI>
 int launch_gemm(wisv_ctx* c, const CUtensorMap& tA, const CUtensorMap* tB, const GemmParams& gp, const Plan& pl,
@@ -734,27 +788,28 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
         gh.head_part = c->head_part; gh.b1 = c->w.b1; gh.w2 = c->w.w2; gh.w1c = c->W1c; gh.csi = b->csi;
         gh.pos_req = c->pos_req; gh.d_c = cf.d_c; gh.act = cf.act;
         const size_t smem = pl.smem > ph.smem ? pl.smem : ph.smem;
-        const int rc = launch_pdl(round_small_kernel, dim3(pl.ctas + ph.ctas), dim3(kGemmThreads), smem, st,
-                                  c->tmX[pl.a_rows / 8 - 1], c->tmW[map_hi(pl)], c->tmW[map_lo(pl)],
-                                  c->tmZ[ph.a_rows / 8 - 1], c->tmW1[map_hi(ph)], c->tmW1[map_lo(ph)], gl, gh, pl.ctas);
-        if (rc != WISV_OK) return rc;
+        if (pl.pair) {
+            const PairParams qp = pair_params(c, pl, R);
+            const int rc = launch_pdl(lmhead_pair_kernel, dim3(pl.ctas + round_up(ph.ctas, 2)), dim3(kGemmThreads), smem,
+                                      st, c->tmX[kNumRowVariants - 1], c->tmW[pair_map_hi(pl)], c->tmW[pair_map_lo(pl)],
+                                      qp, c->tmZ[ph.a_rows / 8 - 1], c->tmW1[map_hi(ph)], c->tmW1[map_lo(ph)], gh,
+                                      pl.ctas, ph.ctas);
+            if (rc != WISV_OK) return rc;
+        } else {
+            const int rc = launch_pdl(round_small_kernel, dim3(pl.ctas + ph.ctas), dim3(kGemmThreads), smem, st,
+                                      c->tmX[pl.a_rows / 8 - 1], c->tmW[map_hi(pl)], c->tmW[map_lo(pl)],
+                                      c->tmZ[ph.a_rows / 8 - 1], c->tmW1[map_hi(ph)], c->tmW1[map_lo(ph)], gl, gh,
+                                      pl.ctas);
+            if (rc != WISV_OK) return rc;
+        }
         c->launches++;
     } else if (!rows_done && pl.pair) {
-        PairParams qp;
-        memset(&qp, 0, sizeof qp);
-        qp.rows = R; qp.n_total = cf.V; qp.k_blocks = (cf.H + kBlockK - 1) / kBlockK; qp.mp_tiles = pl.m_tiles;
-        {
-            // raster groups: keep a group's bf16 rows (256 x H x 2 bytes per row tile) within 32 MB of L2
-            const long long tile_bytes = (long long)kPairTileM * cf.H * 2;
-            int mg_max = (int)((32ll << 20) / tile_bytes);
-            if (mg_max < 1) mg_max = 1;
-            const int groups = (pl.m_tiles + mg_max - 1) / mg_max;
-            qp.m_group = (pl.m_tiles + groups - 1) / groups;
-        }
-        qp.n_tiles = pl.n_tiles; qp.stages = pl.stages; qp.part_stride = pl.parts; qp.err = c->err;
-        qp.lm_part = c->lm_part; qp.row_tok = c->row_tok; qp.tok_logit = c->tok_logit;
+        const PairParams qp = pair_params(c, pl, R);
+        GemmParams none;
+        memset(&none, 0, sizeof none);
         const int rc = launch_pdl(lmhead_pair_kernel, dim3(pl.ctas), dim3(kGemmThreads), pl.smem, st,
-                                  c->tmX[kNumRowVariants - 1], c->tmW[kTileM / 16 - 1], qp);
+                                  c->tmX[kNumRowVariants - 1], c->tmW[pair_map_hi(pl)], c->tmW[pair_map_lo(pl)], qp,
+                                  c->tmZ[0], c->tmW1[0], c->tmW1[0], none, pl.ctas, 0);
         if (rc != WISV_OK) return rc;
         c->launches++;
     } else if (!rows_done) {

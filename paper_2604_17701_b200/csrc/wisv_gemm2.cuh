@@ -29,7 +29,12 @@ struct PairParams {
                          // stay resident in L2 while the weights stream past them
     int32_t n_tiles;     // vocabulary tiles of 256
     int32_t stages;
-    int32_t part_stride; // partials per row (= n_tiles)
+    // One row tile of 256 (carry = 1): the vocabulary is dealt out in units of 32 rows as one contiguous range per
+    // pair - units_base units, one more for the first units_rem pairs - cut into tiles_per_pair tiles of tile_n or
+    // tile_n - 32 rows; a pair carries its running row state across its tiles and writes one partial per (row, pair).
+    // The pairs then finish together for any vocabulary size and any number of pairs.
+    int32_t carry, units_base, units_rem, tiles_per_pair, tile_n;
+    int32_t part_stride; // partials per row (n_tiles, or the number of pairs when carry)
     int32_t* err;
     float4* lm_part;
     const int32_t* row_tok;
@@ -38,10 +43,22 @@ struct PairParams {
 
 __host__ __device__ inline uint32_t pair_fixed_bytes() { return 1024u + 1024u; }   // alignment slack + barriers
 
+// CTAs from lm_ctas on (whole clusters) do not belong to a pair: they evaluate the decision head with the
+// single-CTA GEMM body while the pairs stream the LM head (batches of at most 256 window rows, where the
+// LM head is bound by HBM and the head would otherwise add its whole latency to the round).
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                   const PairParams p)
+                   const __grid_constant__ CUtensorMap tmB2, const PairParams p,
+                   const __grid_constant__ CUtensorMap tmZ, const __grid_constant__ CUtensorMap tmW1,
+                   const __grid_constant__ CUtensorMap tmW1_2, const GemmParams hd, const int lm_ctas,
+                   const int head_ctas)
 {
+    if (static_cast<int>(blockIdx.x) >= lm_ctas) {
+        // (the grid is a whole number of clusters: with an odd head_ctas the last CTA has nothing to do)
+        const int hc = static_cast<int>(blockIdx.x) - lm_ctas;
+        if (hc < head_ctas) gemm_rowreduce_body<EPI_HEAD, false>(tmZ, tmW1, tmW1_2, hd, hc, head_ctas);
+        return;
+    }
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;
@@ -51,7 +68,7 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     const uint32_t rank = cluster_ctarank();
     const bool leader = rank == 0;
     const int pair_id = blockIdx.x >> 1;
-    const int n_pairs = gridDim.x >> 1;
+    const int n_pairs = lm_ctas >> 1;
     const uint32_t half_bytes = kTileM * kBlockK * 2;                 // 16 KB
     const uint32_t ring_bytes = kPairStageBytes * static_cast<uint32_t>(p.stages);
 
@@ -77,6 +94,28 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         *n = idx / gsize;
         *mp = mp0 + idx % gsize;
     };
+    // carry: this pair's contiguous range of 32-row units and how it is cut into tiles
+    const int my_units = p.units_base + (pair_id < p.units_rem ? 1 : 0);
+    const int my_unit0 = pair_id * p.units_base + (pair_id < p.units_rem ? pair_id : p.units_rem);
+    const int my_tiles = p.carry ? (my_units < p.tiles_per_pair ? my_units : p.tiles_per_pair) : 0;
+    const int my_hq = p.carry ? my_units / p.tiles_per_pair : 0;
+    const int my_hr = p.carry ? my_units % p.tiles_per_pair : 0;
+    // the i-th tile of this pair: row tile mp, first vocabulary row n0, height h (a multiple of 32), tile index n
+    struct PTile { int mp, n, n0, h; };
+    auto tile_at = [&](int i, PTile& w) -> bool {
+        if (p.carry) {
+            if (i >= my_tiles) return false;
+            w.mp = 0; w.n = pair_id;
+            w.h = (my_hq + (i < my_hr ? 1 : 0)) * 32;
+            w.n0 = (my_unit0 + i * my_hq + (i < my_hr ? i : my_hr)) * 32;
+            return true;
+        }
+        const int t = pair_id + i * n_pairs;
+        if (t >= total_tiles) return false;
+        tile_mp_n(t, &w.mp, &w.n);
+        w.n0 = w.n * kPairTileN; w.h = kPairTileN;
+        return true;
+    };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -100,8 +139,13 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    griddep_wait();                    // the pack kernel wrote the bf16 rows this kernel loads
-    griddep_launch_dependents();
+    // The pack kernel wrote the bf16 rows this kernel loads: everyone waits for it here, except the producer
+    // thread, which first puts one ring-full of weight tiles in flight (they depend on nothing) and waits then.
+    const bool producer_thread = warp == 0 && lane == 0;
+    if (!producer_thread) {
+        griddep_wait();
+        griddep_launch_dependents();
+    }
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (each CTA)
@@ -110,32 +154,53 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             uint32_t ph = 0;
             long long issued = 0;
             bool ok = true;
-            for (int t = pair_id; t < total_tiles && ok; t += n_pairs) {
-                int mp, n;
-                tile_mp_n(t, &mp, &n);
-                const int row0 = mp * kPairTileM + static_cast<int>(rank) * kTileM;
-                const int col0 = n * kPairTileN + static_cast<int>(rank) * kTileM;
+            PTile w;
+            long long pre = 0;                 // stages whose weight half-tile was requested before the wait
+            for (int i = 0; pre < p.stages && tile_at(i, w); ++i) {
+                const int half_h = w.h >> 1;
+                const int col0 = w.n0 + static_cast<int>(rank) * half_h;
+                const CUtensorMap* mapB = (w.h == p.tile_n) ? &tmB : &tmB2;
+                const uint32_t tx = 2u * (half_bytes + static_cast<uint32_t>(half_h) * kBlockK * 2u);
+                for (int kb = 0; kb < p.k_blocks && pre < p.stages; ++kb, ++pre) {
+                    const uint32_t a_dst = smem_base + kPairStageBytes * static_cast<uint32_t>(pre);
+                    if (leader) mbar_expect_tx(full_bar(static_cast<int>(pre)), tx);
+                    tma_load_2d_pair(a_dst + half_bytes, mapB, kb * kBlockK, col0, full_bar(static_cast<int>(pre)));
+                }
+            }
+            griddep_wait();
+            griddep_launch_dependents();
+            for (int i = 0; ok && tile_at(i, w); ++i) {
+                const int row0 = w.mp * kPairTileM + static_cast<int>(rank) * kTileM;
+                const int half_h = w.h >> 1;                                   // weight rows this CTA loads
+                const int col0 = w.n0 + static_cast<int>(rank) * half_h;
+                const CUtensorMap* mapB = (w.h == p.tile_n) ? &tmB : &tmB2;
+                const uint32_t tx = 2u * (half_bytes + static_cast<uint32_t>(half_h) * kBlockK * 2u);
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
-                    if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, kWaitLimitNs)) { ok = false; break; }
                     const uint32_t a_dst = smem_base + kPairStageBytes * s;
-                    if (leader) mbar_expect_tx(full_bar(s), 2u * kPairStageBytes);   // both CTAs' bytes
-                    tma_load_2d_pair(a_dst, &tmA, kb * kBlockK, row0, full_bar(s));
-                    tma_load_2d_pair(a_dst + half_bytes, &tmB, kb * kBlockK, col0, full_bar(s));
+                    if (issued < pre) {
+                        // first pass over the ring: the stage is free, its bytes are expected and its weight
+                        // half-tile is already on its way
+                        tma_load_2d_pair(a_dst, &tmA, kb * kBlockK, row0, full_bar(s));
+                    } else {
+                        if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, kWaitLimitNs)) { ok = false; break; }
+                        if (leader) mbar_expect_tx(full_bar(s), tx);             // both CTAs' bytes
+                        tma_load_2d_pair(a_dst, &tmA, kb * kBlockK, row0, full_bar(s));
+                        tma_load_2d_pair(a_dst + half_bytes, mapB, kb * kBlockK, col0, full_bar(s));
+                    }
                     ++issued;
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
             }
-            (void)issued;
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (leader CTA only)
         if (lane == 0 && leader) {
-            const uint32_t idesc = idesc_bf16_f32(kPairTileM, kPairTileN);
             int s = 0;
             uint32_t ph = 0;
-            int local = 0;
             bool ok = true;
-            for (int t = pair_id; t < total_tiles && ok; t += n_pairs, ++local) {
+            PTile w;
+            for (int local = 0; ok && tile_at(local, w); ++local) {
+                const uint32_t idesc = idesc_bf16_f32(kPairTileM, static_cast<uint32_t>(w.h));
                 const int as = local & 1;
                 const uint32_t aph = (local >> 1) & 1u;
                 if (!mbar_wait_bounded(acc_empty_bar(as), aph ^ 1u, abort_flag, kWaitLimitNs)) { ok = false; break; }
@@ -163,18 +228,18 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     } else {
         // ------------------------------------------------------------ epilogue (warps 2..5 of each CTA)
         const int q = warp & 3;
-        int local = 0;
         bool ok = true;
         const uint32_t leader_acc_empty0 = mapa_u32(acc_empty_bar(0), 0);
         const uint32_t leader_acc_empty1 = mapa_u32(acc_empty_bar(1), 0);
-        for (int t = pair_id; t < total_tiles && ok; t += n_pairs, ++local) {
-            int mp, n;
-            tile_mp_n(t, &mp, &n);
+        float mx = -CUDART_INF_F, sum = 0.0f;      // running row state: per tile, or per pair when carry
+        int arg = 0;
+        PTile w;
+        int last_row = -1;
+        for (int local = 0; ok && tile_at(local, w); ++local) {
             const int as = local & 1;
             const uint32_t aph = (local >> 1) & 1u;
-            const int row = mp * kPairTileM + static_cast<int>(rank) * kTileM + q * 32 + lane;
+            const int row = w.mp * kPairTileM + static_cast<int>(rank) * kTileM + q * 32 + lane;
             const bool valid = row < p.rows;
-            const int n0 = n * kPairTileN;
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(as * kAccCols);
 
             bool got = mbar_wait_bounded(acc_full_bar(as), aph, abort_flag, kWaitLimitNs);
@@ -182,22 +247,27 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             if (!got) { ok = false; break; }
             tc_fence_after();
 
-            float mx = -CUDART_INF_F, sum = 0.0f;
-            int arg = 0;
+            if (!p.carry) { mx = -CUDART_INF_F; sum = 0.0f; arg = 0; }
             const int tok = valid ? p.row_tok[row] : -1;
-            for (int c0 = 0; c0 < kPairTileN; c0 += 16) {
+            for (int c0 = 0; c0 < w.h; c0 += 16) {
                 uint32_t v[16];
                 __syncwarp();
                 tmem_ld16(taddr + static_cast<uint32_t>(c0), v);
                 tmem_wait_ld();
                 if (!valid) continue;
-                lm_update_chunk(v, n0 + c0, p.n_total, tok, mx, arg, sum, p.tok_logit + row);
+                lm_update_chunk(v, w.n0 + c0, p.n_total, tok, mx, arg, sum, p.tok_logit + row);
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(as ? leader_acc_empty1 : leader_acc_empty0);
-            if (valid) p.lm_part[(size_t)row * p.part_stride + n] = make_float4(mx, __int_as_float(arg), sum, 0.0f);
+            if (valid && !p.carry)
+                p.lm_part[(size_t)row * p.part_stride + w.n] = make_float4(mx, __int_as_float(arg), sum, 0.0f);
+            last_row = valid ? row : -1;
         }
+        // carry: the tiles of a pair ascend through the vocabulary, so the strict '>' of the update kept the
+        // lowest index; a pair without tiles is never launched
+        if (p.carry && ok && last_row >= 0)
+            p.lm_part[(size_t)last_row * p.part_stride + pair_id] = make_float4(mx, __int_as_float(arg), sum, 0.0f);
     }
 
     // neither CTA may retire (or release TMEM) while its partner can still signal or read it

@@ -153,14 +153,55 @@ def test_cta_pair_kernel_matches_single_cta_kernel():
     case, ref, out, _ = _run(cfg)
     d = cases.to_device(case, DEV)
     v = cases.make_verifier(d)
-    assert v.plan(case["R"], case["T"])["lm_tiles"] == 4    # ceil(1000 / 256) tiles of 256 x 256
+    plan = v.plan(case["R"], case["T"])
+    assert plan["lm_ctas"] == 64 and plan["lm_tile_n"] == 32    # 32 units of 32 vocabulary rows, one per CTA pair
+    assert v.plan_kernels(case["R"], case["T"]) == 3            # the decision head rides in the same launch
     v.set_tuning(lm_single_cta=1)
-    assert v.plan(case["R"], case["T"])["lm_tiles"] == 8
+    assert v.plan(case["R"], case["T"])["lm_tiles"] == 8        # 2 row tiles x ceil(1000 / 256) tiles of 128 x 256
+    assert v.plan_kernels(case["R"], case["T"]) == 4
     o2 = cases.run(v, d)
     torch.cuda.synchronize()
     assert v.device_error() == 0
     assert torch.equal(o2.argmax, out.argmax) and torch.equal(o2.accept_len, out.accept_len)
     assert float((o2.lse - out.lse).abs().max()) < 1e-5
+    v.close()
+
+
+@pytest.mark.parametrize("kw", [dict(B=26, K=4), dict(B=16, K=8, V=5000), dict(B=50, K=4, V=1000),
+                                dict(B=28, K=8, d_J=200, V=4099), dict(B=40, K=0, K_lo=1, K_hi=9),
+                                dict(B=30, K=6, mode="SH"), dict(B=25, K=9, stochastic=True)],
+                         ids=["R130", "R144", "R250", "R252odd", "ragged", "SH", "stoch"])
+@pytest.mark.parametrize("head_ctas", [0, 2, 5, -1], ids=["default", "h2", "h5", "separate"])
+def test_two_row_tiles_pairs_with_head_clusters(kw, head_ctas):
+    """129..256 window rows: the LM head runs on CTA pairs, each with one contiguous vocabulary range, and the
+    decision head on extra clusters of the same launch (three kernels per round); -1 launches it separately."""
+    cfg = _small(seed=37, **kw)
+    case = cases.make_case(cfg, oracle_ref_argmax)
+    if cfg.stochastic:
+        base = run_oracle(case)
+        case["draft_q"] = (base["p_draft"] * np.random.default_rng(5).uniform(0.5, 4.0, size=case["T"])).astype(np.float32)
+    assert 128 < case["R"] <= 256
+    ref = run_oracle(case)
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d)
+    v.set_tuning(head_ctas=head_ctas)
+    P = case["T"] if case["sel_pos"] is None else int(case["sel_pos"].shape[0])
+    assert v.plan_kernels(case["R"], P) == (4 if head_ctas < 0 else 3)
+    n0 = v.launch_count()
+    for _ in range(2):
+        out = cases.run(v, d)
+    torch.cuda.synchronize()
+    assert v.launch_count() - n0 == (8 if head_ctas < 0 else 6)
+    assert v.device_error() == 0
+    compare(case, ref, out, cfg.tau)
+    v.set_tuning(lm_single_cta=1)
+    one = cases.run(v, d)
+    torch.cuda.synchronize()
+    assert v.device_error() == 0
+    assert torch.equal(one.argmax, out.argmax) and torch.equal(one.accept_len, out.accept_len)
+    assert torch.equal(one.correction_token, out.correction_token)
+    assert float((one.lse - out.lse).abs().max()) < 1e-5
+    assert float((one.head_prob - out.head_prob).abs().max()) < 1e-5
     v.close()
 
 
