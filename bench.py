@@ -43,12 +43,14 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 SINGLE_CTA_SOURCES = ("wisv_gemm.cuh", "wisv_ptx.cuh")
 CTA_PAIR_SOURCES = ("wisv_gemm2.cuh", "wisv_gemm.cuh", "wisv_ptx.cuh")
 NCU_TRAFFIC = {
-    # LM-head and decision-head CTAs in one launch, 9 window rows: 1.0642 GB read + 4.4 MB written per launch
-    "8b_b1": {"bytes": 1068600000, "files": SINGLE_CTA_SOURCES, "kernel_hash": "246e580b4bdc4e06"},
-    # single-CTA kernel, 576 window rows: 1.0589 GB read + 8.4 MB written per launch
-    "8b_b64": {"bytes": 1067400000, "files": SINGLE_CTA_SOURCES, "kernel_hash": "246e580b4bdc4e06"},
-    # CTA-pair kernel, 8704 window rows: 6.013 GB read + 102.7 MB written per launch (4.6-6.0 GB between captures)
-    "8b_b512": {"bytes": 6115700000, "files": CTA_PAIR_SOURCES, "kernel_hash": "4873c99cd8dddf90"},
+    # LM-head and decision-head CTAs in one launch, 9 window rows: 1.0642 GB read + 3.9 MB written per launch
+    "8b_b1": {"bytes": 1068000000, "files": SINGLE_CTA_SOURCES, "kernel_hash": "0d1c02dd776a3318"},
+    # CTA pairs + decision-head clusters, 144 window rows: 1.0831 GB read + 4.5 MB written per launch
+    "8b_b16": {"bytes": 1087600000, "files": CTA_PAIR_SOURCES, "kernel_hash": "158ceb32802da36d"},
+    # single-CTA kernel, 576 window rows: 1.0585 GB read + 9.2 MB written per launch
+    "8b_b64": {"bytes": 1067800000, "files": SINGLE_CTA_SOURCES, "kernel_hash": "0d1c02dd776a3318"},
+    # CTA-pair kernel, 8704 window rows: 3.898 GB read + 81.8 MB written per launch (3.9-8.5 GB between captures)
+    "8b_b512": {"bytes": 3980000000, "files": CTA_PAIR_SOURCES, "kernel_hash": "158ceb32802da36d"},
 }
 
 
@@ -400,11 +402,14 @@ def run_ours(args, rank, world, local_rank):
             peak = float(peaks["bf16_tflops_sustained" if long_step else "bf16_tflops"])
             roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                     "traffic": captured_traffic(cfg.name)}
-        pair_tiles = -(-R // 256) * -(-cfg.V // 256)
-        on_pairs = R > 128 and plan["lm_tile_n"] == 256 and plan["lm_tiles"] == pair_tiles
+        # which LM-head kernel the library's plan uses (same rule as the planner: CTA pairs for an even number of
+        # 128-row tiles or at least 11 of them)
+        tiles128 = -(-R // 128)
+        on_pairs = tiles128 >= 2 and (tiles128 % 2 == 0 or tiles128 >= 11)
         kernel_name = "lmhead_pair_kernel (CTA pairs)" if on_pairs else "gemm_rowreduce_kernel<LM head>"
         if one_launch:
-            kernel_name = "round_small_kernel (LM-head CTAs + decision-head CTAs)"
+            kernel_name = ("lmhead_pair_kernel (CTA pairs + decision-head clusters)" if on_pairs
+                           else "round_small_kernel (LM-head CTAs + decision-head CTAs)")
         roof.update({"kernel": kernel_name,
                      "kernel_ms": lm_ms, "peak_source": peak_kind,
                      "algorithmic_bytes": w_bytes, "algorithmic_flops": flops,

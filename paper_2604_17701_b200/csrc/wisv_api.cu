@@ -782,8 +782,6 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
     if (fused) {
         // both GEMMs in one launch: LM-head CTAs and decision-head CTAs side by side
         if ((size_t)P * ph.parts > c->head_part_elems) return WISV_ECAPACITY;
-        GemmParams gl = base_params(c, pl, R, cf.V, cf.H);
-        gl.lm_part = c->lm_part; gl.row_tok = c->row_tok; gl.tok_logit = c->tok_logit;
         GemmParams gh = base_params(c, ph, P, cf.d_J, cf.H_d + cf.H);
         gh.head_part = c->head_part; gh.b1 = c->w.b1; gh.w2 = c->w.w2; gh.w1c = c->W1c; gh.csi = b->csi;
         gh.pos_req = c->pos_req; gh.d_c = cf.d_c; gh.act = cf.act;
@@ -796,6 +794,8 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
                                       pl.ctas, ph.ctas);
             if (rc != WISV_OK) return rc;
         } else {
+            GemmParams gl = base_params(c, pl, R, cf.V, cf.H);
+            gl.lm_part = c->lm_part; gl.row_tok = c->row_tok; gl.tok_logit = c->tok_logit;
             const int rc = launch_pdl(round_small_kernel, dim3(pl.ctas + ph.ctas), dim3(kGemmThreads), smem, st,
                                       c->tmX[pl.a_rows / 8 - 1], c->tmW[map_hi(pl)], c->tmW[map_lo(pl)],
                                       c->tmZ[ph.a_rows / 8 - 1], c->tmW1[map_hi(ph)], c->tmW1[map_lo(ph)], gl, gh,

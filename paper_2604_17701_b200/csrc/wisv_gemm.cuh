@@ -93,7 +93,7 @@ __host__ __device__ inline uint32_t gemm_overread_bytes(int a_rows) {
 }
 // bytes after the stage ring: barriers + tmem slot + abort flag, then epilogue constants
 __host__ __device__ inline uint32_t gemm_tail_bytes(int tile_n, int d_c) {
-    return 1024u + 4096u + 2u * (static_cast<uint32_t>(tile_n) * static_cast<uint32_t>(2 + d_c) +
+    return 1024u + 2u * (static_cast<uint32_t>(tile_n) * static_cast<uint32_t>(2 + d_c) +
                         static_cast<uint32_t>(kEpiThreads * d_c)) * 4u;
 }
 
@@ -160,7 +160,7 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + ring_bytes + 8 * (2 * kMaxStages + 5));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [0] abort, [1] drain scratch
     volatile int* last_flag = abort_flag + 2;                                    // split-K: this CTA finishes the tile
-    float* epi_const = reinterpret_cast<float*>(smem + ring_bytes + 1024 + 4096);
+    float* epi_const = reinterpret_cast<float*>(smem + ring_bytes + 1024);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
