@@ -288,21 +288,13 @@ Plan plan_head(const wisv_ctx* c, int P)
 // to stream its weights - and the LM head is planned for the SMs that remain.
 constexpr int kFusedHeadCtas = 6;
 constexpr int kFusedHeadCtasTwoTiles = 8;     // head positions in two row tiles (129..255)
-bool plan_fused(const wisv_ctx* c, int R, int P, Plan* lm, Plan* hd)
+
+// decision-head plan for `want` CTAs that share a launch with the LM head (K never split)
+Plan plan_head_beside(const wisv_ctx* c, int P, int want)
 {
-    if (c->tune.head_ctas < 0 || R < 1 || P < 1) return false;
-    const bool small = R <= kTileM && P <= kTileM;
-    // up to 256 window rows: the LM head runs on CTA pairs (one row tile of 256, still bound by HBM) and the
-    // decision head on a few clusters of the same launch
-    const bool with_pairs = !small && R <= kPairTileM && P <= kPairTileM && c->max_pairs > 2 &&
-                            !c->tune.lm_single_cta && !c->tune.lm_tile_n;
-    if (!small && !with_pairs) return false;
-    const int head_m_tiles = (P + kTileM - 1) / kTileM;
-    int want = c->tune.head_ctas > 0 ? c->tune.head_ctas : (head_m_tiles > 1 ? kFusedHeadCtasTwoTiles : kFusedHeadCtas);
-    if (want > c->sm_count / 2) want = c->sm_count / 2;
-    if (want < 1) return false;
     Plan h{};
     const int N = c->cfg.d_J;
+    const int head_m_tiles = (P + kTileM - 1) / kTileM;
     int tn = head_m_tiles > 1 ? 128 : kSplitTileN;
     if (c->tune.head_tile_n >= 16 && c->tune.head_tile_n <= kMaxTileN && c->tune.head_tile_n % 16 == 0) tn = c->tune.head_tile_n;
     if (tn > round_up(N, 16)) tn = round_up(N, 16);
@@ -311,10 +303,55 @@ bool plan_fused(const wisv_ctx* c, int R, int P, Plan* lm, Plan* hd)
     h.k_splits = 1;
     h.kb_per_split = (c->cfg.H_d + c->cfg.H + kBlockK - 1) / kBlockK;
     finish_plan(c, &h, c->cfg.d_c, h.kb_per_split, c->tune.head_stages, want, N);
-    *hd = h;
-    if (small) *lm = plan_lm(c, R, true, c->sm_count - h.ctas);
-    else *lm = plan_lm(c, R, false, 0, (h.ctas + 1) / 2);
-    return true;
+    return h;
+}
+
+// rounds of tiles the slowest CTA (or pair) of a plan without carried ranges works through
+long long plan_waves(const Plan& p)
+{
+    const long long units = p.pair ? p.ctas / 2 : p.ctas;
+    const long long items = (long long)p.m_tiles * p.n_tiles * (p.k_splits > 0 ? p.k_splits : 1);
+    return units > 0 ? (items + units - 1) / units : 0;
+}
+
+bool plan_fused(const wisv_ctx* c, int R, int P, Plan* lm, Plan* hd)
+{
+    if (c->tune.head_ctas < 0 || R < 1 || P < 1) return false;
+    const bool small = R <= kTileM && P <= kTileM;
+    // up to 256 window rows: the LM head runs on CTA pairs (one row tile of 256, still bound by HBM) and the
+    // decision head on a few clusters of the same launch
+    const bool with_pairs = !small && R <= kPairTileM && P <= kPairTileM && c->max_pairs > 2 &&
+                            !c->tune.lm_single_cta && !c->tune.lm_tile_n;
+    if (small || with_pairs) {
+        const int head_m_tiles = (P + kTileM - 1) / kTileM;
+        int want = c->tune.head_ctas > 0 ? c->tune.head_ctas : (head_m_tiles > 1 ? kFusedHeadCtasTwoTiles : kFusedHeadCtas);
+        if (want > c->sm_count / 2) want = c->sm_count / 2;
+        if (want < 1) return false;
+        const Plan h = plan_head_beside(c, P, want);
+        *hd = h;
+        if (small) *lm = plan_lm(c, R, true, c->sm_count - h.ctas);
+        else *lm = plan_lm(c, R, false, 0, (h.ctas + 1) / 2);
+        return true;
+    }
+    // More rows (tensor-bound, tiles dealt out round-robin): giving SMs to the decision head pays only if the LM
+    // head does not need another round of tiles for it and the head finishes well inside the LM head's time.
+    // Times are counted in tiles: an LM-head tile and a decision-head item both walk a K range of similar cost
+    // (64 K blocks of 128 x 256 against 96 of 128 x 128), so an item is taken as 1.2 tiles.
+    if (c->tune.lm_tile_n) return false;
+    const Plan base = plan_lm(c, R);
+    const long long base_waves = plan_waves(base);
+    for (int want = 2; want <= 16; want += 2) {
+        if (c->tune.head_ctas > 0 && want != round_up(c->tune.head_ctas, 2)) continue;
+        if (want > c->sm_count / 4) break;
+        const Plan h = plan_head_beside(c, P, want);
+        const Plan l = plan_lm(c, R, false, c->sm_count - round_up(h.ctas, 2), (h.ctas + 1) / 2);
+        if (l.pair != base.pair || plan_waves(l) != base_waves) continue;
+        const long long head_rounds = plan_waves(h);
+        if (c->tune.head_ctas == 0 && head_rounds * 12 > base_waves * 8) continue;     // 1.2 tiles each, 80 % of the time
+        *hd = h; *lm = l;
+        return true;
+    }
+    return false;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

@@ -205,6 +205,38 @@ def test_two_row_tiles_pairs_with_head_clusters(kw, head_ctas):
     v.close()
 
 
+@pytest.mark.parametrize("kw", [dict(B=60, K=4), dict(B=40, K=8, d_J=200), dict(B=100, K=4, V=2000),
+                                dict(B=70, K=0, K_lo=2, K_hi=9, V=3000), dict(B=90, K=6, mode="SH")],
+                         ids=["R300", "R360", "R500pairs", "ragged", "SH"])
+def test_more_row_tiles_share_a_launch_when_it_costs_no_extra_round_of_tiles(kw):
+    """More than 256 window rows: decision-head CTAs ride in the LM-head launch (single-CTA or pair kernel)
+    whenever the LM head needs no additional round of tiles for it; the result must equal separate launches."""
+    cfg = _small(seed=43, **kw)
+    case = cases.make_case(cfg, oracle_ref_argmax)
+    assert case["R"] > 256
+    ref = run_oracle(case)
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d)
+    P = case["T"] if case["sel_pos"] is None else int(case["sel_pos"].shape[0])
+    # with so few vocabulary tiles the LM head is a single round of tiles and the automatic plan keeps the launches
+    # apart (the head would outlast it); asking for head CTAs by hand skips that estimate, not the round check
+    v.set_tuning(head_ctas=4)
+    assert v.plan_kernels(case["R"], P) == 3
+    out = cases.run(v, d)
+    torch.cuda.synchronize()
+    assert v.device_error() == 0
+    compare(case, ref, out, cfg.tau)
+    v.set_tuning(head_ctas=-1)
+    assert v.plan_kernels(case["R"], P) == 4
+    sep = cases.run(v, d)
+    torch.cuda.synchronize()
+    assert v.device_error() == 0
+    assert torch.equal(sep.argmax, out.argmax) and torch.equal(sep.accept_len, out.accept_len)
+    assert torch.equal(sep.correction_token, out.correction_token) and torch.equal(sep.lse, out.lse)
+    assert float((sep.head_prob - out.head_prob).abs().max()) < 1e-5
+    v.close()
+
+
 @pytest.mark.parametrize("B,K", [(1, 8), (4, 3), (2, 8), (8, 4), (7, 8), (8, 7), (13, 4)],
                          ids=["R9", "R16", "R18", "R40", "R63", "R64", "R65"])
 @pytest.mark.parametrize("head_ctas", [0, -1], ids=["one_launch", "two_launches"])
