@@ -247,8 +247,9 @@ int wisv_profile_read(wisv_ctx* ctx, int32_t stage, float* ms, int32_t cap, int3
 typedef struct {
     int32_t lm_tile_n, lm_stages, head_tile_n, head_stages;
     int32_t lm_single_cta;   /* 1: never use the CTA-pair LM-head kernel (batches with more than 128 window rows) */
-    int32_t head_ctas;       /* batches of at most 128 window rows and 128 head positions run both GEMMs in one
-                                launch: CTAs given to the decision head there (0 = default), -1 = two launches */
+    int32_t head_ctas;       /* where the two GEMMs share one launch (always up to 256 window rows; with more rows
+                                when it costs the LM head no extra round of tiles): CTAs given to the decision head
+                                there (0 = chosen automatically), -1 = always two launches */
     int32_t lm_mma_m;        /* 128: never use 64-row MMAs (the default for GEMMs with at most 64 valid rows) */
 } wisv_tuning;
 int wisv_set_tuning(wisv_ctx* ctx, const wisv_tuning* tuning);
@@ -266,8 +267,9 @@ int wisv_plan(const wisv_ctx* ctx, int32_t R, int32_t P, int32_t* lm_tile_n, int
 
 /*
  * Kernels one wisv_verify round launches for such a batch: 4 (pack, LM head,
- * decision head, merge + scan), or 3 when the batch has at most 128 window rows
- * and 128 head positions and the two GEMMs share one launch, or when P = 0.
+ * decision head, merge + scan), or 3 when decision-head CTAs ride in the LM-head
+ * launch (every batch of at most 256 window rows; larger ones when the LM head
+ * needs no additional round of tiles for it), or when P = 0.
  * Negative on bad arguments.
  */
 int wisv_plan_kernels(const wisv_ctx* ctx, int32_t R, int32_t P);
