@@ -644,6 +644,14 @@ def test_8b_batch1_full_oracle():
     _sampled_parity("8b_b1", 1)
 
 
+@pytest.mark.parametrize("name", ["8b_b16", "8b_b32"])
+def test_8b_two_and_three_row_tiles_sampled(name):
+    # 144 rows: CTA pairs with balanced vocabulary ranges + decision-head clusters; 288 rows: three row tiles on
+    # the single-CTA kernel with decision-head CTAs in the same launch
+    case, out, A, stats = _sampled_parity(name, 12)
+    assert stats["tainted_requests"] < stats["requests"]
+
+
 @pytest.mark.parametrize("name", ["8b_b64_m30", "8b_b64", "8b_b64_m95"])
 def test_8b_batch64_sampled(name):
     case, out, A, stats = _sampled_parity(name, 16)
