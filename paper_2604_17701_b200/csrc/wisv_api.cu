@@ -532,8 +532,9 @@ GemmParams base_params(const wisv_ctx* c, const Plan& pl, int rows, int n_total,
     gp.tile_n = pl.tile_n; gp.m_tiles = pl.m_tiles; gp.n_tiles = pl.n_tiles; gp.stages = pl.stages;
     gp.a_rows = pl.a_rows; gp.carry = pl.carry; gp.part_stride = pl.parts;
     gp.k_splits = pl.k_splits; gp.kb_per_split = pl.kb_per_split;
-    // one row tile with at most 64 valid rows: MMAs of 64 rows do the same job with half the tensor work
-    gp.mma_m = (pl.m_tiles == 1 && rows <= 64 && c->tune.lm_mma_m != kTileM) ? 64 : kTileM;
+    // row tiles with at most 64 valid rows (a small batch, or the ragged last tile of a large one): MMAs of 64
+    // rows do the same job with half the tensor work
+    gp.mma_m = c->tune.lm_mma_m != kTileM ? 64 : kTileM;
     gp.units_base = pl.units_base; gp.units_rem = pl.units_rem; gp.tiles_per_cta = pl.tiles_per_cta;
     gp.splitk_buf = c->splitk_buf; gp.splitk_count = c->splitk_count;
     gp.err = c->err;

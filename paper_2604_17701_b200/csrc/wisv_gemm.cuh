@@ -48,10 +48,10 @@ struct GemmParams {
     int32_t a_rows;      // rows of A actually loaded per tile (multiple of 8, <= 128); the MMA still spans
                          // 128 rows, the rest of its A operand is whatever follows in shared memory and only
                          // feeds accumulator rows that are never read
-    int32_t mma_m;       // rows of one MMA: 128 (accumulator row i in TMEM lane i), or 64 when the one row tile has
-                         // at most 64 valid rows (row i in lane (i / 16) * 32 + i % 16: sixteen lanes of each
-                         // quadrant) - half the tensor work per weight byte, which the HBM-bound case turns
-                         // into lower power and higher clocks
+    int32_t mma_m;       // 128: every MMA spans 128 rows (accumulator row i in TMEM lane i).  64: a row tile with at
+                         // most 64 valid rows is computed with MMAs of 64 rows (row i in lane (i / 16) * 32 + i % 16:
+                         // sixteen lanes of each quadrant) - half the tensor work for that tile, which under the
+                         // power cap means higher clocks
     int32_t carry;       // 1: one row tile, each CTA keeps its running row state across its tiles and
                          //    writes one partial per (row, CTA); 0: one partial per (row, N-tile)
     // carry only: the rows of Bw are dealt out in units of 16 as one contiguous range per CTA - CTA c gets
@@ -196,6 +196,8 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
         return true;
     };
     auto b_map = [&](int h) -> const CUtensorMap* { return h == p.tile_n ? &tmB : &tmB2; };
+    // rows of the MMAs of row tile m (see GemmParams::mma_m)
+    auto tile_mma_m = [&](int m) { return (p.mma_m == 64 && p.rows - m * kTileM <= 64) ? 64 : kTileM; };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -288,7 +290,7 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
             bool ok = true;
             Item w;
             for (int local = 0; ok && item_at(local, w); ++local) {
-                const uint32_t idesc = idesc_bf16_f32(static_cast<uint32_t>(p.mma_m), static_cast<uint32_t>(w.h));
+                const uint32_t idesc = idesc_bf16_f32(static_cast<uint32_t>(tile_mma_m(w.m)), static_cast<uint32_t>(w.h));
                 const int as = local & 1;
                 const uint32_t aph = (local >> 1) & 1u;
                 if (!mbar_wait_bounded(acc_empty_bar(as), aph ^ 1u, abort_flag, kWaitLimitNs)) { ok = false; break; }
@@ -321,9 +323,6 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
         // ------------------------------------------------------------ epilogue (warps 2..5)
         const int q = warp & 3;                            // TMEM lane quadrant this warp may read
         const int et = threadIdx.x - 64;                   // 0..127 among epilogue threads
-        // row of the tile held by this thread's TMEM lane (see GemmParams::mma_m)
-        const int rit = p.mma_m == 64 ? q * 16 + (lane & 15) : q * 32 + lane;
-        const bool lane_used = p.mma_m == 64 ? lane < 16 : true;
         bool ok = true;
         float mx = -CUDART_INF_F, sum = 0.0f, hs = 0.0f;   // running row state (per tile, or per CTA when carry)
         int arg = 0;
@@ -332,6 +331,10 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
             const int t = w.t, m = w.m, n = w.n;
             const int as = local & 1;
             const uint32_t aph = (local >> 1) & 1u;
+            // row of the tile held by this thread's TMEM lane
+            const bool m64 = tile_mma_m(m) == 64;
+            const int rit = m64 ? q * 16 + (lane & 15) : q * 32 + lane;
+            const bool lane_used = m64 ? lane < 16 : true;
             const int row = m * kTileM + rit;
             const bool valid = lane_used && row < p.rows;
             const int n0 = w.n0;
@@ -485,8 +488,9 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
         if (p.carry && ok) {
             // one row tile: tiles of this CTA ascend through the vocabulary, so the strict '>' above
             // already kept the lowest index; a CTA without tiles is never launched
-            const int row = rit;
-            if (lane_used && row < p.rows) {
+            const bool m64 = tile_mma_m(0) == 64;
+            const int row = m64 ? q * 16 + (lane & 15) : q * 32 + lane;
+            if ((m64 ? lane < 16 : true) && row < p.rows) {
                 if (EPI == EPI_LMHEAD)
                     p.lm_part[(size_t)row * p.part_stride + cta] = make_float4(mx, __int_as_float(arg), sum, 0.0f);
                 else if (EPI == EPI_HEAD)

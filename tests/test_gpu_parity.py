@@ -226,6 +226,13 @@ def test_more_row_tiles_share_a_launch_when_it_costs_no_extra_round_of_tiles(kw)
     torch.cuda.synchronize()
     assert v.device_error() == 0
     compare(case, ref, out, cfg.tau)
+    # a ragged last row tile with at most 64 rows runs on 64-row MMAs: forcing 128-row MMAs changes no bit
+    v.set_tuning(head_ctas=4, lm_mma_m=128)
+    big = cases.run(v, d)
+    torch.cuda.synchronize()
+    assert v.device_error() == 0
+    for k in ("accept_len", "correction_token", "argmax", "lse", "p_draft", "head_prob", "n_mismatch", "status"):
+        assert torch.equal(getattr(big, k), getattr(out, k)), k
     v.set_tuning(head_ctas=-1)
     assert v.plan_kernels(case["R"], P) == 4
     sep = cases.run(v, d)
