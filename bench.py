@@ -43,14 +43,14 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 SINGLE_CTA_SOURCES = ("wisv_gemm.cuh", "wisv_ptx.cuh")
 CTA_PAIR_SOURCES = ("wisv_gemm2.cuh", "wisv_gemm.cuh", "wisv_ptx.cuh")
 NCU_TRAFFIC = {
-    # LM-head and decision-head CTAs in one launch, 9 window rows: 1.0642 GB read + 3.9 MB written per launch
-    "8b_b1": {"bytes": 1068000000, "files": SINGLE_CTA_SOURCES, "kernel_hash": "0d1c02dd776a3318"},
-    # CTA pairs + decision-head clusters, 144 window rows: 1.0831 GB read + 4.5 MB written per launch
-    "8b_b16": {"bytes": 1087600000, "files": CTA_PAIR_SOURCES, "kernel_hash": "158ceb32802da36d"},
-    # single-CTA kernel, 576 window rows: 1.0585 GB read + 9.2 MB written per launch
-    "8b_b64": {"bytes": 1067800000, "files": SINGLE_CTA_SOURCES, "kernel_hash": "0d1c02dd776a3318"},
-    # CTA-pair kernel, 8704 window rows: 3.898 GB read + 81.8 MB written per launch (3.9-8.5 GB between captures)
-    "8b_b512": {"bytes": 3980000000, "files": CTA_PAIR_SOURCES, "kernel_hash": "158ceb32802da36d"},
+    # LM-head and decision-head CTAs in one launch, 9 window rows: 1.0642 GB read + 4.9 MB written per launch
+    "8b_b1": {"bytes": 1069100000, "files": SINGLE_CTA_SOURCES, "kernel_hash": "eed3461d3bffc1f3"},
+    # CTA pairs + decision-head clusters, 144 window rows: 1.0829 GB read + 3.8 MB written per launch
+    "8b_b16": {"bytes": 1086800000, "files": CTA_PAIR_SOURCES, "kernel_hash": "26e869a2e0a21f84"},
+    # single-CTA kernel, 576 window rows: 1.0584 GB read + 8.3 MB written per launch
+    "8b_b64": {"bytes": 1066600000, "files": SINGLE_CTA_SOURCES, "kernel_hash": "eed3461d3bffc1f3"},
+    # CTA-pair kernel, 8704 window rows: 3.263 GB read + 72.8 MB written per launch (3.3-8.5 GB between captures)
+    "8b_b512": {"bytes": 3335600000, "files": CTA_PAIR_SOURCES, "kernel_hash": "26e869a2e0a21f84"},
 }
 
 
