@@ -695,3 +695,44 @@ def test_8b_batch512_sampled(name):
         expect = a * (1 - a ** k) / (1 - a)
         var = np.var(A)
         assert abs(A.mean() - expect) < 4 * np.sqrt(var / len(A)) + 0.05
+
+
+def test_random_shapes_under_every_launch_plan():
+    """Seeded sweep over row counts around the plan boundaries (64/65, 128/129, 256/257, 384/385 rows), odd
+    vocabulary, hidden and head sizes, ragged windows, both upload modes and both acceptance rules: every case
+    must match the oracle under the automatic plan, with the GEMMs launched separately, on the single-CTA LM
+    head only, and with an odd number of decision-head CTAs - and all four must agree on argmax and accept_len."""
+    rng = np.random.default_rng(2024)
+    for it in range(40):
+        ragged = rng.random() < 0.3
+        K = int(rng.integers(1, 13))
+        target_rows = int(rng.choice([5, 16, 17, 63, 64, 65, 127, 128, 129, 200, 255, 256, 257, 300, 384, 385, 520]))
+        kw = dict(B=max(1, target_rows // (K + 1)), K=0 if ragged else K, H=int(rng.choice([64, 72, 128, 256])),
+                  H_d=int(rng.choice([8, 40, 64, 128])), d_c=int(rng.choice([0, 2, 3])),
+                  d_J=int(rng.choice([16, 48, 50, 128, 200, 272])),
+                  V=int(rng.choice([17, 31, 100, 600, 1000, 2049, 4096, 5000, 40000])),
+                  match_rate=float(rng.choice([0.0, 0.5, 0.9, 1.0])), seed=3000 + it,
+                  mode=str(rng.choice(["FH", "SH"])), act=str(rng.choice(["gelu", "relu"])),
+                  stochastic=bool(rng.random() < 0.2))
+        if ragged:
+            kw.update(K_lo=1, K_hi=K + 1)
+        cfg = gen.VerifyConfig("rnd", **kw)
+        case = cases.make_case(cfg, oracle_ref_argmax)
+        if cfg.stochastic:
+            base = run_oracle(case)
+            case["draft_q"] = (base["p_draft"] * rng.uniform(0.5, 4.0, size=case["T"])).astype(np.float32)
+        ref = run_oracle(case)
+        d = cases.to_device(case, DEV)
+        v = cases.make_verifier(d)
+        outs = []
+        for tune in (dict(), dict(head_ctas=-1), dict(lm_single_cta=1), dict(head_ctas=3)):
+            v.set_tuning(**tune)
+            cases.run(v, d)
+            out = cases.run(v, d)                       # twice: nothing may linger from the first call
+            torch.cuda.synchronize()
+            assert v.device_error() == 0, (kw, tune)
+            compare(case, ref, out, cfg.tau)
+            outs.append(out)
+        for o in outs[1:]:
+            assert torch.equal(o.argmax, outs[0].argmax) and torch.equal(o.accept_len, outs[0].accept_len), kw
+        v.close()
