@@ -254,6 +254,26 @@ typedef struct {
 } wisv_tuning;
 int wisv_set_tuning(wisv_ctx* ctx, const wisv_tuning* tuning);
 
+/*
+ * The launch planner on its own (host arithmetic only, no CUDA call, no context): the plan wisv_verify would use
+ * for a batch with R window rows and P head positions on a device with sm_count SMs and max_smem_bytes of
+ * opt-in shared memory per block, for the dimensions in cfg (H, V, H_d, d_c, d_J).  For tests and capacity
+ * planning.  *_carry = 1: every CTA (or CTA pair) owns one contiguous range of the weight rows, units_base units
+ * each (the first units_rem one more; a unit is 16 rows, 32 for pairs), cut into tiles_per_cta tiles of at most
+ * tile_n rows.  lm_rounds / lm_rounds_alone: rounds of tiles the slowest CTA works through with and without
+ * decision-head CTAs in the launch (0 when carried ranges are used).
+ */
+typedef struct {
+    int32_t kernels;                 /* kernels per round: 3 or 4 */
+    int32_t head_in_lm_launch;       /* decision-head CTAs ride in the LM-head launch */
+    int32_t lm_pair, lm_carry, lm_tile_n, lm_ctas, lm_m_tiles, lm_n_tiles, lm_stages, lm_smem_bytes;
+    int32_t lm_units_base, lm_units_rem, lm_tiles_per_cta, lm_rounds, lm_rounds_alone;
+    int32_t head_carry, head_tile_n, head_ctas, head_m_tiles, head_n_tiles, head_k_splits, head_kb_per_split;
+    int32_t head_stages, head_smem_bytes, head_units_base, head_units_rem, head_tiles_per_cta;
+} wisv_plan_info;
+int wisv_plan_host(const wisv_config* cfg, int32_t sm_count, int32_t max_smem_bytes, int32_t R, int32_t P,
+                   wisv_plan_info* out);
+
 /* Number of kernels this context has launched so far. */
 int64_t wisv_launch_count(const wisv_ctx* ctx);
 

@@ -74,6 +74,28 @@ def link_cost_round(link: "LinkParams", V: int, K_r: int, m_r: int) -> dict:
     return {n: getattr(out, n) for n, _ in LinkCost._fields_}
 
 
+class PlanInfo(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in (
+        "kernels", "head_in_lm_launch",
+        "lm_pair", "lm_carry", "lm_tile_n", "lm_ctas", "lm_m_tiles", "lm_n_tiles", "lm_stages", "lm_smem_bytes",
+        "lm_units_base", "lm_units_rem", "lm_tiles_per_cta", "lm_rounds", "lm_rounds_alone",
+        "head_carry", "head_tile_n", "head_ctas", "head_m_tiles", "head_n_tiles", "head_k_splits",
+        "head_kb_per_split", "head_stages", "head_smem_bytes", "head_units_base", "head_units_rem",
+        "head_tiles_per_cta")]
+
+
+def plan_host(*, H: int, V: int, H_d: int, d_c: int, d_J: int, R: int, P: int, sm_count: int = 148,
+              max_smem_bytes: int = 232448):
+    """wisv_plan_host: the launch plan for a batch shape on a device of the given size (host arithmetic only)."""
+    cfg = _Config(H, V, H_d, d_c, d_J, ACT_GELU, 0, 0.5, 1, max(R, 1), 0, 0, 0)
+    out = PlanInfo()
+    lib = load_library()
+    lib.wisv_plan_host.restype = C.c_int
+    lib.wisv_plan_host.argtypes = [C.POINTER(_Config), C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(PlanInfo)]
+    _check(lib.wisv_plan_host(C.byref(cfg), sm_count, max_smem_bytes, R, P, C.byref(out)), "wisv_plan_host")
+    return {n: getattr(out, n) for n, _ in PlanInfo._fields_}
+
+
 def choose_protocol(rtt_s: float) -> int:
     return int(load_library().wisv_choose_protocol(float(rtt_s)))
 

@@ -731,6 +731,42 @@ int wisv_plan_kernels(const wisv_ctx* c, int32_t R, int32_t P)
     return P > 0 ? 4 : 3;
 }
 
+int wisv_plan_host(const wisv_config* cfg, int32_t sm_count, int32_t max_smem_bytes, int32_t R, int32_t P,
+                   wisv_plan_info* out)
+{
+    if (!cfg || !out || R < 1 || P < 0 || sm_count < 2 || max_smem_bytes < 64 * 1024) return WISV_EINVAL;
+    if (cfg->H < 8 || cfg->V < 1 || cfg->H_d < 0 || cfg->d_c < 0 || cfg->d_c > kMaxDc || cfg->d_J < 1) return WISV_ESHAPE;
+    wisv_ctx* c = new (std::nothrow) wisv_ctx();       // a plain record here: nothing is allocated on any device
+    if (!c) return WISV_ENOMEM;
+    c->cfg = *cfg;
+    c->sm_count = sm_count;
+    c->max_smem = max_smem_bytes;
+    c->max_pairs = sm_count / 2;
+    memset(out, 0, sizeof *out);
+    Plan a{}, h{};
+    const bool fused = plan_fused(c, R, P, &a, &h);
+    const Plan alone = plan_lm(c, R);
+    if (!fused) {
+        a = alone;
+        if (P > 0) h = plan_head(c, P);
+    }
+    out->kernels = fused ? 3 : (P > 0 ? 4 : 3);
+    out->head_in_lm_launch = fused ? 1 : 0;
+    out->lm_pair = a.pair; out->lm_carry = a.carry; out->lm_tile_n = a.tile_n; out->lm_ctas = a.ctas;
+    out->lm_m_tiles = a.m_tiles; out->lm_n_tiles = a.n_tiles; out->lm_stages = a.stages; out->lm_smem_bytes = (int32_t)a.smem;
+    out->lm_units_base = a.units_base; out->lm_units_rem = a.units_rem; out->lm_tiles_per_cta = a.tiles_per_cta;
+    out->lm_rounds = a.carry ? 0 : (int32_t)plan_waves(a);
+    out->lm_rounds_alone = alone.carry ? 0 : (int32_t)plan_waves(alone);
+    if (P > 0) {
+        out->head_carry = h.carry; out->head_tile_n = h.tile_n; out->head_ctas = h.ctas; out->head_m_tiles = h.m_tiles;
+        out->head_n_tiles = h.n_tiles; out->head_k_splits = h.k_splits; out->head_kb_per_split = h.kb_per_split;
+        out->head_stages = h.stages; out->head_smem_bytes = (int32_t)h.smem;
+        out->head_units_base = h.units_base; out->head_units_rem = h.units_rem; out->head_tiles_per_cta = h.tiles_per_cta;
+    }
+    delete c;
+    return WISV_OK;
+}
+
 int64_t wisv_launch_count(const wisv_ctx* c) { return c ? c->launches : 0; }
 
 int wisv_set_tuning(wisv_ctx* c, const wisv_tuning* t)

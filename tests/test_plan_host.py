@@ -1,0 +1,92 @@
+"""The launch planner as host arithmetic (wisv_plan_host): invariants that must hold for every batch shape,
+vocabulary size and device size, checked without a GPU."""
+import itertools
+
+import pytest
+
+from paper_2604_17701_b200 import plan_host
+
+DIMS_8B = dict(H=4096, V=128256, H_d=2048, d_c=2, d_J=1024)
+SMEM = 232448
+
+
+def _ranges(units_total, ctas, base, rem):
+    """Units owned by each CTA (or pair) of a carried plan."""
+    assert ctas * base + rem == units_total and 0 <= rem < max(ctas, 1)
+    return [base + (1 if c < rem else 0) for c in range(ctas)]
+
+
+def _check_carry(tile_n, tiles_per_cta, owned, unit):
+    assert tile_n % unit == 0 and unit <= tile_n <= 256
+    for u in owned:
+        assert u >= 1                                        # no CTA is launched without work
+        k = tiles_per_cta
+        heights = [(u // k + (1 if i < u % k else 0)) * unit for i in range(k)]
+        assert sum(heights) == u * unit                      # the tiles cover the range exactly once
+        assert all(h in (0, tile_n - unit, tile_n) for h in heights)   # two tile heights (0: fewer units than tiles)
+        assert max(heights) <= tile_n
+
+
+@pytest.mark.parametrize("V", [17, 100, 1000, 4099, 32000, 128256, 152064, 262144])
+@pytest.mark.parametrize("sm_count", [8, 132, 148, 160])
+def test_carried_ranges_cover_the_vocabulary_exactly_once(V, sm_count):
+    for R, P in ((1, 0), (9, 8), (64, 60), (65, 64), (128, 127), (129, 0), (129, 120), (200, 190), (256, 255)):
+        p = plan_host(H=256, V=V, H_d=128, d_c=2, d_J=128, R=R, P=P, sm_count=sm_count, max_smem_bytes=SMEM)
+        assert p["lm_carry"] == 1                            # up to 256 rows: always contiguous ranges
+        unit = 32 if p["lm_pair"] else 16
+        units_total = -(-V // unit)
+        groups = p["lm_ctas"] // 2 if p["lm_pair"] else p["lm_ctas"]
+        owned = _ranges(units_total, groups, p["lm_units_base"], p["lm_units_rem"])
+        _check_carry(p["lm_tile_n"], p["lm_tiles_per_cta"], owned, unit)
+        assert max(owned) - min(owned) <= 1                  # balanced to one unit
+        assert p["lm_smem_bytes"] <= SMEM and p["lm_stages"] >= 2
+        head_ctas = p["head_ctas"] if p["head_in_lm_launch"] else 0
+        assert p["lm_ctas"] + head_ctas + (head_ctas % 2 if p["lm_pair"] else 0) <= sm_count
+        assert p["kernels"] == (3 if (P == 0 or p["head_in_lm_launch"]) else 4)
+        if P > 0:
+            assert p["head_in_lm_launch"] == 1               # small batches never pay for a head launch
+            assert p["head_smem_bytes"] <= SMEM
+            if p["head_carry"]:
+                owned_h = _ranges(-(-128 // 16), p["head_ctas"], p["head_units_base"], p["head_units_rem"])
+                _check_carry(p["head_tile_n"], p["head_tiles_per_cta"], owned_h, 16)
+
+
+def test_plans_at_the_task_shapes():
+    p = plan_host(R=9, P=8, **DIMS_8B)                       # B=1, K=8
+    assert (p["kernels"], p["lm_pair"], p["lm_carry"], p["lm_ctas"], p["head_ctas"]) == (3, 0, 1, 142, 6)
+    assert p["lm_tile_n"] == 240 and p["lm_tiles_per_cta"] == 4 and p["lm_units_base"] == 56
+    p = plan_host(R=144, P=128, **DIMS_8B)                   # B=16: pairs with head clusters
+    assert (p["kernels"], p["lm_pair"], p["lm_carry"], p["lm_ctas"], p["head_ctas"]) == (3, 1, 1, 142, 6)
+    p = plan_host(R=576, P=512, **DIMS_8B)                   # B=64: 16.9 rounds on 148 SMs, nothing to spare
+    assert (p["kernels"], p["lm_pair"], p["lm_ctas"], p["lm_rounds"]) == (4, 0, 148, 17)
+    p = plan_host(R=8704, P=8192, **DIMS_8B)                 # B=512, K=16: 74 pairs, 230.2 rounds
+    assert (p["kernels"], p["lm_pair"], p["lm_ctas"], p["lm_rounds"]) == (4, 1, 148, 231)
+
+
+@pytest.mark.parametrize("R", [257, 288, 384, 385, 432, 504, 576, 640, 864, 1017, 1152, 1408, 2816, 8704])
+def test_head_rides_along_only_when_the_lm_head_needs_no_extra_round(R):
+    for P in (R - R // 9, max(1, R // 3)):
+        p = plan_host(R=R, P=P, **DIMS_8B)
+        assert p["lm_carry"] == 0
+        groups = p["lm_ctas"] // 2 if p["lm_pair"] else p["lm_ctas"]
+        assert p["lm_rounds"] == -(-(p["lm_m_tiles"] * p["lm_n_tiles"]) // groups)
+        if p["head_in_lm_launch"]:
+            assert p["kernels"] == 3 and p["lm_rounds"] == p["lm_rounds_alone"]
+            assert p["lm_ctas"] + p["head_ctas"] + (p["head_ctas"] % 2 if p["lm_pair"] else 0) <= 148
+            head_rounds = -(-(p["head_m_tiles"] * p["head_n_tiles"]) // p["head_ctas"])
+            assert head_rounds * 12 <= p["lm_rounds"] * 8     # the head finishes well inside the LM head's time
+        else:
+            assert p["kernels"] == 4 and p["lm_ctas"] == 148
+        assert p["lm_smem_bytes"] <= SMEM and p["head_smem_bytes"] <= SMEM
+
+
+def test_pairs_for_an_even_number_of_row_tiles_or_many():
+    for R, pair in ((129, 1), (256, 1), (257, 0), (384, 0), (385, 1), (512, 1), (576, 0), (1152, 0), (1281, 1), (1409, 1)):
+        assert plan_host(R=R, P=0, **DIMS_8B)["lm_pair"] == pair, R
+
+
+def test_bad_arguments_are_refused():
+    from paper_2604_17701_b200 import WisvError
+    for kw in (dict(R=0, P=0), dict(R=4, P=-1), dict(R=4, P=2, sm_count=1), dict(R=4, P=2, max_smem_bytes=1024)):
+        with pytest.raises(WisvError):
+            plan_host(**{**DIMS_8B, **kw})
