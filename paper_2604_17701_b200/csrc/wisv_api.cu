@@ -1,8 +1,9 @@
 // Host side of the WISV verifier library: context, argument validation, launch
-// plan and the C ABI declared in include/wisv.h.  One verification round is four
-// stream-ordered launches: pack -> LM-head GEMM+reduce -> decision-head
-// GEMM+reduce -> merge/localize/scan.  Control never returns to the host between
-// them and nothing is synchronised.
+// plan and the C ABI declared in include/wisv.h.  One verification round is three
+// or four stream-ordered launches: pack -> LM-head GEMM+reduce (with the decision
+// head on CTAs of the same launch where the plan allows, else -> decision-head
+// GEMM+reduce) -> merge/localize/scan, chained by programmatic dependent launch.
+// Control never returns to the host between them and nothing is synchronised.
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <math.h>
