@@ -31,6 +31,7 @@ constexpr int kNumTileVariants = kMaxTileN / 16;   // tile_n = 16, 32, ..., 256
 constexpr int kNumRowVariants = kTileM / 8;        // a_rows = 8, 16, ..., 128
 constexpr int kStages = 4;                         // profiled stages per call
 constexpr int kSplitTileN = 64;                    // head tile height when K is split over CTAs
+constexpr int kSplitMaxRowTiles = 4;               // K is split for decision heads of up to this many row tiles
 
 struct Plan {
     int tile_n, m_tiles, n_tiles, ctas, stages;
@@ -170,12 +171,6 @@ void finish_plan(const wisv_ctx* c, Plan* p, int d_c, int k_blocks, int forced_s
     p->smem = fixed + (size_t)s * stage;
 }
 
-double wave_eff(long long tiles, int sms)
-{
-    const long long waves = (tiles + sms - 1) / sms;
-    return (double)tiles / (double)(waves * sms);
-}
-
 // LM head: with a single row tile the kernel streams the weights once and is
 // HBM-bound, so the tile height over the vocabulary is chosen to fill the last
 // wave of CTAs; with many row tiles it is tensor-bound and takes the largest tile.
@@ -266,14 +261,31 @@ Plan plan_head(const wisv_ctx* c, int P)
             p.kb_per_split = (k_blocks + splits - 1) / splits;
             p.k_splits = (k_blocks + p.kb_per_split - 1) / p.kb_per_split;     // no empty split
         }
+    } else if (p.m_tiles <= kSplitMaxRowTiles &&
+               c->sm_count / (p.m_tiles * ((N + kSplitTileN - 1) / kSplitTileN)) >= 2) {
+        // a few row tiles (B=64, K=8: four): still far fewer column tiles than SMs, and every CTA would walk all of
+        // K at the issue-bound pace of narrow tiles, so K is split here too while the work items fit the GPU once
+        best = kSplitTileN;
+        const int nt = (N + best - 1) / best;
+        int splits = c->sm_count / (p.m_tiles * nt);
+        if (splits > k_blocks) splits = k_blocks;
+        if (splits > kMaxKSplits) splits = kMaxKSplits;
+        p.kb_per_split = (k_blocks + splits - 1) / splits;
+        p.k_splits = (k_blocks + p.kb_per_split - 1) / p.kb_per_split;
     } else if (p.m_tiles >= 8) {
         best = kMaxTileN;
     } else {
-        double best_eff = -1.0;
+        // Every work item walks all of K, and below about 200 columns a K block costs the same whatever the tile
+        // width (four MMAs at their issue-bound pace); wider tiles take proportionally longer.  So: fewest rounds
+        // of items first, at equal time the wider tile (fewer re-reads of the activation rows: with six row tiles
+        // one round of 48 items 128 columns wide ran 7 % faster than one round of 96 items 64 wide).
+        double best_cost = 1e30;
         for (int tn = 16; tn <= kMaxTileN; tn *= 2) {
             const long long tiles = (long long)p.m_tiles * ((N + tn - 1) / tn);
-            const double e = wave_eff(tiles, c->sm_count);
-            if (e >= best_eff - 1e-9) { best_eff = e > best_eff ? e : best_eff; best = tn; }
+            const long long rounds = (tiles + c->sm_count - 1) / c->sm_count;
+            const double per_item = tn > 208 ? tn / 208.0 : 1.0;
+            const double cost = (double)rounds * per_item;
+            if (cost <= best_cost + 1e-9) { best_cost = cost; best = tn; }
         }
     }
     if (best > round_up(N, 16)) best = round_up(N, 16);
@@ -667,7 +679,7 @@ int wisv_create(const wisv_config* cfg, const wisv_weights* w, wisv_ctx** out)
         if (cudaMemset(c->done_count, 0, sizeof(int32_t)) != cudaSuccess) { rc = WISV_ECUDA; break; }
         if ((rc = dev_alloc(&c->saved_arg, (size_t)c->rows_alloc))) break;
         if ((rc = dev_alloc(&c->saved_mask, (size_t)cfg->max_requests))) break;
-        c->splitk_tiles = (cfg->d_J + 15) / 16;
+        c->splitk_tiles = kSplitMaxRowTiles * ((cfg->d_J + 15) / 16);
         if ((rc = dev_alloc(&c->splitk_buf, (size_t)c->sm_count * kTileM * kSplitTileN))) break;
         if ((rc = dev_alloc(&c->splitk_count, (size_t)c->splitk_tiles))) break;
         if (cudaMemset(c->splitk_count, 0, sizeof(int32_t) * c->splitk_tiles) != cudaSuccess) { rc = WISV_ECUDA; break; }

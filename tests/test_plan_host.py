@@ -85,6 +85,25 @@ def test_pairs_for_an_even_number_of_row_tiles_or_many():
         assert plan_host(R=R, P=0, **DIMS_8B)["lm_pair"] == pair, R
 
 
+def test_decision_head_in_a_launch_of_its_own():
+    # one row tile of positions: K split over about one work item per SM
+    p = plan_host(R=8 * 9, P=64, **{**DIMS_8B, "V": 128256}, sm_count=148)
+    assert p["head_in_lm_launch"] == 1                        # (small batches ride along; no split there)
+    assert p["head_k_splits"] == 1
+    # four row tiles (B=64, K=8): 64 column tiles of 64, K split in two, 128 work items for 148 SMs
+    p = plan_host(R=576, P=512, **DIMS_8B)
+    assert (p["head_in_lm_launch"], p["head_tile_n"], p["head_m_tiles"], p["head_n_tiles"]) == (0, 64, 4, 16)
+    assert p["head_k_splits"] == 2 and p["head_kb_per_split"] == 48 and p["head_ctas"] == 128
+    assert p["head_k_splits"] * p["head_kb_per_split"] >= 96  # the splits cover all 96 K blocks
+    # six row tiles: no split; one round of 128-wide items rather than three rounds of 16-wide ones
+    p = plan_host(R=864, P=768, **DIMS_8B)
+    assert (p["head_in_lm_launch"], p["head_k_splits"], p["head_tile_n"]) == (0, 1, 128)
+    assert p["head_m_tiles"] * p["head_n_tiles"] <= 148
+    # many row tiles: the widest tiles
+    p = plan_host(R=8704, P=8192, **DIMS_8B)
+    assert (p["head_k_splits"], p["head_tile_n"]) == (1, 256)
+
+
 def test_bad_arguments_are_refused():
     from paper_2604_17701_b200 import WisvError
     for kw in (dict(R=0, P=0), dict(R=4, P=-1), dict(R=4, P=2, sm_count=1), dict(R=4, P=2, max_smem_bytes=1024)):
