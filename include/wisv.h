@@ -210,9 +210,13 @@ int wisv_verify_gathered(wisv_ctx* ctx, const wisv_batch* batch, const wisv_row_
  * array of at most 1 MiB in pinned, 16-byte aligned memory is read in place by
  * the first kernel; otherwise it is copied to a staging buffer owned by the
  * context (allocated on first use).  All other inputs are packed into one
- * pinned block and travel in one copy.  The last kernel writes the requested
- * results into a device-mapped pinned block, from which they are written to
- * the caller's arrays once the stream has been synchronised, before returning.
+ * pinned block, which the kernels read in place when it is at most 8 KB and
+ * which travels in one copy otherwise.  The last kernel writes the requested
+ * results into a device-mapped pinned block and then a completion word; the
+ * call waits for that word (looking at the stream now and then, so a failed
+ * launch or kernel ends the wait with WISV_ECUDA), copies the results to the
+ * caller's arrays and returns: the results are valid on return, the stream may
+ * still be retiring the last kernel.  Not for use during stream capture.
  * One call at a time per context: the staging memory is reused by the next
  * call.  Returns WISV_EDEVICE if a kernel reported a time-out.
  */
