@@ -144,6 +144,10 @@ class ClockSampler:
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.Q,
                                        "--format=csv,noheader,nounits", "-lms", "100"],
                                       stdout=self.f, stderr=subprocess.DEVNULL)
+            # the first sample takes a moment: wait for it (bounded) so that short regions are covered too
+            t0 = time.time()
+            while time.time() - t0 < 3.0 and os.path.getsize(self.f.name) == 0:
+                time.sleep(0.02)
         except Exception:
             self.p = None
 
@@ -258,7 +262,7 @@ def run_reference(args, rank, world):
     if rank != 0:
         return
     import oracle
-    from paper_2604_17701_b200 import cases
+    from gen import cases
     cfg = workload_config(args.workload)
     try:
         import torch
@@ -290,23 +294,105 @@ def run_reference(args, rank, world):
 
 # ------------------------------------------------------------------------------------- CUDA arm
 
-def run_ours(args, rank, world, local_rank):
+NOMINAL_PEAKS = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0}       # HGX B200 data-sheet figures (dense bf16)
+DEFAULT_LEGS = ("8b_b64", "8b_sh256", "8b_b512")                 # tensor-bound configurations of the same 8B model
+SHM_DIR = "/dev/shm"
+
+
+def shared_weights(cfg, rank, ranks):
+    """Model weights of a workload; with several ranks the LM head (1 GB at 8B shapes) is generated once.
+
+    Rank 0 writes it to a file in shared memory named after its shape and seed, the other ranks map that file
+    instead of all regenerating it at once on the same host cores; rank 0 removes the file when the job ends.
+    Returns (weights, path or None).
+    """
+    if ranks.world == 1:
+        return gen.make_weights(cfg), None
+    ws = cfg.weight_seed if cfg.weight_seed >= 0 else cfg.seed
+    path = os.path.join(SHM_DIR, "wisv_lm_head_%dx%d_seed%d_%s.npy" % (cfg.V, cfg.H, ws, os.environ.get("MASTER_PORT", "0")))
+    w = None
+    if rank == 0:
+        w = gen.make_weights(cfg)
+        tmp = path + ".tmp%d" % os.getpid()
+        np.save(tmp, w["lm_head"])
+        os.replace(tmp + ".npy" if not tmp.endswith(".npy") else tmp, path)
+    ranks.barrier()
+    if rank != 0:
+        w = gen.make_weights(cfg, lm_head=np.load(path, mmap_mode="r"))
+    ranks.barrier()
+    return w, (path if rank == 0 else None)
+
+
+def device_weights(w, dev):
     import torch
-    from paper_2604_17701_b200 import cases
+    out = {k: torch.from_numpy(np.ascontiguousarray(w[k]).view(np.int16)).view(torch.bfloat16).to(dev)
+           for k in ("lm_head", "W1")}
+    out.update({k: torch.from_numpy(np.ascontiguousarray(w[k])).to(dev) for k in ("b1", "w2")})
+    return out
 
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the verifier has no CPU path")
-    if local_rank == 0:
-        from paper_2604_17701_b200 import build as cuda_build
-        cuda_build.build()          # compiles the in-tree library only if it is missing or stale
-    torch.cuda.set_device(local_rank)
+
+def region_stats(ms_list):
+    return {"median": float(statistics.median(ms_list)), "min": float(min(ms_list)), "max": float(max(ms_list)),
+            "regions": len(ms_list)}
+
+
+def decision_stats(case, out, cfg):
+    """What the round decided, from the device outputs: accepted lengths, |S| histogram, closed-form mean."""
+    A = out.accept_len.cpu().numpy().astype(np.int64)
+    nm = out.n_mismatch.cpu().numpy().astype(np.int64)
+    d = {"mean_accept_len": float(A.mean()), "accepted_tokens": int(A.sum()),
+         "m_r_histogram": np.bincount(nm, minlength=1).tolist(), "mean_m_r": float(nm.mean())}
+    if cfg.K_hi == 0 and cfg.mode == "FH" and not cfg.stochastic and cfg.B >= 32:
+        # positions are i.i.d. by construction of the synthetic batch: each one lets the window continue with
+        # probability a = 1 - P(candidate and head probability >= tau), so E[A] = a (1 - a^K) / (1 - a)
+        k = cfg.K
+        am = out.argmax.cpu().numpy()
+        rows = np.repeat(case["row_off"][:-1], case["k_len"]) + (np.arange(case["T"]) - np.repeat(case["k_off"][:-1], case["k_len"]))
+        stop = (case["draft_tokens"] != am[rows]) & (out.head_prob.cpu().numpy() >= cfg.tau)
+        a = 1.0 - float(stop.mean())
+        expect = float(k) if a >= 1.0 else a * (1 - a ** k) / (1 - a)
+        sigma = float(A.std() / np.sqrt(len(A)))
+        d["closed_form_accept_len"] = {"per_position_continue_prob": a, "expected": expect, "measured": float(A.mean()),
+                                       "sigma_of_mean": sigma, "within_3_sigma": bool(abs(A.mean() - expect) <= 3 * sigma + 1e-9)}
+    return d
+
+
+def oracle_check(case, out, cfg, rows_budget, seconds, repeat):
+    """The CPU oracle on a bounded sample of whole requests: its rate, and what it says about the device results."""
+    import oracle
+    n_req = oracle_sample_size(case, rows_budget)
+    reqs = pick_requests(case, n_req)
+    sub = subset_case(case, reqs)
+    t0 = time.perf_counter()
+    ref = oracle_round(sub)
+    rounds = 1
+    while repeat and (time.perf_counter() - t0) < seconds and rounds < 200:
+        oracle_round(sub)                               # small workloads: repeat to reach the time budget
+        rounds += 1
+    dt = (time.perf_counter() - t0) / rounds
+    A = out.accept_len.cpu().numpy()[reqs]
+    am = out.argmax.cpu().numpy()
+    row_idx = np.concatenate([np.arange(case["row_off"][b], case["row_off"][b + 1]) for b in reqs])
+    gap = ref["top2_gap"]
+    near = (gap < 1e-2) & (gap > 0)
+    differs = am[row_idx] != ref["argmax"]
+    return {"value": sub["T"] / dt, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "sample": "%d of %d requests (%d window rows, %d draft tokens) per oracle round, %d round(s) of %.2f s"
+                      % (n_req, cfg.B, sub["R"], sub["T"], rounds, dt),
+            "accept_len_equal": int(np.sum(A == ref["accept_len"])), "requests_compared": len(reqs),
+            "rows_compared": int(row_idx.size), "near_tie_rows": int(near.sum()),
+            "argmax_differs_outside_near_ties": int((differs & ~near).sum()),
+            "near_tie_head_probs": int((np.abs(ref["head_prob"] - cfg.tau) < 2e-3).sum())}
+
+
+def measure(cfg, w, wdev, args, rank, world, local_rank, ranks, with_baseline, baseline_repeat):
+    """All timings of one workload on this rank's GPU; rank 0 gets the record (the others None)."""
+    import torch
+    from gen import cases
+
     dev = "cuda:%d" % local_rank
-    ranks = Ranks(world, "nccl", dev)
-    ranks.barrier()                 # the other ranks load the library only after rank 0 has it in place
-
-    cfg = workload_config(args.workload, rank)
-    case = cases.make_case(cfg, lambda w, h: cases.library_ref_argmax(w, h, device=dev))
-    d = cases.to_device(case, dev)
+    case = cases.make_case(cfg, lambda wb, h: cases.library_ref_argmax(wb, h, device=dev), weights=w)
+    d = cases.to_device(case, dev, weights_dev=wdev)
     v = cases.make_verifier(d)
     T, R = case["T"], case["R"]
     P = T if case["sel_pos"] is None else int(case["sel_pos"].shape[0])
@@ -323,37 +409,49 @@ def run_ours(args, rank, world, local_rank):
         ranks.barrier()
         torch.cuda.synchronize()
 
-    max_over_ranks = ranks.max
-
     stream = torch.cuda.current_stream()
+    steps = args.steps
+    fast_out = cases.run(v, d, extras=False)
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def region(fn, n):
+        """n calls of fn between two events on the launching stream, a barrier and a synchronise on both sides."""
+        barrier()
+        e0, e1 = ev(), ev()
+        e0.record(stream)
+        for _ in range(n):
+            fn()
+        e1.record(stream)
+        barrier()
+        return ranks.max(e0.elapsed_time(e1) / n)
+
+    round_fn = lambda: cases.run(v, d, extras=False, out=fast_out)
+    for _ in range(args.warmup):
+        round_fn()
+    est_ms = region(round_fn, min(steps, 5))
+    # every region is exactly `steps` rounds; it is repeated so that the timed regions add up to args.min_seconds
+    repeats = args.repeats if args.repeats > 0 else int(min(400, max(3, np.ceil(args.min_seconds * 1e3 / (steps * est_ms)))))
+
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-
-    # ---- (1) device-resident inputs, K back-to-back rounds, CUDA events on the launching stream
-    fast_out = cases.run(v, d, extras=False)
-    for _ in range(args.warmup):
-        cases.run(v, d, extras=False, out=fast_out)
-    barrier()
+    # ---- (1) device-resident inputs: `repeats` regions of `steps` back-to-back rounds
     n0 = v.launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(args.steps):
-        cases.run(v, d, extras=False, out=fast_out)
-    e1.record(stream)
-    barrier()
-    launches = v.launch_count() - n0
-    ms_step = max_over_ranks(e0.elapsed_time(e1) / args.steps)
+    regions = [region(round_fn, steps) for _ in range(repeats)]
+    launches = (v.launch_count() - n0) // repeats
+    ms_step = float(statistics.median(regions))
+    # ---- (1b) the same number of rounds in ONE region: no idle gaps, the clocks the power cap allows in steady state
+    sustained_ms = region(round_fn, steps * repeats)
 
     # ---- (2) the same rounds with the library's per-kernel events switched on (roofline of the LM head)
-    prof_steps = min(args.steps, 1000)
+    prof_steps = int(min(steps * repeats, 1000))
     v.profile_enable(prof_steps)
     for _ in range(prof_steps):
-        cases.run(v, d, extras=False, out=fast_out)
+        round_fn()
     torch.cuda.synchronize()
     stage_ms = [v.profile_read(s, prof_steps) for s in range(4)]
     v.profile_enable(0)
-    lm_ms = max_over_ranks(float(np.mean(stage_ms[1])))
+    lm_ms = ranks.max(float(np.mean(stage_ms[1])))
     stage_mean = [float(np.mean(s)) if s else 0.0 for s in stage_ms]
 
     # ---- (3) end to end through the host-buffer entry point: H2D + round + D2H + sync per step
@@ -366,22 +464,17 @@ def run_ours(args, rank, world, local_rank):
     # the serving-loop form of the call: the pinned buffers are bound once, every step is one wisv_verify_host on them
     host_call = v.bind_host(hc["target_hidden"], hc["draft_tokens"], hc["draft_hidden"], hc["csi"], **hkw)
     host_out = host_call()
-    e2e_steps = max(3, min(args.steps, 500))
     for _ in range(min(args.warmup, 10)):
         host_call()
-    barrier()
-    e0.record(stream)
-    for _ in range(e2e_steps):
-        host_call()
-    e1.record(stream)
-    barrier()
-    e2e_ms = max_over_ranks(e0.elapsed_time(e1) / e2e_steps)
+    e2e_repeats = max(3, min(repeats, int(np.ceil(0.5 * args.min_seconds * 1e3 / (steps * est_ms)))))
+    e2e_regions = [region(host_call, steps) for _ in range(e2e_repeats)]
+    e2e_ms = float(statistics.median(e2e_regions))
     h2d = sum(int(t.numel() * t.element_size()) for t in list(hc.values()) + [hk] if t is not None)
     d2h = 2 * 4 * cfg.B
     same = bool(torch.equal(host_out.accept_len, fast_out.accept_len.cpu()))
-
     clocks = sampler.stop() if rank == 0 else None
 
+    rec = None
     if rank == 0:
         peaks, peak_kind = load_peaks()
         w_bytes = cfg.V * cfg.H * 2
@@ -394,63 +487,111 @@ def run_ours(args, rank, world, local_rank):
         if hbm_bound:
             achieved = w_bytes / (lm_ms * 1e-3) / 1e9
             peak = float(peaks["hbm_gbs"])
+            # the measured peak is a copy (read + write); a read-only stream can exceed it, so the fraction of the
+            # data-sheet bandwidth is printed beside it
             roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                    "frac_nominal": achieved / NOMINAL_PEAKS["hbm_gbs"], "nominal_peak": NOMINAL_PEAKS["hbm_gbs"],
                     "traffic": captured_traffic(cfg.name)}
         else:
             achieved = flops / (lm_ms * 1e-3) / 1e12
-            long_step = lm_ms > 50.0
-            peak = float(peaks["bf16_tflops_sustained" if long_step else "bf16_tflops"])
+            peak = float(peaks["bf16_tflops"])
+            sus = float(peaks.get("bf16_tflops_sustained", peak))
             roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                    "frac_sustained": achieved / sus, "sustained_peak": sus,
+                    "frac_nominal": achieved / NOMINAL_PEAKS["bf16_tflops"], "nominal_peak": NOMINAL_PEAKS["bf16_tflops"],
                     "traffic": captured_traffic(cfg.name)}
-        # which LM-head kernel the library's plan uses (same rule as the planner: CTA pairs for an even number of
-        # 128-row tiles or at least 11 of them)
-        tiles128 = -(-R // 128)
-        on_pairs = tiles128 >= 2 and (tiles128 % 2 == 0 or tiles128 >= 11)
-        kernel_name = "lmhead_pair_kernel (CTA pairs)" if on_pairs else "gemm_rowreduce_kernel<LM head>"
-        if one_launch:
-            kernel_name = ("lmhead_pair_kernel (CTA pairs + decision-head clusters)" if on_pairs
-                           else "round_small_kernel (LM-head CTAs + decision-head CTAs)")
-        roof.update({"kernel": kernel_name,
-                     "kernel_ms": lm_ms, "peak_source": peak_kind,
+        kernel_name = lm_kernel_name(R, one_launch)
+        roof.update({"kernel": kernel_name, "kernel_ms": lm_ms, "peak_source": peak_kind,
                      "algorithmic_bytes": w_bytes, "algorithmic_flops": flops,
                      "stage_ms": {"pack": stage_mean[0], "lm_head": stage_mean[1], "decision_head": stage_mean[2],
                                   "merge_scan": stage_mean[3]}})
-
-        line = {"metric": METRIC, "value": aggregate(world, T, ms_step), "unit": UNIT, "n_gpus": world,
-                "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                "config": config_block(cfg, case, {"parallelism": "requests sharded, 1 batch per GPU", "plan": plan}),
-                "clocks": clocks, "gpu_launches": int(launches),
-                "e2e": {"value": aggregate(world, T, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                        "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps,
-                        "matches_device_path": same},
-                "roofline": roof,
-                "accepted_tokens_per_s": world * float(fast_out.accept_len.sum().item()) / (ms_step * 1e-3),
-                "mean_accept_len": float(out.accept_len.float().mean().item())}
-
-        if world == 1 and not args.no_cpu_baseline:
-            import oracle
-            n_req = oracle_sample_size(case, args.oracle_rows)
-            reqs = pick_requests(case, n_req)
-            sub = subset_case(case, reqs)
-            t0 = time.perf_counter()
-            ref = oracle_round(sub)
-            dt = time.perf_counter() - t0
-            rounds = 1
-            while (time.perf_counter() - t0) < args.oracle_seconds and rounds < 200:
-                oracle_round(sub)                       # small workloads: repeat to reach the time budget
-                rounds += 1
-            dt = (time.perf_counter() - t0) / rounds
-            A = out.accept_len.cpu().numpy()[reqs]
-            line["cpu_baseline"] = {
-                "value": sub["T"] / dt, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
-                "sample": "%d of %d requests (%d window rows, %d draft tokens) per oracle round, %d round(s) of %.2f s"
-                          % (n_req, cfg.B, sub["R"], sub["T"], rounds, dt),
-                "accept_len_equal": int(np.sum(A == ref["accept_len"])), "requests_compared": len(reqs)}
-        print(json.dumps(line), flush=True)
-
+        mhz = clocks.get("sm_mhz") if clocks else None
+        dec = decision_stats(case, out, cfg)
+        rec = {"value": aggregate(world, T, ms_step), "ms_per_step": ms_step, "steps": steps, "repeats": repeats,
+               "ms_per_step_regions": region_stats(regions),
+               "sustained": {"ms_per_step": sustained_ms, "rounds": steps * repeats,
+                             "value": aggregate(world, T, sustained_ms)},
+               "kcycles_per_step": (ms_step * mhz) if mhz else None,
+               "config": config_block(cfg, case, {"parallelism": "requests sharded, 1 batch per GPU", "plan": plan}),
+               "clocks": clocks, "gpu_launches": int(launches),
+               "e2e": {"value": aggregate(world, T, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                       "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": steps, "repeats": e2e_repeats,
+                       "ms_per_step_regions": region_stats(e2e_regions), "matches_device_path": same},
+               "roofline": roof,
+               "accepted_tokens_per_s": world * dec["accepted_tokens"] / (ms_step * 1e-3),
+               "decisions": dec}
+        if with_baseline:
+            rec["cpu_baseline"] = oracle_check(case, out, cfg, args.oracle_rows if baseline_repeat else args.leg_oracle_rows,
+                                               args.oracle_seconds, baseline_repeat)
     v.close()
+    del d, v, out, fast_out
+    torch.cuda.empty_cache()
+    return rec
+
+
+def lm_kernel_name(R, one_launch):
+    # which LM-head kernel the library's plan uses (same rule as the planner: CTA pairs for an even number of
+    # 128-row tiles or at least 11 of them)
+    tiles128 = -(-R // 128)
+    on_pairs = tiles128 >= 2 and (tiles128 % 2 == 0 or tiles128 >= 11)
+    if one_launch:
+        return ("lmhead_pair_kernel (CTA pairs + decision-head clusters)" if on_pairs
+                else "round_small_kernel (LM-head CTAs + decision-head CTAs)")
+    return "lmhead_pair_kernel (CTA pairs)" if on_pairs else "gemm_rowreduce_kernel<LM head>"
+
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the verifier has no CPU path")
+    if local_rank == 0:
+        from paper_2604_17701_b200 import build as cuda_build
+        cuda_build.build()          # compiles the in-tree library only if it is missing or stale
+    torch.cuda.set_device(local_rank)
+    dev = "cuda:%d" % local_rank
+    ranks = Ranks(world, "nccl", dev)
+    ranks.barrier()                 # the other ranks load the library only after rank 0 has it in place
+
+    cfg = workload_config(args.workload, rank)
+    legs = [n for n in args.legs if n != cfg.name and same_model(gen.config(n), cfg)]
+    w, shm_path = shared_weights(cfg, rank, ranks)
+    wdev = device_weights(w, dev)                       # one upload of the model for the headline and every leg
+    try:
+        head = measure(cfg, w, wdev, args, rank, world, local_rank, ranks, world == 1 and not args.no_cpu_baseline, True)
+        leg_recs = {}
+        for name in legs:
+            lcfg = workload_config(name, rank)
+            largs = argparse.Namespace(**vars(args))
+            rec = measure(lcfg, w, wdev, largs, rank, world, local_rank, ranks,
+                          world == 1 and not args.no_cpu_baseline, False)
+            if rec is not None:
+                rec.update({"metric": METRIC, "unit": UNIT, "dtype": "bf16"})
+                leg_recs[name] = rec
+    finally:
+        if shm_path:
+            try:
+                os.unlink(shm_path)
+            except OSError:
+                pass
+    if rank == 0:
+        line = {"metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic"}
+        line.update({k: v for k, v in head.items() if k not in ("value", "ms_per_step", "steps")})
+        # the accepted-token rate of Table I's "throughput" column needs rounds that accept something: one request at
+        # B = 1 may reject at position 0, so the job-level figures average over the headline batch and the legs
+        allrecs = [head] + list(leg_recs.values())
+        line["mean_accept_len"] = float(np.mean([r["decisions"]["mean_accept_len"] for r in allrecs]))
+        line["accepted_tokens_per_s_by_workload"] = {r["config"]["workload"]: r["accepted_tokens_per_s"] for r in allrecs}
+        if leg_recs:
+            line["legs"] = leg_recs
+        print(json.dumps(line), flush=True)
     ranks.close()
+
+
+def same_model(a, b):
+    return (a.H, a.V, a.H_d, a.d_c, a.d_J, a.weight_seed) == (b.H, b.V, b.H_d, b.d_c, b.d_J, b.weight_seed) and a.weight_seed >= 0
 
 
 def shard_bounds(V, world):
@@ -463,7 +604,7 @@ def shard_bounds(V, world):
 def run_sharded(args, rank, world, local_rank):
     """The same batch on every GPU, the LM head split by vocabulary: shard rows -> all-gather -> merge (strong scaling)."""
     import torch
-    from paper_2604_17701_b200 import cases
+    from gen import cases
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the verifier has no CPU path")
@@ -566,6 +707,15 @@ def main():
     ap.add_argument("--shard", default="requests", choices=["requests", "vocab"],
                     help="multi-GPU split: independent batches per GPU (default), or one batch with the LM head "
                          "sharded by vocabulary")
+    ap.add_argument("--legs", default=None,
+                    help="comma-separated workloads of the same model measured after the headline one and printed under "
+                         "'legs' (default at 1 GPU with the default workload: %s; 'none' switches them off)" % ",".join(DEFAULT_LEGS))
+    ap.add_argument("--repeats", type=int, default=0,
+                    help="timed regions of --steps rounds each (0: as many as add up to --min-seconds, at least 3)")
+    ap.add_argument("--min-seconds", type=float, default=0.6,
+                    help="the timed regions of a workload add up to about this much device time")
+    ap.add_argument("--leg-oracle-rows", type=int, default=96,
+                    help="window rows the oracle checks per leg (one round)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--oracle-seconds", type=float, default=10.0,
                     help="CPU-baseline leg: repeat the oracle round until this much time has passed")
@@ -583,11 +733,17 @@ def main():
         args.oracle_rows = 64 if args.oracle_rows is None else args.oracle_rows
         run_reference(args, rank, world)
     else:
-        big = gen.config(args.workload).B >= 64
-        args.steps = (200 if big else 5000) if args.steps is None else args.steps
-        args.warmup = (5 if big else 50) if args.warmup is None else args.warmup
+        args.steps = 20 if args.steps is None else args.steps
+        args.warmup = 5 if args.warmup is None else args.warmup
         args.warmup = max(3, args.warmup)
         args.oracle_rows = 800 if args.oracle_rows is None else args.oracle_rows
+        if args.legs is None:
+            args.legs = list(DEFAULT_LEGS) if (world == 1 and args.workload == "8b_b1" and args.shard == "requests") else []
+        else:
+            args.legs = [n for n in args.legs.split(",") if n and n != "none"]
+            for n in args.legs:
+                if n not in gen.CONFIGS:
+                    raise SystemExit("unknown leg workload %r" % n)
         if args.shard == "vocab":
             run_sharded(args, rank, world, local_rank)
         else:

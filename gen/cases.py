@@ -1,10 +1,11 @@
-"""Workload assembly shared by the tests, the smoke check and the benchmark.
+"""Workload assembly shared by the tests, the smoke check and the benchmark (harness, not product).
 
-Builds one verification batch from the seeded generators (``gen``), moves it to
-the device and runs it through the binding.  Nothing here computes any part of
-the verification round: the reference argmax that the input recipe needs (draft
+Builds one verification batch from the seeded generators, moves it to the device
+and runs it through the binding of the CUDA library.  Nothing here is part of the
+verification round: the reference argmax that the input recipe needs (draft
 tokens are forced to match the target's prediction with a given probability) is
-passed in by the caller.
+passed in by the caller.  ``gen/__init__`` does not import this module, so the
+generators stay free of the CUDA package.
 """
 from __future__ import annotations
 
@@ -12,18 +13,17 @@ from typing import Callable, Dict, Optional
 
 import numpy as np
 
-import gen
-from . import binding
+from . import synth as gen
 
 
-def make_case(cfg: gen.VerifyConfig, ref_argmax_fn: Callable[[np.ndarray, np.ndarray], np.ndarray],
+def make_case(cfg: "gen.VerifyConfig", ref_argmax_fn: Callable[[np.ndarray, np.ndarray], np.ndarray],
               weights: Optional[Dict[str, np.ndarray]] = None) -> Dict[str, object]:
     """All inputs of one batch as numpy arrays.
 
     ref_argmax_fn(lm_head_bits [V,H], target_hidden [R,H]) -> int32 [R] supplies the
     target's greedy prediction per window row (an oracle or a library routine).
     """
-    k_len = gen.synth.window_lengths(cfg)
+    k_len = gen.window_lengths(cfg)
     k_off, row_off = gen.row_offsets(k_len)
     w = weights if weights is not None else gen.make_weights(cfg)
     h = gen.make_hidden(cfg, k_len)
@@ -66,10 +66,11 @@ def library_ref_argmax(lm_head_bits: np.ndarray, target_hidden: np.ndarray, devi
         torch.backends.cuda.matmul.allow_tf32 = prev
 
 
-ACT = {"relu": binding.ACT_RELU, "gelu": binding.ACT_GELU}
+ACT = {"relu": 0, "gelu": 1}      # WISV_ACT_RELU, WISV_ACT_GELU
 
 
-def to_device(case: Dict[str, object], device="cuda:0") -> Dict[str, object]:
+def to_device(case: Dict[str, object], device="cuda:0", weights_dev=None) -> Dict[str, object]:
+    """The case with every array as a device tensor (weights_dev: model tensors already on the device, reused)."""
     import torch
 
     def dev(a, dtype=None):
@@ -79,9 +80,12 @@ def to_device(case: Dict[str, object], device="cuda:0") -> Dict[str, object]:
         return t.to(device)
 
     d = dict(case)
-    d["lm_head"] = torch.from_numpy(case["lm_head"].view(np.int16)).view(torch.bfloat16).to(device)
-    d["W1"] = torch.from_numpy(case["W1"].view(np.int16)).view(torch.bfloat16).to(device)
-    for k in ("b1", "w2", "target_hidden", "draft_tokens", "draft_hidden", "csi", "sel_off", "sel_pos",
+    if weights_dev is not None:
+        d.update({k: weights_dev[k] for k in ("lm_head", "W1", "b1", "w2")})
+    else:
+        d["lm_head"] = torch.from_numpy(case["lm_head"].view(np.int16)).view(torch.bfloat16).to(device)
+        d["W1"] = torch.from_numpy(case["W1"].view(np.int16)).view(torch.bfloat16).to(device)
+    for k in (("b1", "w2") if weights_dev is None else ()) + ("target_hidden", "draft_tokens", "draft_hidden", "csi", "sel_off", "sel_pos",
               "draft_q", "uniforms"):
         d[k] = dev(case[k])
     cfg = case["cfg"]
@@ -91,7 +95,8 @@ def to_device(case: Dict[str, object], device="cuda:0") -> Dict[str, object]:
 
 def make_verifier(dcase: Dict[str, object], *, act: Optional[str] = None, tau: Optional[float] = None,
                   head_row_shift: int = 0, max_requests: Optional[int] = None, max_rows: Optional[int] = None,
-                  max_sel: int = 0, vocab_slice=None) -> binding.Verifier:
+                  max_sel: int = 0, vocab_slice=None):
+    from paper_2604_17701_b200 import binding
     cfg = dcase["cfg"]
     if vocab_slice is not None:
         # a context on rows [lo, hi) of the LM head (one vocabulary shard)
@@ -107,7 +112,7 @@ def make_verifier(dcase: Dict[str, object], *, act: Optional[str] = None, tau: O
                             max_requests=max_requests or cfg.B, max_rows=max_rows or dcase["R"], max_sel=max_sel)
 
 
-def run(verifier: binding.Verifier, dcase: Dict[str, object], *, tau: Optional[float] = None, extras: bool = True,
+def run(verifier, dcase: Dict[str, object], *, tau: Optional[float] = None, extras: bool = True,
         out=None):
     """One wisv_verify call on a device-resident case."""
     cfg = dcase["cfg"]

@@ -136,15 +136,16 @@ def row_offsets(k_len: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
     return k_off, row_off
 
 
-def make_weights(cfg: VerifyConfig) -> Dict[str, np.ndarray]:
-    """LM head and decision-head parameters.
+def make_weights(cfg: VerifyConfig, lm_head: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
+    """LM head and decision-head parameters (lm_head given: reuse that array instead of drawing it again).
 
     lm_head: bf16 bits [V, H] ~ N(0, 0.02).  W1: bf16 bits [d_J, d_in] with columns
     ordered [h^D | h^T | c] (the order of Eq. 23), each column block drawn from its own
     sub-stream so a different concatenation order is a pure column permutation.
     """
     ws = cfg.weight_seed if cfg.weight_seed >= 0 else cfg.seed
-    lm_head = _normal_bf16(ws, _S_LM_HEAD, (cfg.V, cfg.H), 0.02)
+    if lm_head is None:
+        lm_head = _normal_bf16(ws, _S_LM_HEAD, (cfg.V, cfg.H), 0.02)
     # hidden-state columns ~ N(0, 1/sqrt(d_in)); CSI columns ~ N(0, 1/128) because the CSI
     # features are consumed unnormalised (tens of dB / Mbps) and would otherwise swamp z
     std1 = 1.0 / np.sqrt(cfg.d_in)

@@ -78,6 +78,9 @@ extern "C" {
 #define WISV_ST_BAD_TOKEN      2   /* a draft token id was outside [0, V): clamped */
 #define WISV_ST_NONFINITE      4   /* a non-finite log-sum-exp or head logit was seen */
 #define WISV_ST_BAD_SELECT     8   /* a sel_pos entry was outside [0, K_b): ignored */
+#define WISV_ST_BAD_WINDOW    16   /* k_off gave this request a window outside 0..WISV_MAX_K tokens: only its first
+                                      WISV_MAX_K positions (or none) were verified.  k_off lives on the device, so
+                                      wisv_verify cannot check it; wisv_verify_host does and returns WISV_ESHAPE */
 
 #define WISV_MAX_K   64
 #define WISV_MAX_DC  16
@@ -375,6 +378,18 @@ int wisv_lm_head_reduce_static(const void* lm_head, int32_t V, int32_t H, const 
  * wisv_device_error then reports and clears; the context stays usable.
  */
 int wisv_debug_wait_probe(wisv_ctx* ctx, uint64_t limit_cycles, void* cuda_stream);
+
+/*
+ * Test hooks standing in for a memory checker (no counterpart in the paper): fill every scratch buffer the
+ * context owns - the bf16 copies of the hidden states, the LM-head and decision-head partials, the split-K
+ * scratch, the row and position maps, the state kept between wisv_localize and wisv_decide (a pending localize
+ * is dropped) - with NaN / out-of-range patterns, stream-ordered on `cuda_stream`.  The arrival counters and the
+ * error word keep their values: zero between calls is their documented invariant, not stale data.
+ * A following round must give the same results as without the call: every byte a round reads it has written
+ * itself.  wisv_debug_poison_static does the same to the scratch array of wisv_lm_head_reduce_static.
+ */
+int wisv_debug_poison(wisv_ctx* ctx, void* cuda_stream);
+int wisv_debug_poison_static(void* cuda_stream);
 
 const char* wisv_strerror(int code);
 int wisv_version(void);

@@ -157,6 +157,10 @@ def load_library(build_if_missing: bool = False):
     lib.wisv_plan_kernels.argtypes = [P, C.c_int32, C.c_int32]
     lib.wisv_set_tuning.restype = C.c_int
     lib.wisv_set_tuning.argtypes = [P, C.POINTER(_Tuning)]
+    lib.wisv_debug_poison.restype = C.c_int
+    lib.wisv_debug_poison.argtypes = [P, P]
+    lib.wisv_debug_poison_static.restype = C.c_int
+    lib.wisv_debug_poison_static.argtypes = [P]
     lib.wisv_lm_head_reduce_static.restype = C.c_int
     lib.wisv_lm_head_reduce_static.argtypes = [P, C.c_int32, C.c_int32, P, C.c_int32, P, P, P]
     _lib = lib
@@ -438,6 +442,10 @@ class Verifier:
         st = self._torch.cuda.current_stream(self.device)
         _check(self.lib.wisv_debug_wait_probe(self._h, limit_cycles, C.c_void_p(st.cuda_stream)),
                "wisv_debug_wait_probe")
+
+    def poison(self):
+        st = self._torch.cuda.current_stream(self.device)
+        _check(self.lib.wisv_debug_poison(self._h, C.c_void_p(st.cuda_stream)), "wisv_debug_poison")
 
     def device_error(self) -> int:
         st = self._torch.cuda.current_stream(self.device)

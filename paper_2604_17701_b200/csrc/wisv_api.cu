@@ -526,14 +526,23 @@ PairParams pair_params(const wisv_ctx* c, const Plan& pl, int R)
     return qp;
 }
 
-template <int EPI>
+template <int EPI, bool HEAD_WAITS_LAST = true>
 int launch_gemm(wisv_ctx* c, const CUtensorMap& tA, const CUtensorMap* tB, const GemmParams& gp, const Plan& pl,
                 cudaStream_t st)
 {
-    const int rc = launch_pdl(gemm_rowreduce_kernel<EPI>, dim3(pl.ctas), dim3(kGemmThreads), pl.smem, st, tA,
-                              tB[map_hi(pl)], tB[map_lo(pl)], gp);
+    const int rc = launch_pdl(gemm_rowreduce_kernel<EPI, HEAD_WAITS_LAST>, dim3(pl.ctas), dim3(kGemmThreads), pl.smem,
+                              st, tA, tB[map_hi(pl)], tB[map_lo(pl)], gp);
     if (rc != WISV_OK) return rc;
     c->launches++;
+    return WISV_OK;
+}
+
+// After a reported time-out: clear the error word and the split-K arrival counters (an aborted launch may have left
+// them part-way, and a later round would then take an early item for the last arriver of its tile).
+int reset_after_device_error(wisv_ctx* c)
+{
+    WISV_CUDA(cudaMemset(c->err, 0, sizeof(int32_t)));
+    WISV_CUDA(cudaMemset(c->splitk_count, 0, sizeof(int32_t) * c->splitk_tiles));
     return WISV_OK;
 }
 
@@ -603,6 +612,8 @@ int wisv_create(const wisv_config* cfg, const wisv_weights* w, wisv_ctx** out)
     WISV_CUDA(cudaFuncSetAttribute(gemm_rowreduce_kernel<EPI_LMHEAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)prop.sharedMemPerBlockOptin));
     WISV_CUDA(cudaFuncSetAttribute(gemm_rowreduce_kernel<EPI_HEAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)prop.sharedMemPerBlockOptin));
+    WISV_CUDA(cudaFuncSetAttribute(gemm_rowreduce_kernel<EPI_HEAD, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)prop.sharedMemPerBlockOptin));
     WISV_CUDA(cudaFuncSetAttribute(gemm_rowreduce_kernel<EPI_RAW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)prop.sharedMemPerBlockOptin));
@@ -849,7 +860,7 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
     const int pack_rows = rows_done ? 0 : R;
     pp.vocab_base = cf.vocab_base; pp.vocab_total = cf.vocab_total > 0 ? cf.vocab_total : cf.V;
     pp.ix = ix; pp.R = pack_rows; pp.P = P; pp.H = cf.H; pp.H_d = cf.H_d; pp.V = cf.V; pp.shift = cf.head_row_shift;
-    pp.mode_sh = sh ? 1 : 0;
+    pp.mode_sh = sh ? 1 : 0; pp.R_total = R; pp.T_total = T;
     pp.target_hidden = b->target_hidden; pp.draft_hidden = b->draft_hidden; pp.draft_tokens = b->draft_tokens;
     pp.sel_off = b->sel_off; pp.sel_pos = b->sel_pos;
     pp.X = c->X; pp.Z = c->Z; pp.row_tok = c->row_tok; pp.row_flag = c->row_flag; pp.tok_logit = c->tok_logit;
@@ -925,7 +936,10 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
         GemmParams gp = base_params(c, ph, P, cf.d_J, cf.H_d + cf.H);
         gp.head_part = c->head_part; gp.b1 = c->w.b1; gp.w2 = c->w.w2; gp.w1c = c->W1c; gp.csi = b->csi;
         gp.pos_req = c->pos_req; gp.d_c = cf.d_c; gp.act = cf.act;
-        const int rc = launch_gemm<EPI_HEAD>(c, c->tmZ[ph.a_rows / 8 - 1], c->tmW1, gp, ph, st);
+        // Where an LM-head launch precedes it in this round the head may start early and wait at its end; in the
+        // decide and gathered phases it follows the pack kernel directly and must wait before its first read.
+        const int rc = rows_done ? launch_gemm<EPI_HEAD, false>(c, c->tmZ[ph.a_rows / 8 - 1], c->tmW1, gp, ph, st)
+                                 : launch_gemm<EPI_HEAD, true>(c, c->tmZ[ph.a_rows / 8 - 1], c->tmW1, gp, ph, st);
         if (rc != WISV_OK) return rc;
     }
 
@@ -934,7 +948,7 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
     TailParams tp;
     memset(&tp, 0, sizeof tp);
     tp.ix = ix; tp.P = P; tp.V = cf.V; tp.n_tiles_lm = pl.parts; tp.n_tiles_head = ph.parts; tp.mode_sh = sh ? 1 : 0;
-    tp.phase = phase; tp.saved_arg = c->saved_arg; tp.saved_mask = c->saved_mask;
+    tp.T_total = T; tp.phase = phase; tp.saved_arg = c->saved_arg; tp.saved_mask = c->saved_mask;
     tp.vocab_base = cf.vocab_base; tp.part_rstride = pl.parts; tp.part_nstride = 1;
     tp.stochastic = stoch ? 1 : 0; tp.b2 = c->w.b2; tp.tau = (b->tau != b->tau) ? cf.tau : b->tau;
     tp.lm_part = c->lm_part;
@@ -1008,7 +1022,7 @@ int wisv_debug_logits(wisv_ctx* c, const float* target_hidden, int32_t R, float*
     // rows are cast with the pack kernel, as a batch of R one-row windows without tokens
     PackParams pp;
     memset(&pp, 0, sizeof pp);
-    pp.ix = BatchIndex{R, 0, nullptr}; pp.R = R; pp.P = 0; pp.H = c->cfg.H; pp.H_d = c->cfg.H_d; pp.V = c->cfg.V;
+    pp.ix = BatchIndex{R, 0, nullptr}; pp.R = R; pp.R_total = R; pp.T_total = 0; pp.P = 0; pp.H = c->cfg.H; pp.H_d = c->cfg.H_d; pp.V = c->cfg.V;
     pp.target_hidden = target_hidden; pp.X = c->X; pp.row_tok = c->row_tok; pp.row_flag = c->row_flag;
     pp.tok_logit = c->tok_logit;
     pack_kernel<<<R, 256, 0, st>>>(pp);
@@ -1029,6 +1043,29 @@ int wisv_debug_wait_probe(wisv_ctx* c, uint64_t limit_cycles, void* cuda_stream)
     return WISV_OK;
 }
 
+int wisv_debug_poison(wisv_ctx* c, void* cuda_stream)
+{
+    if (!c) return WISV_EINVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const wisv_config& cf = c->cfg;
+    const size_t hd_h = (size_t)cf.H_d + cf.H;
+    // 0xFF bytes: NaN as bf16 and as fp32; 0x7F bytes: 0x7F7F7F7F as int32 (no valid token, row or request)
+    WISV_CUDA(cudaMemsetAsync(c->X, 0xFF, (size_t)c->rows_alloc * cf.H * 2, st));
+    WISV_CUDA(cudaMemsetAsync(c->Z, 0xFF, (size_t)c->pos_alloc * hd_h * 2, st));
+    WISV_CUDA(cudaMemsetAsync(c->lm_part, 0xFF, c->lm_part_elems * sizeof(float4), st));
+    WISV_CUDA(cudaMemsetAsync(c->head_part, 0xFF, c->head_part_elems * sizeof(float), st));
+    WISV_CUDA(cudaMemsetAsync(c->splitk_buf, 0xFF, (size_t)c->sm_count * kTileM * kSplitTileN * sizeof(float), st));
+    WISV_CUDA(cudaMemsetAsync(c->tok_logit, 0xFF, (size_t)c->rows_alloc * sizeof(float), st));
+    WISV_CUDA(cudaMemsetAsync(c->row_tok, 0x7F, (size_t)c->rows_alloc * sizeof(int32_t), st));
+    WISV_CUDA(cudaMemsetAsync(c->row_flag, 0x7F, (size_t)c->rows_alloc * sizeof(int32_t), st));
+    WISV_CUDA(cudaMemsetAsync(c->pos_req, 0x7F, (size_t)c->pos_alloc * sizeof(int32_t), st));
+    WISV_CUDA(cudaMemsetAsync(c->pos_i, 0x7F, (size_t)c->pos_alloc * sizeof(int32_t), st));
+    WISV_CUDA(cudaMemsetAsync(c->saved_arg, 0x7F, (size_t)c->rows_alloc * sizeof(int32_t), st));
+    WISV_CUDA(cudaMemsetAsync(c->saved_mask, 0xFF, (size_t)cf.max_requests * sizeof(unsigned long long), st));
+    c->loc_valid = false;
+    return WISV_OK;
+}
+
 int wisv_device_error(wisv_ctx* c, void* cuda_stream, int32_t* flags)
 {
     if (!c || !flags) return WISV_EINVAL;
@@ -1037,9 +1074,8 @@ int wisv_device_error(wisv_ctx* c, void* cuda_stream, int32_t* flags)
     int32_t v = 0;
     WISV_CUDA(cudaMemcpy(&v, c->err, sizeof v, cudaMemcpyDeviceToHost));
     if (v != 0) {
-        // an aborted launch may have left split-K arrival counters half-way
-        WISV_CUDA(cudaMemset(c->err, 0, sizeof v));
-        WISV_CUDA(cudaMemset(c->splitk_count, 0, sizeof(int32_t) * c->splitk_tiles));
+        const int rc = reset_after_device_error(c);
+        if (rc != WISV_OK) return rc;
     }
     *flags = v;
     return WISV_OK;
@@ -1163,6 +1199,14 @@ int wisv_verify_host(wisv_ctx* c, const wisv_batch* hb, const wisv_result* hr, v
     if (vrc != WISV_OK) return vrc;
     if (!fits) return WISV_ESHAPE;
     if (B == 0) return WISV_OK;
+    if (hb->k_off) {
+        // here the row offsets are host memory: check what wisv_verify has to leave to the device's status bits
+        if (hb->k_off[0] != 0 || hb->k_off[B] != T) return WISV_ESHAPE;
+        for (int i = 0; i < B; ++i) {
+            const long long kb = (long long)hb->k_off[i + 1] - hb->k_off[i];
+            if (kb < 0 || kb > WISV_MAX_K) return WISV_ESHAPE;
+        }
+    }
     for (int i = 0; i < IN_FIELDS; ++i)
         if (src[i] && ibytes[i] > 0) memcpy(pin_in + ioff[i], src[i], ibytes[i]);
     if (!small_in_place) WISV_CUDA(cudaMemcpyAsync(h.dev_in, pin_in, in_used, cudaMemcpyHostToDevice, st));
@@ -1198,7 +1242,12 @@ int wisv_verify_host(wisv_ctx* c, const wisv_batch* hb, const wisv_result* hr, v
     __atomic_thread_fence(__ATOMIC_ACQUIRE);
     int32_t dev_err = 0;
     memcpy(&dev_err, pin_out, sizeof dev_err);
-    if (dev_err != 0) { (void)cudaMemset(c->err, 0, sizeof dev_err); return WISV_EDEVICE; }
+    if (dev_err != 0) {
+        // the stream has to be idle before the counters are cleared: the round's kernels may still be retiring
+        if (cudaStreamSynchronize(st) != cudaSuccess) { (void)cudaGetLastError(); return WISV_ECUDA; }
+        (void)reset_after_device_error(c);
+        return WISV_EDEVICE;
+    }
     const uint8_t* po = pin_out + 16;
     void* dst[OUT_FIELDS] = {hr->accept_len, hr->correction_token, hr->argmax, hr->lse, hr->p_draft,
                              hr->head_prob, hr->mismatch_mask, hr->n_mismatch, hr->status};

@@ -39,6 +39,7 @@ struct BatchIndex {
 struct PackParams {
     BatchIndex ix;
     int32_t R, P, H, H_d, V, shift, mode_sh;
+    int32_t R_total, T_total;     // window rows and draft tokens of the batch (bounds for indices derived from k_off)
     int32_t vocab_base, vocab_total;   // this context's LM-head rows are tokens [vocab_base, vocab_base + V) of vocab_total
     const float* target_hidden;   // [R, H]
     const float* draft_hidden;    // [P, H_d]
@@ -98,8 +99,9 @@ __global__ void __launch_bounds__(256) pack_kernel(const PackParams p)
             const int i = r - p.ix.roff(b);
             const int Kb = p.ix.koff(b + 1) - p.ix.koff(b);
             int tok = -1, flag = 0;
-            if (i < Kb) {
-                tok = p.draft_tokens[p.ix.koff(b) + i];
+            const int t = p.ix.koff(b) + i;
+            if (i >= 0 && i < Kb && t >= 0 && t < p.T_total) {       // (the last two only fail on a corrupt k_off)
+                tok = p.draft_tokens[t];
                 if (tok < 0 || tok >= p.vocab_total) { flag = 2; tok = tok < 0 ? 0 : p.vocab_total - 1; }
                 tok -= p.vocab_base;                       // row index in this context's LM head
                 if (tok < 0 || tok >= p.V) tok = -1;       // another shard owns the token
@@ -126,7 +128,7 @@ __global__ void __launch_bounds__(256) pack_kernel(const PackParams p)
             const bool good = (i >= 0 && i < Kb);
             p.pos_req[j] = b;
             p.pos_i[j] = good ? i : -1;
-            s_src_row = p.ix.roff(b) + (good ? i + p.shift : 0);
+            s_src_row = max(0, min(p.ix.roff(b) + (good ? i + p.shift : 0), p.R_total - 1));
         }
         __syncthreads();
         const size_t zw = (size_t)(p.H_d + p.H);
@@ -148,6 +150,7 @@ __global__ void split_w1_kernel(const __nv_bfloat16* __restrict__ W1, __nv_bfloa
 struct TailParams {
     BatchIndex ix;
     int32_t P, V, n_tiles_lm, n_tiles_head, mode_sh, stochastic;
+    int32_t T_total;              // draft tokens of the batch
     int32_t phase;                // 0: whole round; 1: localize only (no head); 2: decide from a saved localize;
                                   // 3: whole round on per-shard row partials gathered from G vocabulary shards
     int32_t vocab_base;           // added to the argidx of per-tile partials (phases 0 and 1)
@@ -214,8 +217,13 @@ __global__ void __launch_bounds__(1024) tail_kernel(const TailParams p)
     // partials of the LM-head and decision-head kernels must be complete and visible
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    const int k0 = p.ix.koff(b);
-    const int Kb = min(p.ix.koff(b + 1) - k0, kMaxK);
+    // A window outside 0..64 tokens, or offsets outside 0..T, can only come from a device-side k_off the host never
+    // saw: the window is cut to what is in range (the scan covers at most 64 positions) and the request's status
+    // word says so.
+    const int k0_raw = p.ix.koff(b);
+    const int k0 = max(0, min(k0_raw, p.T_total));
+    const int Kb_raw = p.ix.koff(b + 1) - k0_raw;
+    const int Kb = max(0, min(min(Kb_raw, kMaxK), p.T_total - k0));
     const int r0 = k0 + b;
 
     if (p.err_copy && b == 0 && threadIdx.x == 0) *p.err_copy = *p.err_src;
@@ -363,7 +371,7 @@ __global__ void __launch_bounds__(1024) tail_kernel(const TailParams p)
             if (p.phase == 1) p.saved_mask[b] = cnd;
             if (p.mismatch_mask) p.mismatch_mask[b] = cnd;
             if (p.n_mismatch) p.n_mismatch[b] = __popcll(cnd);
-            if (p.status) p.status[b] = s_flag | (missing ? 1 : 0);
+            if (p.status) p.status[b] = s_flag | (missing ? 1 : 0) | ((Kb != Kb_raw || k0 != k0_raw) ? 16 : 0);
         }
     }
     if (p.done_flag) {

@@ -32,7 +32,7 @@ constexpr int kTmemCols = 512;
 constexpr int kGemmThreads = 192;
 constexpr int kEpiThreads = 128;
 constexpr int kMaxStages = 32;
-constexpr uint64_t kWaitLimitNs = 4000000000ull;   // SM clocks: 2 s at 2 GHz, 3.3 s at 1.2 GHz
+constexpr uint64_t kWaitLimitClocks = 4000000000ull;   // SM clocks: 2 s at 2 GHz, 3.3 s at 1.2 GHz
 constexpr int kMaxDc = 16;
 constexpr int kMaxKSplits = 16;      // split-K work items per tile (their partial loads are issued together)
 
@@ -262,7 +262,7 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
                         // first pass over the ring: the stage is free and its weight tile is already on its way
                         tma_load_2d(a_dst, &tmA, kb * kBlockK, w.m * kTileM, full_bar(s));
                     } else {
-                        if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, kWaitLimitNs)) { ok = false; break; }
+                        if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, kWaitLimitClocks)) { ok = false; break; }
                         mbar_expect_tx(full_bar(s), tx);
                         tma_load_2d(a_dst, &tmA, kb * kBlockK, w.m * kTileM, full_bar(s));
                         tma_load_2d(a_dst + a_bytes, b_map(w.h), kb * kBlockK, w.n0, full_bar(s));
@@ -278,7 +278,7 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
                 uint32_t wph = ph;
                 for (int i = 0; i < inflight; ++i) {
                     if (--ws < 0) { ws = p.stages - 1; wph ^= 1u; }
-                    mbar_wait_bounded(full_bar(ws), wph, abort_flag + 1, kWaitLimitNs);
+                    mbar_wait_bounded(full_bar(ws), wph, abort_flag + 1, kWaitLimitClocks);
                 }
             }
         }
@@ -293,12 +293,12 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
                 const uint32_t idesc = idesc_bf16_f32(static_cast<uint32_t>(tile_mma_m(w.m)), static_cast<uint32_t>(w.h));
                 const int as = local & 1;
                 const uint32_t aph = (local >> 1) & 1u;
-                if (!mbar_wait_bounded(acc_empty_bar(as), aph ^ 1u, abort_flag, kWaitLimitNs)) { ok = false; break; }
+                if (!mbar_wait_bounded(acc_empty_bar(as), aph ^ 1u, abort_flag, kWaitLimitClocks)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(as * kAccCols);
                 const int kb0 = w.kb0, kb1 = w.kb1;
                 for (int kb = kb0; kb < kb1; ++kb) {
-                    if (!mbar_wait_bounded(full_bar(s), ph, abort_flag, kWaitLimitNs)) { ok = false; break; }
+                    if (!mbar_wait_bounded(full_bar(s), ph, abort_flag, kWaitLimitClocks)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_addr = smem_base + stage_bytes * s;
                     const uint64_t a_desc = smem_desc_k128(a_addr);
@@ -316,7 +316,7 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
             if (!ok) {
                 // drain whatever was issued before TMEM is released
                 umma_commit(drain_bar);
-                mbar_wait_bounded(drain_bar, 0, abort_flag + 1, kWaitLimitNs);
+                mbar_wait_bounded(drain_bar, 0, abort_flag + 1, kWaitLimitClocks);
             }
         }
     } else {
@@ -354,15 +354,16 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
                     for (int c = 0; c < p.d_c; ++c)
                         wwc[c * p.tile_n + j] = in ? p.w1c[(size_t)(n0 + j) * p.d_c + c] : 0.0f;
                 }
-                const int rq = valid ? p.pos_req[row] : 0;
+                // (read through L2: a late-waiting head kernel may share an SM, and its L1, with earlier rounds)
+                const int rq = valid ? __ldcg(p.pos_req + row) : 0;
                 // indexed by row within the tile (this thread's TMEM lane), not by thread number
                 if (lane_used)
                     for (int c = 0; c < p.d_c; ++c)
-                        wcs[c * kEpiThreads + rit] = valid ? p.csi[(size_t)rq * p.d_c + c] : 0.0f;
+                        wcs[c * kEpiThreads + rit] = valid ? __ldcg(p.csi + (size_t)rq * p.d_c + c) : 0.0f;
                 cb1 = wb1; cw2 = ww2; cwc = wwc; ccs = wcs;
             }
 
-            bool got = mbar_wait_bounded(acc_full_bar(as), aph, abort_flag, kWaitLimitNs);
+            bool got = mbar_wait_bounded(acc_full_bar(as), aph, abort_flag, kWaitLimitClocks);
             if (EPI == EPI_HEAD) {
                 // barrier over the 128 epilogue threads that also agrees on `got`
                 uint32_t all;
@@ -509,12 +510,16 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
     if (threadIdx.x == 0 && (abort_flag[0] != 0)) atomicOr(p.err, 1);
 }
 
-template <int EPI>
+// HEAD_WAITS_LAST (decision-head epilogue only): true when an LM-head launch that waited for the pack kernel sits
+// between the pack kernel and this launch in the stream; false when this launch follows the pack kernel directly
+// (the decide and gathered phases), where the head must wait before its first read like every other consumer.
+template <int EPI, bool HEAD_WAITS_LAST = true>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_rowreduce_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                       const __grid_constant__ CUtensorMap tmB2, const GemmParams p)
 {
-    gemm_rowreduce_body<EPI, true>(tmA, tmB, tmB2, p, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x));
+    gemm_rowreduce_body<EPI, HEAD_WAITS_LAST>(tmA, tmB, tmB2, p, static_cast<int>(blockIdx.x),
+                                              static_cast<int>(gridDim.x));
 }
 
 // One row tile of window rows and one of head positions (small batches, where the LM head streams the

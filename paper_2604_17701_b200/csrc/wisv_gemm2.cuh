@@ -147,12 +147,17 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         griddep_launch_dependents();
     }
 
+    // producer thread only: ring position and stages issued so far (read again by the drain before the kernel ends)
+    int prod_s = 0;
+    uint32_t prod_ph = 0;
+    long long prod_issued = 0;
+
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (each CTA)
         if (lane == 0) {
-            int s = 0;
-            uint32_t ph = 0;
-            long long issued = 0;
+            int& s = prod_s;
+            uint32_t& ph = prod_ph;
+            long long& issued = prod_issued;
             bool ok = true;
             PTile w;
             long long pre = 0;                 // stages whose weight half-tile was requested before the wait
@@ -182,7 +187,7 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                         // half-tile is already on its way
                         tma_load_2d_pair(a_dst, &tmA, kb * kBlockK, row0, full_bar(s));
                     } else {
-                        if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, kWaitLimitNs)) { ok = false; break; }
+                        if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, kWaitLimitClocks)) { ok = false; break; }
                         if (leader) mbar_expect_tx(full_bar(s), tx);             // both CTAs' bytes
                         tma_load_2d_pair(a_dst, &tmA, kb * kBlockK, row0, full_bar(s));
                         tma_load_2d_pair(a_dst + half_bytes, mapB, kb * kBlockK, col0, full_bar(s));
@@ -203,11 +208,11 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 const uint32_t idesc = idesc_bf16_f32(kPairTileM, static_cast<uint32_t>(w.h));
                 const int as = local & 1;
                 const uint32_t aph = (local >> 1) & 1u;
-                if (!mbar_wait_bounded(acc_empty_bar(as), aph ^ 1u, abort_flag, kWaitLimitNs)) { ok = false; break; }
+                if (!mbar_wait_bounded(acc_empty_bar(as), aph ^ 1u, abort_flag, kWaitLimitClocks)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(as * kAccCols);
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
-                    if (!mbar_wait_bounded(full_bar(s), ph, abort_flag, kWaitLimitNs)) { ok = false; break; }
+                    if (!mbar_wait_bounded(full_bar(s), ph, abort_flag, kWaitLimitClocks)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_addr = smem_base + kPairStageBytes * s;
                     const uint64_t a_desc = smem_desc_k128(a_addr);
@@ -222,7 +227,7 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             }
             if (!ok) {
                 umma_commit_pair(drain_bar);
-                mbar_wait_bounded(drain_bar, 0, abort_flag + 1, kWaitLimitNs);
+                mbar_wait_bounded(drain_bar, 0, abort_flag + 1, kWaitLimitClocks);
             }
         }
     } else {
@@ -242,7 +247,7 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             const bool valid = row < p.rows;
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(as * kAccCols);
 
-            bool got = mbar_wait_bounded(acc_full_bar(as), aph, abort_flag, kWaitLimitNs);
+            bool got = mbar_wait_bounded(acc_full_bar(as), aph, abort_flag, kWaitLimitClocks);
             got = __all_sync(0xffffffffu, got);
             if (!got) { ok = false; break; }
             tc_fence_after();
@@ -270,6 +275,19 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             p.lm_part[(size_t)last_row * p.part_stride + pair_id] = make_float4(mx, __int_as_float(arg), sum, 0.0f);
     }
 
+    // After a time-out copies may still be heading for the shared memory of either CTA.  Their bytes are counted on
+    // the leader's full barriers, so the leader's producer thread waits (bounded) for the stages it issued last
+    // before it arrives at the closing cluster barrier, which in turn keeps the partner from retiring earlier.
+    __syncthreads();
+    if (leader && producer_thread && abort_flag[0] != 0) {
+        const int inflight = prod_issued < p.stages ? static_cast<int>(prod_issued) : p.stages;
+        int ws = prod_s;
+        uint32_t wph = prod_ph;
+        for (int i = 0; i < inflight; ++i) {
+            if (--ws < 0) { ws = p.stages - 1; wph ^= 1u; }
+            mbar_wait_bounded(full_bar(ws), wph, abort_flag + 1, kWaitLimitClocks);
+        }
+    }
     // neither CTA may retire (or release TMEM) while its partner can still signal or read it
     tc_fence_before();
     __syncwarp();

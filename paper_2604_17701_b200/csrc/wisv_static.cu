@@ -222,3 +222,17 @@ extern "C" int wisv_lm_head_reduce_static(const void* lm_head, int32_t V, int32_
     if (cudaGetLastError() != cudaSuccess) return WISV_ECUDA;
     return WISV_OK;
 }
+
+extern "C" int wisv_debug_poison_static(void* cuda_stream)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return WISV_ECUDA; }
+    DeviceSetup* s = nullptr;
+    const int src = setup_device(dev, &s);
+    if (src != WISV_OK) return src;
+    if (cudaMemsetAsync(s->scratch, 0xFF, kScratchBytes, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return WISV_ECUDA;
+    }
+    return WISV_OK;
+}

@@ -2,8 +2,12 @@
 
 Bars: argmax / accept_len / correction_token bit-exact outside near-ties (top-2
 logit gap < 1e-2, |head prob - tau| < 2e-3, and for the stochastic test
-|u - alpha| < 1e-2), which are excluded and counted; log-sum-exp within 1e-2
-absolute; decision-head probabilities within 2e-3 absolute; the draft-token
+|u - alpha| < 1e-2), which are excluded from the exact comparison and counted;
+on a near-tie row several indices are correct, so the CUDA argmax is still
+checked for validity: the oracle's logit at that index must lie within 1e-2 of
+the oracle's maximum, and where the oracle's gap is exactly zero (duplicate
+vocabulary rows) the lowest index is required bit-exactly.  Log-sum-exp within
+1e-2 absolute; decision-head probabilities within 2e-3 absolute; the draft-token
 probability within 2 % relative (it inherits the log-sum-exp tolerance).
 """
 import numpy as np
@@ -46,13 +50,26 @@ def compare(case, ref, out, tau, requests=None):
     B = k_len.shape[0]
     k_off, row_off = ref["k_off"], ref["row_off"]
     gap = ref["top2_gap"]
-    row_tie = gap < GAP_TIE
+    # a gap of exactly zero means bit-identical weight rows: both sides see equal logits and the lowest index is
+    # the one correct answer, so such rows are compared exactly like any other
+    row_tie = (gap < GAP_TIE) & (gap > 0.0)
 
     # per-row quantities
     assert np.max(np.abs(g["lse"] - ref["lse"])) <= LSE_TOL, "log-sum-exp outside tolerance"
-    bad = (g["argmax"] != ref["argmax"]) & ~row_tie
+    differs = g["argmax"] != ref["argmax"]
+    bad = differs & ~row_tie
     assert not bad.any(), "argmax differs on rows %s (gaps %s)" % (np.nonzero(bad)[0][:8], gap[bad][:8])
-    # near-tie rows must still pick one of the two leading logits' neighbourhood: lse equality covers the value
+    # near-tie rows: any index whose oracle logit is within the band of the oracle maximum is valid
+    near = np.nonzero(differs & row_tie)[0]
+    if near.size:
+        V = np.asarray(case["lm_head"]).shape[0]
+        assert np.all((g["argmax"][near] >= 0) & (g["argmax"][near] < V)), "argmax out of range on a near-tie row"
+        rows2 = np.concatenate([near, near])
+        toks2 = np.concatenate([g["argmax"][near], ref["argmax"][near]]).astype(np.int32)
+        at = oracle.lm_head(case["lm_head"], np.asarray(case["target_hidden"])[rows2], row_token=toks2)["tok_logit"]
+        short = at[near.size:] - at[:near.size]            # oracle maximum minus oracle logit at the GPU's index
+        assert np.all(short >= 0.0) and np.all(short < GAP_TIE), \
+            "near-tie rows %s: GPU argmax is not among the leading logits (short by %s)" % (near[:8], short[:8])
     rel = np.abs(g["p_draft"] - ref["p_draft"]) / np.maximum(ref["p_draft"], 1e-30)
     assert np.all(rel <= 2e-2), "draft-token probability outside tolerance"
     assert np.max(np.abs(g["head_prob"] - ref["head_prob"]), initial=0.0) <= PROB_TOL, "head probability outside tolerance"
@@ -84,5 +101,5 @@ def compare(case, ref, out, tau, requests=None):
             assert g["n_mismatch"][b] == ref["n_mismatch"][b]
             mask = sum(1 << i for i in range(k_len[b]) if ref["cand"][k_off[b] + i])
             assert int(g["mismatch_mask"][b]) & ((1 << 64) - 1) == mask or int(g["mismatch_mask"][b]) == mask - (1 << 64)
-    return dict(row_ties=int(row_tie.sum()), rows=int(row_tie.shape[0]), tainted_requests=tainted, requests=B,
+    return dict(row_ties=int(row_tie.sum()), near_tie_rows_checked=int(near.size), rows=int(row_tie.shape[0]), tainted_requests=tainted, requests=B,
                 prob_ties=int(prob_tie_t.sum()), alpha_ties=int(alpha_tie_t.sum()))

@@ -92,3 +92,36 @@ def test_row_partials_are_gathered_rank_major_with_two_gloo_ranks(tmp_path):
     assert out.returncode == 0, out.stderr[-2000:]
     recs = [json.loads(l) for l in out.stdout.splitlines() if l.startswith("{")]
     assert len(recs) == 2 and all(r["ok"] and r["shape"] == [2, 5, 4] for r in recs)
+
+
+def test_model_weights_are_generated_once_and_shared_between_two_gloo_ranks(tmp_path):
+    """With several ranks rank 0 draws the LM head once and the others map its file; all ranks end up with the same
+    model, the batches still differ, and the file is gone after the job."""
+    script = tmp_path / "weights.py"
+    script.write_text(textwrap.dedent("""
+        import hashlib, json, os, sys
+        sys.path.insert(0, %r)
+        import numpy as np
+        import bench, gen
+        bench.SHM_DIR = %r
+        rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+        r = bench.Ranks(world, backend="gloo")
+        cfg = bench.workload_config("tiny", rank)
+        w, path = bench.shared_weights(cfg, rank, r)
+        same = all(np.array_equal(np.asarray(w[k]), gen.make_weights(cfg)[k]) for k in ("lm_head", "W1", "b1", "w2"))
+        rec = {"rank": rank, "same": bool(same), "owner": path is not None,
+               "mapped": isinstance(w["lm_head"], np.memmap), "files": sorted(os.listdir(%r))}
+        r.barrier()
+        if path:
+            os.unlink(path)
+        os.write(1, (json.dumps(rec) + chr(10)).encode())
+        r.close()
+    """ % (ROOT, str(tmp_path / "shm"), str(tmp_path / "shm"))))
+    (tmp_path / "shm").mkdir()
+    out = _torchrun(2, [str(script)])
+    assert out.returncode == 0, out.stderr[-2000:]
+    recs = sorted((json.loads(l) for l in out.stdout.splitlines() if l.startswith("{")), key=lambda r: r["rank"])
+    assert [r["rank"] for r in recs] == [0, 1] and all(r["same"] for r in recs)
+    assert recs[0]["owner"] and not recs[1]["owner"] and recs[1]["mapped"] and not recs[0]["mapped"]
+    assert all(len(r["files"]) == 1 and r["files"][0].endswith(".npy") for r in recs)
+    assert os.listdir(tmp_path / "shm") == []

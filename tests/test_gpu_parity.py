@@ -7,7 +7,7 @@ import torch
 
 import gen
 import oracle
-from paper_2604_17701_b200 import cases
+from gen import cases
 from parity import compare, oracle_ref_argmax, run_oracle
 
 pytestmark = pytest.mark.gpu
@@ -532,6 +532,54 @@ def test_host_entry_point_with_selective_upload_and_sampling_test():
     for k in ("accept_len", "correction_token", "argmax", "lse", "p_draft", "head_prob", "n_mismatch", "status"):
         assert torch.equal(getattr(ho, k), getattr(out, k).cpu()), k
     compare(case, run_oracle(case), out, cfg.tau)
+    v.close()
+
+
+def test_window_longer_than_the_limit_in_device_offsets_is_cut_and_flagged():
+    """k_off lives on the device, so wisv_verify cannot see a window of more than 64 tokens: the device verifies its
+    first 64 positions and says so in the request's status word; the other requests are untouched.  With host
+    buffers the library sees the offsets and refuses the batch."""
+    cfg = _small(B=4, K=0, K_lo=3, K_hi=9, seed=61, V=1000)
+    k_len = np.array([5, 70, 3, 9], np.int32)                       # request 1 is too long; T = 87 <= 64 * B
+    k_off, row_off = gen.row_offsets(k_len)
+    w = _shared_weights(cfg)
+    T, R = int(k_off[-1]), int(row_off[-1])
+    g = np.random.default_rng(61)
+    ht = g.standard_normal((R, cfg.H), dtype=np.float32)
+    hd = g.standard_normal((T, cfg.H_d), dtype=np.float32)
+    csi = g.uniform(1.0, 30.0, size=(cfg.B, cfg.d_c)).astype(np.float32)
+    ref_am = oracle_ref_argmax(w["lm_head"], ht)
+    rows = np.concatenate([row_off[b] + np.arange(k_len[b]) for b in range(cfg.B)])
+    toks = np.where(g.random(T) < 0.8, ref_am[rows], g.integers(0, cfg.V, size=T)).astype(np.int32)
+    case = dict(cfg=cfg, k_len=k_len, k_off=k_off, row_off=row_off, T=T, R=R, draft_tokens=toks, target_hidden=ht,
+                csi=csi, draft_hidden=hd, sel_off=None, sel_pos=None, draft_q=None, uniforms=None, **w)
+    d = cases.to_device(case, DEV)
+    v = cases.make_verifier(d, max_requests=cfg.B, max_rows=R)
+    out = cases.run(v, d)
+    torch.cuda.synchronize()
+    assert v.device_error() == 0
+    st = out.status.cpu().numpy()
+    assert st[1] & 16 and not any(st[b] & 16 for b in (0, 2, 3))
+    ref = run_oracle(case)                                          # the oracle has no window limit
+    A, corr = out.accept_len.cpu().numpy(), out.correction_token.cpu().numpy()
+    tie = ref["top2_gap"] < 1e-2
+    ptie = np.abs(ref["head_prob"] - cfg.tau) < 2e-3
+    for b in (0, 2, 3):
+        if tie[row_off[b]:row_off[b + 1]].any() or ptie[k_off[b]:k_off[b + 1]].any():
+            continue
+        assert A[b] == ref["accept_len"][b] and corr[b] == ref["correction_token"][b]
+    # the long window: verified over its first 64 positions only
+    assert 0 <= A[1] <= 64
+    if not tie[row_off[1]:row_off[1] + 65].any() and not ptie[k_off[1]:k_off[1] + 64].any():
+        assert A[1] == min(int(ref["accept_len"][1]), 64)
+    seen_rows = np.ones(R, bool)
+    seen_rows[row_off[1] + 65:row_off[2]] = False                   # rows past the cut are not reported
+    assert np.max(np.abs(out.lse.cpu().numpy() - ref["lse"])[seen_rows]) <= 1e-2
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    from paper_2604_17701_b200 import WisvError
+    with pytest.raises(WisvError) as e:
+        v.verify_host(pin(ht), pin(toks), pin(hd), pin(csi), B=cfg.B, k_off=pin(k_off), T=T)
+    assert e.value.code == -2
     v.close()
 
 

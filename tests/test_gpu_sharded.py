@@ -8,7 +8,7 @@ import pytest
 import torch
 
 import gen
-from paper_2604_17701_b200 import cases
+from gen import cases
 from parity import compare, oracle_ref_argmax, run_oracle
 
 pytestmark = pytest.mark.gpu

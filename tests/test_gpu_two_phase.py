@@ -4,7 +4,8 @@ import pytest
 import torch
 
 import gen
-from paper_2604_17701_b200 import WisvError, cases
+from paper_2604_17701_b200 import WisvError
+from gen import cases
 from parity import compare, oracle_ref_argmax, run_oracle
 
 pytestmark = pytest.mark.gpu
@@ -90,4 +91,40 @@ def test_decide_needs_a_matching_localize():
     assert torch.equal(out.accept_len, ref.accept_len)
     with pytest.raises(WisvError):                          # consumed by the verify above
         v.decide(d["target_hidden"], d["draft_hidden"], d["csi"], B=4, K=4, T=16)
+    v.close()
+
+
+def test_decide_enqueued_right_behind_other_rounds_reads_its_own_inputs():
+    """The decision-head launch of wisv_decide follows the pack kernel directly (no LM-head launch in between), so it
+    must wait for the pack kernel before its first read.  A full-hidden round on other hidden states, then localize and
+    decide with several hundred selected positions, all enqueued back to back with no host synchronisation: the
+    result must equal one wisv_verify on the second batch."""
+    cfg_a = _cfg(B=60, K=8, seed=91, match_rate=0.2, weight_seed=90)
+    cfg_b = _cfg(B=60, K=8, seed=92, match_rate=0.2, weight_seed=90)
+    w = gen.make_weights(cfg_a)
+    case_a = cases.make_case(cfg_a, oracle_ref_argmax, weights=w)
+    case_b = cases.make_case(cfg_b, oracle_ref_argmax, weights=w)
+    da, db = cases.to_device(case_a, DEV), cases.to_device(case_b, DEV)
+    v = cases.make_verifier(db, max_sel=case_b["T"])
+    one = cases.run(v, db)
+    torch.cuda.synchronize()
+    mask = one.mismatch_mask.cpu().numpy().astype(np.uint64)
+    sel = np.zeros(case_b["T"], bool)
+    for b in range(cfg_b.B):
+        for i in range(cfg_b.K):
+            sel[b * cfg_b.K + i] = (int(mask[b]) >> i) & 1
+    assert sel.sum() >= 300
+    packed, sel_off, sel_pos = gen.pack_selective(case_b["draft_hidden"], case_b["k_len"], sel)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+    packed_d, sel_off_d, sel_pos_d = dev(packed), dev(sel_off), dev(sel_pos)
+    geo = dict(B=cfg_b.B, K=cfg_b.K, T=case_b["T"])
+    torch.cuda.synchronize()
+    for _ in range(20):
+        cases.run(v, da)                                    # leaves batch A's head inputs in the workspace
+        v.localize(db["target_hidden"], db["draft_tokens"], **geo)
+        dec = v.decide(db["target_hidden"], packed_d, db["csi"], sel_off=sel_off_d, sel_pos=sel_pos_d, **geo)
+    torch.cuda.synchronize()
+    assert v.device_error() == 0
+    assert torch.equal(dec.accept_len, one.accept_len) and torch.equal(dec.correction_token, one.correction_token)
+    assert np.allclose(dec.head_prob.cpu().numpy(), one.head_prob.cpu().numpy()[sel], atol=1e-5)
     v.close()
