@@ -306,7 +306,7 @@ def shared_weights(cfg, rank, ranks):
     instead of all regenerating it at once on the same host cores; rank 0 removes the file when the job ends.
     Returns (weights, path or None).
     """
-    if ranks.world == 1:
+    if ranks.world == 1 or cfg.weight_seed < 0:         # (no model seed of its own: every rank's batch seed makes its model)
         return gen.make_weights(cfg), None
     ws = cfg.weight_seed if cfg.weight_seed >= 0 else cfg.seed
     path = os.path.join(SHM_DIR, "wisv_lm_head_%dx%d_seed%d_%s.npy" % (cfg.V, cfg.H, ws, os.environ.get("MASTER_PORT", "0")))

@@ -106,7 +106,7 @@ def test_model_weights_are_generated_once_and_shared_between_two_gloo_ranks(tmp_
         bench.SHM_DIR = %r
         rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
         r = bench.Ranks(world, backend="gloo")
-        cfg = bench.workload_config("tiny", rank)
+        cfg = gen.config("tiny").with_(weight_seed=77, seed=5 + 1000 * rank)     # one model, a batch per rank
         w, path = bench.shared_weights(cfg, rank, r)
         same = all(np.array_equal(np.asarray(w[k]), gen.make_weights(cfg)[k]) for k in ("lm_head", "W1", "b1", "w2"))
         rec = {"rank": rank, "same": bool(same), "owner": path is not None,
