@@ -68,6 +68,7 @@ CONFIGS: Dict[str, VerifyConfig] = {
     "8b_b64": VerifyConfig("8b_b64", B=64, K=8, match_rate=0.7, seed=3, **_8B),
     "8b_b64_m30": VerifyConfig("8b_b64_m30", B=64, K=8, match_rate=0.30, seed=2, **_8B),
     "8b_b64_m95": VerifyConfig("8b_b64_m95", B=64, K=8, match_rate=0.95, seed=4, **_8B),
+    "8b_sh64": VerifyConfig("8b_sh64", B=64, K=8, match_rate=0.65, mode="SH", seed=13, **_8B),
     "8b_sh256": VerifyConfig("8b_sh256", B=256, K=0, K_lo=4, K_hi=16, match_rate=0.65,
                              mode="SH", seed=5, **_8B),
     "8b_b512": VerifyConfig("8b_b512", B=512, K=16, match_rate=0.7, seed=6, **_8B),
