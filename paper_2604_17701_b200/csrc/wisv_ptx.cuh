@@ -61,6 +61,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// Non-blocking test of a phase (try_wait may suspend the thread for a while; a thread that polls several
+// barriers in turn must not).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ void fence_barrier_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
@@ -68,15 +83,13 @@ __device__ __forceinline__ void fence_proxy_async() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
-// Bounded wait: gives up after `limit_cycles` SM clocks (or as soon as *abort_flag
-// is set by another role), so a broken pipeline ends with an error word, never a
-// hang.  The deadline uses the SM's own cycle counter, which is cheap to read; the
-// first polls take no timestamp at all so a short wait costs nothing extra.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
-                                                  volatile int* abort_flag, uint64_t limit_cycles) {
-#pragma unroll 1
-    for (int i = 0; i < 8; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
+// Bounded wait: gives up after `limit_cycles` SM clocks (or as soon as *abort_flag is set by another role), so a
+// broken pipeline ends with an error word, never a hang.  The deadline uses the SM's own cycle counter.
+//
+// The shape of this function matters: measured on the MMA-issuing thread (4 MMAs + commit per K block, barrier
+// already complete), one try_wait in straight-line code costs about 70 clocks per K block, the same try_wait as the
+// condition of a loop about 370 - so the fast path is a single inline try and everything else lives out of line.
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint64_t limit_cycles) {
     const long long t0 = clock64();
     uint32_t it = 0;
     while (!mbar_try_wait(bar, parity)) {
@@ -86,6 +99,11 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
         }
     }
     return true;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
+                                                  volatile int* abort_flag, uint64_t limit_cycles) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, limit_cycles);
 }
 
 // ---------------------------------------------------------------- TMA

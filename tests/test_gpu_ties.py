@@ -159,9 +159,9 @@ def test_lowest_token_id_wins_at_every_merge_site(shape):
     if shape == "R200_pair_ranges":
         assert plan["lm_pair"] and plan["lm_carry"] and plan["lm_tiles_per_cta"] > 1
     if shape == "R512_pair_tiles":
-        assert plan["lm_pair"] and not plan["lm_carry"]
+        assert plan["lm_pair"] and not plan["lm_carry"] and plan["lm_n_cols"] == 256
     if shape == "R300_three_row_tiles":
-        assert not plan["lm_pair"] and not plan["lm_carry"]
+        assert plan["lm_swap"] and not plan["lm_carry"] and plan["lm_n_cols"] == 160      # two row blocks of 160
     if R <= 128:
         assert plan["lm_carry"] and plan["lm_tiles_per_cta"] > 1
     d = cases.to_device(case, DEV)
@@ -169,7 +169,7 @@ def test_lowest_token_id_wins_at_every_merge_site(shape):
     geo = dict(B=cfg.B, K=cfg.K, T=case["T"])
 
     # one-call round: automatic plan, then other MMA heights, tile heights, kernels and launch splits
-    tunings = [dict(), dict(lm_mma_m=128), dict(lm_single_cta=1), dict(head_ctas=-1),
+    tunings = [dict(), dict(lm_mma_m=128), dict(lm_single_cta=1), dict(head_ctas=-1), dict(lm_swap=-1),
                dict(head_ctas=-1, lm_single_cta=1, lm_mma_m=128)]
     if R <= 128:
         # other tile heights (with more rows the partial buffer is sized for the automatic tile and refuses finer ones)
