@@ -258,8 +258,7 @@ typedef struct {
                                 when it costs the LM head no extra round of tiles): CTAs given to the decision head
                                 there (0 = chosen automatically), -1 = always two launches */
     int32_t lm_mma_m;        /* 128: never use 64-row MMAs (the default for GEMMs with at most 64 valid rows) */
-    int32_t lm_swap;         /* -1: batches of 129..256 window rows keep the window rows on the M side of the pair MMA
-                                (the default puts the vocabulary there and the rows on the N side) */
+    int32_t lm_kb_per_stage; /* CTA-pair LM-head kernel: K blocks (of 64) per shared-memory stage: 1, 2 or 4 */
 } wisv_tuning;
 int wisv_set_tuning(wisv_ctx* ctx, const wisv_tuning* tuning);
 
@@ -279,7 +278,8 @@ typedef struct {
     int32_t lm_units_base, lm_units_rem, lm_tiles_per_cta, lm_rounds, lm_rounds_alone;
     int32_t head_carry, head_tile_n, head_ctas, head_m_tiles, head_n_tiles, head_k_splits, head_kb_per_split;
     int32_t head_stages, head_smem_bytes, head_units_base, head_units_rem, head_tiles_per_cta;
-    int32_t lm_swap, lm_n_cols;      /* CTA pairs with the vocabulary on the M side; the N of their MMAs (rows up to 16) */
+    int32_t lm_n_cols, lm_row_blocks;  /* CTA pairs: the window rows are cut into lm_row_blocks blocks of lm_n_cols rows (the N
+                                          of the MMAs, a multiple of 16) */
     int32_t lm_parts;                /* LM-head partials per window row */
 } wisv_plan_info;
 int wisv_plan_host(const wisv_config* cfg, int32_t sm_count, int32_t max_smem_bytes, int32_t R, int32_t P,

@@ -52,7 +52,7 @@ class _Result(C.Structure):
 class _Tuning(C.Structure):
     _fields_ = [("lm_tile_n", C.c_int32), ("lm_stages", C.c_int32), ("head_tile_n", C.c_int32),
                 ("head_stages", C.c_int32), ("lm_single_cta", C.c_int32), ("head_ctas", C.c_int32),
-                ("lm_mma_m", C.c_int32), ("lm_swap", C.c_int32)]
+                ("lm_mma_m", C.c_int32), ("lm_kb_per_stage", C.c_int32)]
 
 
 class LinkParams(C.Structure):
@@ -81,7 +81,7 @@ class PlanInfo(C.Structure):
         "lm_units_base", "lm_units_rem", "lm_tiles_per_cta", "lm_rounds", "lm_rounds_alone",
         "head_carry", "head_tile_n", "head_ctas", "head_m_tiles", "head_n_tiles", "head_k_splits",
         "head_kb_per_split", "head_stages", "head_smem_bytes", "head_units_base", "head_units_rem",
-        "head_tiles_per_cta", "lm_swap", "lm_n_cols", "lm_parts")]
+        "head_tiles_per_cta", "lm_n_cols", "lm_row_blocks", "lm_parts")]
 
 
 def plan_host(*, H: int, V: int, H_d: int, d_c: int, d_J: int, R: int, P: int, sm_count: int = 148,
@@ -465,8 +465,8 @@ class Verifier:
         return n
 
     def set_tuning(self, lm_tile_n: int = 0, lm_stages: int = 0, head_tile_n: int = 0, head_stages: int = 0,
-                   lm_single_cta: int = 0, head_ctas: int = 0, lm_mma_m: int = 0, lm_swap: int = 0):
-        t = _Tuning(lm_tile_n, lm_stages, head_tile_n, head_stages, lm_single_cta, head_ctas, lm_mma_m, lm_swap)
+                   lm_single_cta: int = 0, head_ctas: int = 0, lm_mma_m: int = 0, lm_kb_per_stage: int = 0):
+        t = _Tuning(lm_tile_n, lm_stages, head_tile_n, head_stages, lm_single_cta, head_ctas, lm_mma_m, lm_kb_per_stage)
         _check(self.lib.wisv_set_tuning(self._h, C.byref(t)), "wisv_set_tuning")
 
     def launch_count(self) -> int:

@@ -10,7 +10,7 @@ CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libwisv.so")
 SOURCES = [os.path.join(CSRC, "wisv_api.cu"), os.path.join(CSRC, "wisv_static.cu"),
            os.path.join(CSRC, "wisv_link.cu")]
-DEPS = SOURCES + [os.path.join(CSRC, n) for n in ("wisv_gemm.cuh", "wisv_gemm2.cuh", "wisv_gemm3.cuh", "wisv_aux.cuh", "wisv_ptx.cuh")] + \
+DEPS = SOURCES + [os.path.join(CSRC, n) for n in ("wisv_gemm.cuh", "wisv_gemm2.cuh", "wisv_aux.cuh", "wisv_ptx.cuh")] + \
     [os.path.join(os.path.dirname(_HERE), "include", "wisv.h")]
 
 

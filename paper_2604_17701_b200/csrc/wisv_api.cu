@@ -18,7 +18,6 @@
 #include "wisv_aux.cuh"
 #include "wisv_gemm.cuh"
 #include "wisv_gemm2.cuh"
-#include "wisv_gemm3.cuh"
 
 using namespace wisv;
 
@@ -33,17 +32,17 @@ constexpr int kNumRowVariants = kTileM / 8;        // a_rows = 8, 16, ..., 128
 constexpr int kStages = 4;                         // profiled stages per call
 constexpr int kSplitTileN = 64;                    // head tile height when K is split over CTAs
 constexpr int kSplitMaxRowTiles = 4;               // K is split for decision heads of up to this many row tiles
-constexpr int kSwapMaxRowTiles = 1 << 20;          // LM head: batches of up to this many 128-row tiles run with swapped operands
+constexpr int kPairKbPerStage = 2;                 // CTA-pair LM head: K blocks per shared-memory stage
 
 struct Plan {
     int tile_n, m_tiles, n_tiles, ctas, stages;
     int a_rows;      // activation rows loaded per tile (8..128)
     int carry;       // one partial per (row, CTA) instead of per (row, N-tile)
     int parts;       // partials per row
-    int pair;        // LM head on CTA pairs (256 x 256 tiles): m_tiles then counts tiles of 256 rows
-    int swap;        // pairs with the vocabulary on the M side and the window rows on the N side (129..256 rows)
-    int n_cols;      // swap: N of the MMA (window rows rounded up to 16)
-    int n_blocks;    // swap: row blocks of n_cols rows
+    int pair;        // LM head on CTA pairs (vocabulary on the M side, window rows on the N side): m_tiles = row blocks
+    int n_cols;      // pairs: N of the MMA = width of a row block (a multiple of 16)
+    int n_blocks;    // pairs: row blocks of n_cols rows
+    int kbs;         // pairs: K blocks per shared-memory stage
     int k_splits;    // work items per (m, n) tile along K (decision head with one row tile)
     int kb_per_split;
     int units_base, units_rem, tiles_per_cta;   // carry: contiguous ranges of 16-row units per CTA
@@ -176,45 +175,49 @@ void finish_plan(const wisv_ctx* c, Plan* p, int d_c, int k_blocks, int forced_s
     p->smem = fixed + (size_t)s * stage;
 }
 
-// Several row blocks with the operands swapped (wisv_gemm3.cuh) instead of row tiles of 128 / 256 on the M side:
-// worth it while the padding of the last row tile is a visible share of the batch.
-bool swap_pays(int m_tiles128) { return m_tiles128 <= kSwapMaxRowTiles; }
+// CTA-pair LM head: K blocks per stage and ring depth for row blocks of n_cols rows.
+void pair_ring(const wisv_ctx* c, Plan* p)
+{
+    int kbs = c->tune.lm_kb_per_stage > 0 ? c->tune.lm_kb_per_stage : kPairKbPerStage;
+    const int k_blocks = (c->cfg.H + kBlockK - 1) / kBlockK;
+    while (kbs > 1 && (kbs > k_blocks || ((size_t)c->max_smem - pair_fixed_bytes()) / pair_stage_bytes(p->n_cols, kbs) < 2)) kbs /= 2;
+    const size_t stage = pair_stage_bytes(p->n_cols, kbs);
+    int ss = (int)(((size_t)c->max_smem - pair_fixed_bytes()) / stage);
+    if (ss > kMaxStages) ss = kMaxStages;
+    if (c->tune.lm_stages >= 2 && c->tune.lm_stages < ss) ss = c->tune.lm_stages;
+    p->kbs = kbs;
+    p->stages = ss;
+    p->smem = pair_fixed_bytes() + (size_t)ss * stage;
+}
 
-// LM head: with a single row tile the kernel streams the weights once and is
-// HBM-bound, so the tile height over the vocabulary is chosen to fill the last
-// wave of CTAs; with many row tiles it is tensor-bound and takes the largest tile.
+// LM head.  Up to 128 window rows: single CTAs with the rows on the M side, each with one contiguous range of the
+// vocabulary (HBM-bound).  More rows: CTA pairs with the vocabulary on the M side and the rows on the N side
+// (wisv_gemm3.cuh) - one row block with carried vocabulary ranges up to 256 rows, several row blocks dealt out as
+// (vocabulary tile, row block) items above.  The tuning switches lm_single_cta / lm_tile_n keep every size on the
+// single-CTA kernel.
 Plan plan_lm(const wisv_ctx* c, int R, bool single_only = false, int sms = 0, int reserved_pairs = 0)
 {
     Plan p{};
     if (sms <= 0) sms = c->sm_count;
     const int V = c->cfg.V;
     p.m_tiles = (R + kTileM - 1) / kTileM;
-    // More than one row tile: CTA pairs on 256 x 256 tiles, each weight tile fetched once per pair.  A pair
-    // always computes 256 rows, so with an odd number of 128-row tiles its last tile is half padding.
-    // The pair kernel keeps the tensor pipe about 10 % busier than the single-CTA kernel (95 % against
-    // 86 %), so the padding pays off from 11 row tiles on.
-    const bool pair_fits = p.m_tiles % 2 == 0 || p.m_tiles >= 11;
-    const bool swap_blocks = R > kPairTileM && c->tune.lm_swap >= 0 && swap_pays(p.m_tiles);   // handled further down
-    if (p.m_tiles >= 2 && pair_fits && !swap_blocks && c->max_pairs > 0 && !single_only && !c->tune.lm_single_cta &&
-        !c->tune.lm_tile_n) {
+    if (p.m_tiles >= 2 && c->max_pairs > 0 && !single_only && !c->tune.lm_single_cta && !c->tune.lm_tile_n) {
         p.pair = 1;
-        p.m_tiles = (R + kPairTileM - 1) / kPairTileM;
-        p.tile_n = kPairTileN;
-        p.n_tiles = (V + kPairTileN - 1) / kPairTileN;
         p.a_rows = kTileM;
         p.k_splits = 1;
         p.kb_per_split = (c->cfg.H + kBlockK - 1) / kBlockK;
-        int s = (int)(((size_t)c->max_smem - pair_fixed_bytes()) / kPairStageBytes);
-        if (s > kMaxStages) s = kMaxStages;
-        if (c->tune.lm_stages >= 2 && c->tune.lm_stages < s) s = c->tune.lm_stages;
-        p.stages = s;
-        p.smem = pair_fixed_bytes() + (size_t)s * kPairStageBytes;
         int pairs_free = c->max_pairs - reserved_pairs;
         if (pairs_free < 1) pairs_free = 1;
-        if (p.m_tiles == 1) {
-            // One row tile of 256 (HBM-bound): like the single-CTA kernel with one row tile, every pair gets one
-            // contiguous range of the vocabulary, here in units of 32 rows (each CTA of a pair loads half a tile,
-            // a multiple of 16 rows), cut into tiles of nearly equal height; one partial per (row, pair).
+        // the rows are cut into ceil(R / 256) blocks of equal width (a multiple of 16): no block is padded by more
+        // than 15 rows, and an MMA of N columns costs N / 2 clocks
+        p.n_blocks = (R + kPairMaxCols - 1) / kPairMaxCols;
+        p.n_cols = round_up((R + p.n_blocks - 1) / p.n_blocks, 16);
+        p.m_tiles = p.n_blocks;
+        pair_ring(c, &p);
+        if (p.n_blocks == 1) {
+            // One row block (HBM-bound): like the single-CTA kernel with one row tile, every pair gets one contiguous
+            // range of the vocabulary, here in units of 32 rows (each CTA of a pair loads half a tile, a multiple of
+            // 16 rows), cut into tiles of nearly equal height; one partial per (row, CTA).
             const int units = (V + 31) / 32;
             const int pairs = units < pairs_free ? units : pairs_free;
             p.units_base = units / pairs;
@@ -226,52 +229,14 @@ Plan plan_lm(const wisv_ctx* c, int R, bool single_only = false, int sms = 0, in
             p.n_tiles = pairs * p.tiles_per_cta;
             p.ctas = 2 * pairs;
             p.carry = 1;
-            p.parts = pairs;
-            if (c->tune.lm_swap >= 0) {
-                // Operands swapped (wisv_gemm3.cuh): the vocabulary tile on the 256-row M side of the pair MMA, the
-                // window rows on its N side, so the tensor pipe is busy in proportion to the rows that exist; each
-                // CTA writes its own partial per row.
-                p.swap = 1;
-                p.n_cols = round_up(R, 16);
-                p.n_blocks = 1;
-                const size_t stage = swap_stage_bytes(p.n_cols);
-                int ss = (int)(((size_t)c->max_smem - swap_fixed_bytes()) / stage);
-                if (ss > kMaxStages) ss = kMaxStages;
-                if (c->tune.lm_stages >= 2 && c->tune.lm_stages < ss) ss = c->tune.lm_stages;
-                p.stages = ss;
-                p.smem = swap_fixed_bytes() + (size_t)ss * stage;
-                p.parts = 2 * pairs;
-            }
+            p.parts = 2 * pairs;
             return p;
         }
-        const long long tiles = (long long)p.m_tiles * p.n_tiles;
-        p.ctas = 2 * (int)(tiles < pairs_free ? tiles : pairs_free);
+        // Several row blocks (tensor-bound): work items (vocabulary tile of 256, row block) dealt out round-robin; one
+        // partial per (row, vocabulary tile, CTA).
         p.carry = 0;
-        p.parts = p.n_tiles;
-        return p;
-    }
-    if (p.m_tiles >= 2 && c->max_pairs > 0 && !single_only && !c->tune.lm_single_cta && !c->tune.lm_tile_n &&
-        c->tune.lm_swap >= 0 && swap_pays(p.m_tiles)) {
-        // Operands swapped, several row blocks: the rows are cut into ceil(R / 256) blocks of equal width (a multiple of
-        // 16), so no block is padded by more than 15 rows; work items (vocabulary tile of 256, row block) dealt out
-        // round-robin; one partial per (row, vocabulary tile, CTA).
-        p.pair = 1; p.swap = 1; p.carry = 0;
-        p.n_blocks = (R + kSwapMaxCols - 1) / kSwapMaxCols;
-        p.n_cols = round_up((R + p.n_blocks - 1) / p.n_blocks, 16);
-        p.m_tiles = p.n_blocks;
         p.tile_n = kPairTileN;
         p.n_tiles = (V + kPairTileN - 1) / kPairTileN;
-        p.a_rows = kTileM;
-        p.k_splits = 1;
-        p.kb_per_split = (c->cfg.H + kBlockK - 1) / kBlockK;
-        const size_t stage = swap_stage_bytes(p.n_cols);
-        int ss = (int)(((size_t)c->max_smem - swap_fixed_bytes()) / stage);
-        if (ss > kMaxStages) ss = kMaxStages;
-        if (c->tune.lm_stages >= 2 && c->tune.lm_stages < ss) ss = c->tune.lm_stages;
-        p.stages = ss;
-        p.smem = swap_fixed_bytes() + (size_t)ss * stage;
-        int pairs_free = c->max_pairs - reserved_pairs;
-        if (pairs_free < 1) pairs_free = 1;
         const long long items = (long long)p.n_blocks * p.n_tiles;
         p.ctas = 2 * (int)(items < pairs_free ? items : pairs_free);
         p.parts = 2 * p.n_tiles;
@@ -561,28 +526,7 @@ inline int pair_map_lo(const Plan& pl) { return pl.tile_n / 32 - 2 > 0 ? pl.tile
 PairParams pair_params(const wisv_ctx* c, const Plan& pl, int R)
 {
     const wisv_config& cf = c->cfg;
-    PairParams qp;
-    memset(&qp, 0, sizeof qp);
-    qp.rows = R; qp.n_total = cf.V; qp.k_blocks = (cf.H + kBlockK - 1) / kBlockK; qp.mp_tiles = pl.m_tiles;
-    {
-        // raster groups: keep a group's bf16 rows (256 x H x 2 bytes per row tile) within 32 MB of L2
-        const long long tile_bytes = (long long)kPairTileM * cf.H * 2;
-        int mg_max = (int)((32ll << 20) / tile_bytes);
-        if (mg_max < 1) mg_max = 1;
-        const int groups = (pl.m_tiles + mg_max - 1) / mg_max;
-        qp.m_group = (pl.m_tiles + groups - 1) / groups;
-    }
-    qp.n_tiles = pl.n_tiles; qp.stages = pl.stages; qp.part_stride = pl.parts; qp.err = c->err;
-    qp.carry = pl.carry; qp.units_base = pl.units_base; qp.units_rem = pl.units_rem;
-    qp.tiles_per_pair = pl.tiles_per_cta > 0 ? pl.tiles_per_cta : 1; qp.tile_n = pl.tile_n;
-    qp.lm_part = c->lm_part; qp.row_tok = c->row_tok; qp.tok_logit = c->tok_logit;
-    return qp;
-}
-
-SwapParams swap_params(const wisv_ctx* c, const Plan& pl, int R)
-{
-    const wisv_config& cf = c->cfg;
-    SwapParams sp;
+    PairParams sp;
     memset(&sp, 0, sizeof sp);
     sp.rows = R; sp.n_cols = pl.n_cols; sp.row_blocks = pl.n_blocks; sp.n_total = cf.V;
     sp.k_blocks = (cf.H + kBlockK - 1) / kBlockK; sp.carry = pl.carry; sp.n_tiles = pl.n_tiles;
@@ -594,7 +538,7 @@ SwapParams swap_params(const wisv_ctx* c, const Plan& pl, int R)
         const int groups = (pl.n_blocks + bg_max - 1) / bg_max;
         sp.b_group = (pl.n_blocks + groups - 1) / groups;
     }
-    sp.stages = pl.stages; sp.units_base = pl.units_base; sp.units_rem = pl.units_rem;
+    sp.stages = pl.stages; sp.kbs = pl.kbs > 0 ? pl.kbs : 1; sp.units_base = pl.units_base; sp.units_rem = pl.units_rem;
     sp.tiles_per_pair = pl.tiles_per_cta > 0 ? pl.tiles_per_cta : 1; sp.tile_m = pl.tile_n;
     sp.part_stride = pl.parts; sp.err = c->err;
     sp.lm_part = c->lm_part; sp.row_tok = c->row_tok; sp.tok_logit = c->tok_logit;
@@ -694,8 +638,6 @@ int wisv_create(const wisv_config* cfg, const wisv_weights* w, wisv_ctx** out)
                                    (int)prop.sharedMemPerBlockOptin));
     WISV_CUDA(cudaFuncSetAttribute(lmhead_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)prop.sharedMemPerBlockOptin));
-    WISV_CUDA(cudaFuncSetAttribute(lmhead_swap_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   (int)prop.sharedMemPerBlockOptin));
     WISV_CUDA(cudaFuncSetAttribute(round_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)prop.sharedMemPerBlockOptin));
 
@@ -747,13 +689,10 @@ int wisv_create(const wisv_config* cfg, const wisv_weights* w, wisv_ctx** out)
             if (e2 > lm_elems) lm_elems = e2;
         }
         if (cfg->max_rows > kTileM) {
-            // several row tiles or row blocks: one partial per (row, vocabulary tile of 256), two with swapped
-            // operands (one per CTA of a pair); automatic plans only, a finer tuned tile is refused
+            // several row tiles (single CTAs, when tuned so): one partial per (row, vocabulary tile of 256); several row
+            // blocks on pairs: two, one per CTA; automatic plans only, a finer tuned tile is refused
             const size_t nt = (size_t)(cfg->V + kPairTileN - 1) / kPairTileN;
-            const long long swap_rows = (long long)kSwapMaxRowTiles * kTileM;
-            const size_t rs = (size_t)(cfg->max_rows < swap_rows ? cfg->max_rows : swap_rows);
-            size_t e = (size_t)cfg->max_rows * nt;
-            if (rs * 2 * nt > e) e = rs * 2 * nt;
+            const size_t e = (size_t)cfg->max_rows * 2 * nt;
             if (e > lm_elems) lm_elems = e;
         }
         head_elems = (size_t)c->max_pos * ((cfg->d_J + 15) / 16);
@@ -865,7 +804,7 @@ int wisv_plan_host(const wisv_config* cfg, int32_t sm_count, int32_t max_smem_by
     }
     out->kernels = fused ? 3 : (P > 0 ? 4 : 3);
     out->head_in_lm_launch = fused ? 1 : 0;
-    out->lm_swap = a.swap; out->lm_n_cols = a.n_cols; out->lm_parts = a.parts;
+    out->lm_n_cols = a.n_cols; out->lm_row_blocks = a.n_blocks; out->lm_parts = a.parts;
     out->lm_pair = a.pair; out->lm_carry = a.carry; out->lm_tile_n = a.tile_n; out->lm_ctas = a.ctas;
     out->lm_m_tiles = a.m_tiles; out->lm_n_tiles = a.n_tiles; out->lm_stages = a.stages; out->lm_smem_bytes = (int32_t)a.smem;
     out->lm_units_base = a.units_base; out->lm_units_rem = a.units_rem; out->lm_tiles_per_cta = a.tiles_per_cta;
@@ -892,7 +831,7 @@ int wisv_set_tuning(wisv_ctx* c, const wisv_tuning* t)
         if (tn[i] != 0 && (tn[i] < 16 || tn[i] > kMaxTileN || tn[i] % 16)) return WISV_ESHAPE;
     if (t->lm_stages < 0 || t->head_stages < 0 || t->lm_stages == 1 || t->head_stages == 1) return WISV_ESHAPE;
     if (t->lm_mma_m != 0 && t->lm_mma_m != 64 && t->lm_mma_m != 128) return WISV_ESHAPE;
-    if (t->lm_swap != 0 && t->lm_swap != -1) return WISV_ESHAPE;
+    if (t->lm_kb_per_stage != 0 && t->lm_kb_per_stage != 1 && t->lm_kb_per_stage != 2 && t->lm_kb_per_stage != 4) return WISV_ESHAPE;
     c->tune = *t;
     return WISV_OK;
 }
@@ -975,18 +914,11 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
         gh.head_part = c->head_part; gh.b1 = c->w.b1; gh.w2 = c->w.w2; gh.w1c = c->W1c; gh.csi = b->csi;
         gh.pos_req = c->pos_req; gh.d_c = cf.d_c; gh.act = cf.act;
         const size_t smem = pl.smem > ph.smem ? pl.smem : ph.smem;
-        if (pl.swap) {
-            const SwapParams sp = swap_params(c, pl, R);
-            const int rc = launch_pdl(lmhead_swap_kernel, dim3(pl.ctas + round_up(ph.ctas, 2)), dim3(kGemmThreads), smem,
+        if (pl.pair) {
+            const PairParams sp = pair_params(c, pl, R);
+            const int rc = launch_pdl(lmhead_pair_kernel, dim3(pl.ctas + round_up(ph.ctas, 2)), dim3(kGemmThreads), smem,
                                       st, c->tmX[pl.n_cols / 16 - 1], c->tmW[pair_map_hi(pl)], c->tmW[pair_map_lo(pl)],
                                       sp, c->tmZ[ph.a_rows / 8 - 1], c->tmW1[map_hi(ph)], c->tmW1[map_lo(ph)], gh,
-                                      pl.ctas, ph.ctas);
-            if (rc != WISV_OK) return rc;
-        } else if (pl.pair) {
-            const PairParams qp = pair_params(c, pl, R);
-            const int rc = launch_pdl(lmhead_pair_kernel, dim3(pl.ctas + round_up(ph.ctas, 2)), dim3(kGemmThreads), smem,
-                                      st, c->tmX[kNumRowVariants - 1], c->tmW[pair_map_hi(pl)], c->tmW[pair_map_lo(pl)],
-                                      qp, c->tmZ[ph.a_rows / 8 - 1], c->tmW1[map_hi(ph)], c->tmW1[map_lo(ph)], gh,
                                       pl.ctas, ph.ctas);
             if (rc != WISV_OK) return rc;
         } else {
@@ -999,21 +931,12 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
             if (rc != WISV_OK) return rc;
         }
         c->launches++;
-    } else if (!rows_done && pl.swap) {
-        const SwapParams sp = swap_params(c, pl, R);
-        GemmParams none;
-        memset(&none, 0, sizeof none);
-        const int rc = launch_pdl(lmhead_swap_kernel, dim3(pl.ctas), dim3(kGemmThreads), pl.smem, st,
-                                  c->tmX[pl.n_cols / 16 - 1], c->tmW[pair_map_hi(pl)], c->tmW[pair_map_lo(pl)], sp,
-                                  c->tmZ[0], c->tmW1[0], c->tmW1[0], none, pl.ctas, 0);
-        if (rc != WISV_OK) return rc;
-        c->launches++;
     } else if (!rows_done && pl.pair) {
-        const PairParams qp = pair_params(c, pl, R);
+        const PairParams sp = pair_params(c, pl, R);
         GemmParams none;
         memset(&none, 0, sizeof none);
         const int rc = launch_pdl(lmhead_pair_kernel, dim3(pl.ctas), dim3(kGemmThreads), pl.smem, st,
-                                  c->tmX[kNumRowVariants - 1], c->tmW[pair_map_hi(pl)], c->tmW[pair_map_lo(pl)], qp,
+                                  c->tmX[pl.n_cols / 16 - 1], c->tmW[pair_map_hi(pl)], c->tmW[pair_map_lo(pl)], sp,
                                   c->tmZ[0], c->tmW1[0], c->tmW1[0], none, pl.ctas, 0);
         if (rc != WISV_OK) return rc;
         c->launches++;

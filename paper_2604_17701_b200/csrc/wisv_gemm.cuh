@@ -227,22 +227,20 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
     // kernel directly and wait here like the others.
     // The producer thread of the early waiters waits a little later: weight tiles do not depend on the
     // pack kernel, so it first puts one ring-full of them in flight.
+    // (The whole producer warp waits later, not just its issuing lane: lanes of one warp that sit in
+    // griddepcontrol.wait hold back the lane that diverged from them.)
     constexpr bool kWaitLast = (EPI == EPI_HEAD) && HEAD_WAITS_LAST;
-    const bool producer_thread = warp == 0 && lane == 0;
-    if (!kWaitLast && !producer_thread) griddep_wait();
+    const bool producer_warp = warp == 0;
+    if (!kWaitLast && !producer_warp) griddep_wait();
     // no thread of an early waiter lets the next kernel start before it has passed its own wait
-    if (kWaitLast || !producer_thread) griddep_launch_dependents();
+    if (kWaitLast || !producer_warp) griddep_launch_dependents();
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            int s = 0;
-            uint32_t ph = 0;
-            long long issued = 0;
-            bool ok = true;
-            long long pre = 0;                 // stages whose weight tile was requested before the wait
-            Item w;
-            if (!kWaitLast) {
+        long long pre = 0;                     // stages whose weight tile was requested before the wait
+        Item w;
+        if (!kWaitLast) {
+            if (lane == 0) {
                 for (int i = 0; pre < p.stages && item_at(i, w); ++i) {
                     const uint32_t tx = a_bytes + static_cast<uint32_t>(w.h) * kBlockK * 2;
                     for (int kb = w.kb0; kb < w.kb1 && pre < p.stages; ++kb, ++pre) {
@@ -251,9 +249,15 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
                         tma_load_2d(a_dst + a_bytes, b_map(w.h), kb * kBlockK, w.n0, full_bar(static_cast<int>(pre)));
                     }
                 }
-                griddep_wait();                // from here on the activation rows may be read
-                griddep_launch_dependents();
             }
+            griddep_wait();                    // from here on the activation rows may be read
+            griddep_launch_dependents();
+        }
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            long long issued = 0;
+            bool ok = true;
             for (int i = 0; ok && item_at(i, w); ++i) {
                 const uint32_t tx = a_bytes + static_cast<uint32_t>(w.h) * kBlockK * 2;
                 for (int kb = w.kb0; kb < w.kb1; ++kb) {

@@ -1,59 +1,94 @@
-// LM-head GEMM + row reduction on CTA pairs (tcgen05 cta_group::2), used when the batch has more
-// than one row tile.  Two CTAs of a cluster share one 256 x 256 output tile: CTA r holds rows
-// r*128 .. r*128+127 of the tile in its own TMEM and loads, per K block, its own 128 activation rows
-// and its half (128 rows) of the 256 weight rows - so every weight tile enters shared memory once
-// per pair instead of once per CTA, which is what limits the single-CTA kernel (shared-memory fill
-// and L2 -> SM traffic, and with it power).  One thread of the even CTA issues the MMAs for both.
+// LM-head GEMM + row reduction with the operands swapped: the VOCABULARY on the M side of a CTA-pair MMA
+// (tcgen05 cta_group::2, M = 256: 128 weight rows per CTA) and the WINDOW ROWS on the N side, for batches of
+// more than 128 window rows.
 //
-// Barriers: full[s] lives in the leader and counts the bytes of both CTAs' loads; empty[s] and
-// acc_full[a] exist in both CTAs and are signalled by a multicast tcgen05.commit; acc_empty[a] lives in
-// the leader and is arrived on by the epilogue warps of both CTAs.  No load uses multicast.  Every
-// wait is bounded; both CTAs meet at a cluster barrier before TMEM is released.
+// Why: one tcgen05.mma (K = 16) occupies the tensor pipe for max(57, N / 2) SM clocks per CTA whatever its M
+// (measured: 128 x N and 64 x N cost the same).  With the window rows on the 128-row M side a batch pays for its
+// row count rounded up to 128 (256 for a pair): 144 rows cost as much as 256, 288 rows as much as 384, 576 as
+// much as 640.  On the N side the granularity is 16 rows: the batch is cut into ceil(R / 256) row blocks of equal
+// width N (a multiple of 16, at most 256) and an MMA costs N / 2 clocks, so the tensor pipe is busy in proportion to
+// the rows that exist.  Each CTA also loads only half of a block's activation rows per K block (the pair MMA takes
+// the two halves of its B operand from the two CTAs).
+//
+// D[vocabulary row (TMEM lane), window row (TMEM column)].  A window row's statistics therefore run ACROSS lanes:
+// each epilogue warp moves 32 lanes x 32 columns at a time through a padded shared-memory buffer, after which
+// lane L owns column L of the chunk and scans that window row's 32 logits in ascending vocabulary order (strict
+// '>' keeps the lowest token id).  The running (max, argidx, sum exp) of a window row lives in the registers of
+// the lane that owns its column, per warp; the four warps of a CTA are then merged in vocabulary order.
+//
+// Two ways of dealing out the work:
+//  * one row block (up to 256 rows, bound by HBM): every pair owns one contiguous range of the vocabulary (units of
+//    32 rows, tiles of tile_m or tile_m - 32 rows, balanced to one unit), carries its running row state across its
+//    tiles and writes one partial per (row, CTA) at the end;
+//  * several row blocks (bound by the tensor pipe): work items (vocabulary tile of 256 rows, row block) are dealt
+//    out round-robin, row blocks of a group fastest, so the pairs that run at the same time share a weight tile
+//    through L2 and a group's activation rows stay resident there; one partial per (row, vocabulary tile, CTA).
+//
+// Barriers: full[s] in the leader counts both CTAs' bytes, empty[s] / acc_full[a] are signalled
+// in both CTAs by a multicast tcgen05.commit, acc_empty[a] in the leader collects the epilogue warps of both CTAs.
+// No load uses multicast; every wait is bounded.
 #pragma once
 
 #include "wisv_gemm.cuh"
 
 namespace wisv {
 
-constexpr int kPairTileM = 256;
-constexpr int kPairTileN = 256;
-constexpr uint32_t kPairStageBytes = 2u * kTileM * kBlockK * 2u;   // 128 activation rows + 128 weight rows
+constexpr int kPairTileM = 256;              // vocabulary rows of a pair tile (the M of the MMA): 128 per CTA
+constexpr int kPairTileN = kPairTileM;       // (the same number where it counts rows of the weight matrix)
+constexpr int kPairMaxCols = 256;            // window rows per row block (the N of the MMA)
+constexpr int kPairChunk = 32;               // columns moved through shared memory at a time
+constexpr int kPairPitch = 36;               // floats per column in the transposition buffer (16-byte rows, no bank conflicts)
+constexpr int kPairMaxChunks = kPairMaxCols / kPairChunk;
 
 struct PairParams {
     int32_t rows;        // valid window rows
+    int32_t n_cols;      // N of the MMA = width of a row block: a multiple of 16, at most 256
+    int32_t row_blocks;  // ceil(rows / n_cols)
     int32_t n_total;     // vocabulary size
     int32_t k_blocks;
-    int32_t mp_tiles;    // row tiles of 256
-    int32_t m_group;     // row tiles per raster group: tiles run group by group (all vocabulary tiles of a
-                         // group of row tiles before the next group) so that the activation rows of a group
-                         // stay resident in L2 while the weights stream past them
-    int32_t n_tiles;     // vocabulary tiles of 256
     int32_t stages;
-    // One row tile of 256 (carry = 1): the vocabulary is dealt out in units of 32 rows as one contiguous range per
-    // pair - units_base units, one more for the first units_rem pairs - cut into tiles_per_pair tiles of tile_n or
-    // tile_n - 32 rows; a pair carries its running row state across its tiles and writes one partial per (row, pair).
-    // The pairs then finish together for any vocabulary size and any number of pairs.
-    int32_t carry, units_base, units_rem, tiles_per_pair, tile_n;
-    int32_t part_stride; // partials per row (n_tiles, or the number of pairs when carry)
+    int32_t kbs;         // K blocks per stage (1, 2 or 4): one barrier round trip, on both sides of the ring, serves kbs K blocks
+    // one row block (carry = 1): vocabulary ranges in units of 32 rows per pair - units_base units, one more for the
+    // first units_rem pairs - cut into tiles_per_pair tiles of tile_m or tile_m - 32 rows
+    int32_t carry, units_base, units_rem, tiles_per_pair, tile_m;
+    // several row blocks (carry = 0): n_tiles vocabulary tiles of 256 rows; items run group by group (all vocabulary
+    // tiles of a group of b_group row blocks before the next group)
+    int32_t n_tiles, b_group;
+    int32_t part_stride; // partials per row: 2 per pair (carry) or 2 per vocabulary tile
     int32_t* err;
     float4* lm_part;
     const int32_t* row_tok;
     float* tok_logit;
 };
 
-__host__ __device__ inline uint32_t pair_fixed_bytes() { return 1024u + 1024u; }   // alignment slack + barriers
+__host__ __device__ inline uint32_t pair_stage_bytes(int n_cols, int kbs = 1) {
+    return static_cast<uint32_t>(kbs) * static_cast<uint32_t>(kTileM * kBlockK * 2 + (n_cols / 2) * kBlockK * 2);
+}
+// alignment slack + barriers, then the four warps' transposition buffers
+__host__ __device__ inline uint32_t pair_fixed_bytes() {
+    return 1024u + 1024u + 4u * kPairChunk * kPairPitch * 4u;
+}
 
-// CTAs from lm_ctas on (whole clusters) do not belong to a pair: they evaluate the decision head with the
-// single-CTA GEMM body while the pairs stream the LM head (batches of at most 256 window rows, where the
-// LM head is bound by HBM and the head would otherwise add its whole latency to the round).
+__device__ __forceinline__ void pair_merge(float& mx, int& arg, float& sum, float omx, int oarg, float osum) {
+    if (omx == -CUDART_INF_F && osum == 0.0f) return;
+    if (omx > mx) {
+        sum = sum * exp2f((mx - omx) * 1.4426950408889634f) + osum;      // exp2(-inf) = 0 covers an empty left side
+        mx = omx; arg = oarg;
+    } else {
+        sum += osum * exp2f((omx - mx) * 1.4426950408889634f);
+        if (omx == mx && oarg < arg) arg = oarg;
+    }
+}
+
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
-lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                   const __grid_constant__ CUtensorMap tmB2, const PairParams p,
+lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
+                   const __grid_constant__ CUtensorMap tmW2, const PairParams p,
                    const __grid_constant__ CUtensorMap tmZ, const __grid_constant__ CUtensorMap tmW1,
                    const __grid_constant__ CUtensorMap tmW1_2, const GemmParams hd, const int lm_ctas,
                    const int head_ctas)
 {
     if (static_cast<int>(blockIdx.x) >= lm_ctas) {
+        // whole clusters beyond the pairs evaluate the decision head with the single-CTA GEMM body
         // (the grid is a whole number of clusters: with an odd head_ctas the last CTA has nothing to do)
         const int hc = static_cast<int>(blockIdx.x) - lm_ctas;
         if (hc < head_ctas) gemm_rowreduce_body<EPI_HEAD, false>(tmZ, tmW1, tmW1_2, hd, hc, head_ctas);
@@ -69,8 +104,12 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     const bool leader = rank == 0;
     const int pair_id = blockIdx.x >> 1;
     const int n_pairs = lm_ctas >> 1;
-    const uint32_t half_bytes = kTileM * kBlockK * 2;                 // 16 KB
-    const uint32_t ring_bytes = kPairStageBytes * static_cast<uint32_t>(p.stages);
+    const uint32_t a_bytes = kTileM * kBlockK * 2;                                   // weight slot: 128 rows
+    const uint32_t b_bytes = static_cast<uint32_t>(p.n_cols / 2) * kBlockK * 2;     // this CTA's half of a row block
+    // a stage holds kbs K blocks: [weights of block 0 .. kbs-1][window rows of block 0 .. kbs-1]
+    const uint32_t stage_bytes = static_cast<uint32_t>(p.kbs) * (a_bytes + b_bytes);
+    const uint32_t x_off = static_cast<uint32_t>(p.kbs) * a_bytes;
+    const uint32_t ring_bytes = stage_bytes * static_cast<uint32_t>(p.stages);
 
     const uint32_t bar_base = smem_base + ring_bytes;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
@@ -80,40 +119,39 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     const uint32_t drain_bar = bar_base + 8u * (2 * kMaxStages + 4);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + ring_bytes + 8 * (2 * kMaxStages + 5));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [0] abort, [1] drain scratch
+    float* trans_base = reinterpret_cast<float*>(smem + ring_bytes + 1024);      // 4 x [32 columns][36]
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int total_tiles = p.mp_tiles * p.n_tiles;
-    // tile t -> (row tile mp, vocabulary tile n): groups of m_group row tiles, row tile fastest inside a group
-    auto tile_mp_n = [&](int t, int* mp, int* n) {
-        const int per_group = p.m_group * p.n_tiles;
-        const int g = t / per_group;
-        const int mp0 = g * p.m_group;
-        const int gsize = min(p.m_group, p.mp_tiles - mp0);
-        const int idx = t - g * per_group;
-        *n = idx / gsize;
-        *mp = mp0 + idx % gsize;
-    };
     // carry: this pair's contiguous range of 32-row units and how it is cut into tiles
     const int my_units = p.units_base + (pair_id < p.units_rem ? 1 : 0);
     const int my_unit0 = pair_id * p.units_base + (pair_id < p.units_rem ? pair_id : p.units_rem);
     const int my_tiles = p.carry ? (my_units < p.tiles_per_pair ? my_units : p.tiles_per_pair) : 0;
     const int my_hq = p.carry ? my_units / p.tiles_per_pair : 0;
     const int my_hr = p.carry ? my_units % p.tiles_per_pair : 0;
-    // the i-th tile of this pair: row tile mp, first vocabulary row n0, height h (a multiple of 32), tile index n
-    struct PTile { int mp, n, n0, h; };
-    auto tile_at = [&](int i, PTile& w) -> bool {
+    const int total_items = p.n_tiles * p.row_blocks;
+    // the i-th work item of this pair: vocabulary tile (index n, first row n0, height h, a multiple of 32) x row block j
+    struct Item { int n, n0, h, j; };
+    auto item_at = [&](int i, Item& w) -> bool {
         if (p.carry) {
             if (i >= my_tiles) return false;
-            w.mp = 0; w.n = pair_id;
+            w.n = pair_id; w.j = 0;
             w.h = (my_hq + (i < my_hr ? 1 : 0)) * 32;
             w.n0 = (my_unit0 + i * my_hq + (i < my_hr ? i : my_hr)) * 32;
             return true;
         }
         const int t = pair_id + i * n_pairs;
-        if (t >= total_tiles) return false;
-        tile_mp_n(t, &w.mp, &w.n);
-        w.n0 = w.n * kPairTileN; w.h = kPairTileN;
+        if (t >= total_items) return false;
+        // groups of b_group row blocks; inside a group the row block runs fastest
+        const int per_group = p.b_group * p.n_tiles;
+        const int g = t / per_group;
+        const int j0 = g * p.b_group;
+        const int gsize = min(p.b_group, p.row_blocks - j0);
+        const int idx = t - g * per_group;
+        w.n = idx / gsize;
+        w.j = j0 + idx % gsize;
+        w.n0 = w.n * kPairTileN;
+        w.h = kPairTileN;
         return true;
     };
 
@@ -124,8 +162,8 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         abort_flag[0] = 0;
         abort_flag[1] = 0;
         fence_barrier_init();
-        tma_prefetch_desc(&tmA);
-        tma_prefetch_desc(&tmB);
+        tma_prefetch_desc(&tmX);
+        tma_prefetch_desc(&tmW);
     }
     if (warp == 1) {
         tmem_alloc_pair(smem_u32(tmem_slot), kTmemCols);
@@ -139,60 +177,63 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    // The pack kernel wrote the bf16 rows this kernel loads: everyone waits for it here, except the producer
-    // thread, which first puts one ring-full of weight tiles in flight (they depend on nothing) and waits then.
-    const bool producer_thread = warp == 0 && lane == 0;
-    if (!producer_thread) {
+    // The pack kernel wrote the bf16 rows this kernel loads: everyone waits for it here, except the producer warp,
+    // which first puts one ring-full of weight tiles in flight (they depend on nothing) and waits then.
+    if (warp != 0) {
         griddep_wait();
         griddep_launch_dependents();
     }
 
-    // producer thread only: ring position and stages issued so far (read again by the drain before the kernel ends)
-    int prod_s = 0;
-    uint32_t prod_ph = 0;
+    // producer thread only: stages issued so far (read again by the drain before the kernel ends)
     long long prod_issued = 0;
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (each CTA)
+        // One pass of this loop (barrier test, expect_tx, TMA issues: each a round trip of its own) costs the thread
+        // about 500 clocks whatever the tile sizes, more than the MMAs of one K block take when the row block is
+        // narrow; a stage of kbs K blocks spreads that over kbs blocks.  Plain counters and nested loops only: a 64-bit
+        // division per K block in this loop doubled the kernel's time.
+        Item w;
+        int pre = 0;                               // stages whose weight half-tiles were requested before the wait
         if (lane == 0) {
-            int& s = prod_s;
-            uint32_t& ph = prod_ph;
-            long long& issued = prod_issued;
-            bool ok = true;
-            PTile w;
-            long long pre = 0;                 // stages whose weight half-tile was requested before the wait
-            for (int i = 0; pre < p.stages && tile_at(i, w); ++i) {
+            for (int i = 0; pre < p.stages && item_at(i, w); ++i) {
                 const int half_h = w.h >> 1;
-                const int col0 = w.n0 + static_cast<int>(rank) * half_h;
-                const CUtensorMap* mapB = (w.h == p.tile_n) ? &tmB : &tmB2;
-                const uint32_t tx = 2u * (half_bytes + static_cast<uint32_t>(half_h) * kBlockK * 2u);
-                for (int kb = 0; kb < p.k_blocks && pre < p.stages; ++kb, ++pre) {
-                    const uint32_t a_dst = smem_base + kPairStageBytes * static_cast<uint32_t>(pre);
-                    if (leader) mbar_expect_tx(full_bar(static_cast<int>(pre)), tx);
-                    tma_load_2d_pair(a_dst + half_bytes, mapB, kb * kBlockK, col0, full_bar(static_cast<int>(pre)));
+                const int w_row0 = w.n0 + static_cast<int>(rank) * half_h;
+                const CUtensorMap* mapW = (w.h == p.tile_m) ? &tmW : &tmW2;
+                for (int kb = 0; kb < p.k_blocks && pre < p.stages; kb += p.kbs, ++pre) {
+                    const int nb = min(p.kbs, p.k_blocks - kb);
+                    const uint32_t dst = smem_base + stage_bytes * static_cast<uint32_t>(pre);
+                    if (leader)                    // both CTAs' bytes
+                        mbar_expect_tx(full_bar(pre), 2u * static_cast<uint32_t>(nb) * (static_cast<uint32_t>(half_h) * kBlockK * 2u + b_bytes));
+                    for (int u = 0; u < nb; ++u)
+                        tma_load_2d_pair(dst + static_cast<uint32_t>(u) * a_bytes, mapW, (kb + u) * kBlockK, w_row0, full_bar(pre));
                 }
             }
-            griddep_wait();
-            griddep_launch_dependents();
-            for (int i = 0; ok && tile_at(i, w); ++i) {
-                const int row0 = w.mp * kPairTileM + static_cast<int>(rank) * kTileM;
+        }
+        griddep_wait();
+        griddep_launch_dependents();
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int i = 0; ok && item_at(i, w); ++i) {
                 const int half_h = w.h >> 1;                                   // weight rows this CTA loads
-                const int col0 = w.n0 + static_cast<int>(rank) * half_h;
-                const CUtensorMap* mapB = (w.h == p.tile_n) ? &tmB : &tmB2;
-                const uint32_t tx = 2u * (half_bytes + static_cast<uint32_t>(half_h) * kBlockK * 2u);
-                for (int kb = 0; kb < p.k_blocks; ++kb) {
-                    const uint32_t a_dst = smem_base + kPairStageBytes * s;
-                    if (issued < pre) {
-                        // first pass over the ring: the stage is free, its bytes are expected and its weight
-                        // half-tile is already on its way
-                        tma_load_2d_pair(a_dst, &tmA, kb * kBlockK, row0, full_bar(s));
-                    } else {
+                const int w_row0 = w.n0 + static_cast<int>(rank) * half_h;
+                const int x_row0 = w.j * p.n_cols + static_cast<int>(rank) * (p.n_cols / 2);   // its half of the row block
+                const CUtensorMap* mapW = (w.h == p.tile_m) ? &tmW : &tmW2;
+                for (int kb = 0; kb < p.k_blocks; kb += p.kbs) {
+                    const int nb = min(p.kbs, p.k_blocks - kb);
+                    const uint32_t dst = smem_base + stage_bytes * static_cast<uint32_t>(s);
+                    if (prod_issued >= pre) {
                         if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, kWaitLimitClocks)) { ok = false; break; }
-                        if (leader) mbar_expect_tx(full_bar(s), tx);             // both CTAs' bytes
-                        tma_load_2d_pair(a_dst, &tmA, kb * kBlockK, row0, full_bar(s));
-                        tma_load_2d_pair(a_dst + half_bytes, mapB, kb * kBlockK, col0, full_bar(s));
-                    }
-                    ++issued;
+                        if (leader)
+                            mbar_expect_tx(full_bar(s), 2u * static_cast<uint32_t>(nb) * (static_cast<uint32_t>(half_h) * kBlockK * 2u + b_bytes));
+                        for (int u = 0; u < nb; ++u)
+                            tma_load_2d_pair(dst + static_cast<uint32_t>(u) * a_bytes, mapW, (kb + u) * kBlockK, w_row0, full_bar(s));
+                    }   // else: first pass over the ring, the stage is free and its weight half-tiles are on their way
+                    for (int u = 0; u < nb; ++u)
+                        tma_load_2d_pair(dst + x_off + static_cast<uint32_t>(u) * b_bytes, &tmX, (kb + u) * kBlockK, x_row0, full_bar(s));
+                    ++prod_issued;
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
             }
@@ -203,23 +244,27 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
-            PTile w;
-            for (int local = 0; ok && tile_at(local, w); ++local) {
-                const uint32_t idesc = idesc_bf16_f32(kPairTileM, static_cast<uint32_t>(w.h));
+            Item w;
+            // M = 256 whatever the tile height: weight rows that were not loaded feed lanes nobody reads
+            const uint32_t idesc = idesc_bf16_f32(kPairTileM, static_cast<uint32_t>(p.n_cols));
+            for (int local = 0; ok && item_at(local, w); ++local) {
                 const int as = local & 1;
                 const uint32_t aph = (local >> 1) & 1u;
                 if (!mbar_wait_bounded(acc_empty_bar(as), aph ^ 1u, abort_flag, kWaitLimitClocks)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(as * kAccCols);
-                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                for (int kb = 0; kb < p.k_blocks; kb += p.kbs) {
+                    const int nb = min(p.kbs, p.k_blocks - kb);
                     if (!mbar_wait_bounded(full_bar(s), ph, abort_flag, kWaitLimitClocks)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_addr = smem_base + kPairStageBytes * s;
-                    const uint64_t a_desc = smem_desc_k128(a_addr);
-                    const uint64_t b_desc = smem_desc_k128(a_addr + half_bytes);
+                    const uint32_t st_addr = smem_base + stage_bytes * s;
+                    for (int u = 0; u < nb; ++u) {
+                        const uint64_t a_desc = smem_desc_k128(st_addr + static_cast<uint32_t>(u) * a_bytes);          // weights: the M side
+                        const uint64_t b_desc = smem_desc_k128(st_addr + x_off + static_cast<uint32_t>(u) * b_bytes);  // window rows: the N side
 #pragma unroll
-                    for (int k = 0; k < kBlockK / kUmmaK; ++k)
-                        umma_bf16_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        for (int k = 0; k < kBlockK / kUmmaK; ++k)
+                            umma_bf16_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | u | k) != 0 ? 1u : 0u);
+                    }
                     umma_commit_pair(empty_bar(s));          // frees the stage in both CTAs
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
@@ -232,61 +277,151 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         }
     } else {
         // ------------------------------------------------------------ epilogue (warps 2..5 of each CTA)
-        const int q = warp & 3;
+        const int q = warp & 3;                                  // TMEM lane quadrant of this warp
+        const int ew = warp - 2;                                 // buffer of this warp
+        const int et = threadIdx.x - 64;                         // 0..127 among the epilogue threads
+        float* tbuf = trans_base + ew * (kPairChunk * kPairPitch);
+        // merge buffer [quadrant][column] (float4): 4 * 256 * 16 B = 16 KB, laid over the transposition buffers
+        float4* comb = reinterpret_cast<float4*>(trans_base);
         bool ok = true;
         const uint32_t leader_acc_empty0 = mapa_u32(acc_empty_bar(0), 0);
         const uint32_t leader_acc_empty1 = mapa_u32(acc_empty_bar(1), 0);
-        float mx = -CUDART_INF_F, sum = 0.0f;      // running row state: per tile, or per pair when carry
-        int arg = 0;
-        PTile w;
-        int last_row = -1;
-        for (int local = 0; ok && tile_at(local, w); ++local) {
+        const int n_chunks = (p.n_cols + kPairChunk - 1) / kPairChunk;
+        // lane L owns columns L, L + 32, ... of the row block: running state and draft token of each
+        float mx[kPairMaxChunks], sum[kPairMaxChunks];
+        int arg[kPairMaxChunks], tokc[kPairMaxChunks];
+        auto reset_state = [&](int j) {
+#pragma unroll
+            for (int u = 0; u < kPairMaxChunks; ++u) {
+                mx[u] = -CUDART_INF_F; sum[u] = 0.0f; arg[u] = 0x7fffffff;
+                const int r = j * p.n_cols + u * kPairChunk + lane;
+                tokc[u] = (u < n_chunks && u * kPairChunk + lane < p.n_cols && r < p.rows) ? p.row_tok[r] : -1;
+            }
+        };
+        // merge the four warps of this CTA in vocabulary order (warp q covers TMEM lanes 32q..) and write one
+        // partial per row of row block j to slot `slot` of the row's partials
+        auto flush_state = [&](int j, int slot) {
+            asm volatile("bar.sync 1, 128;" ::: "memory");        // every warp is done with its transposition buffer
+#pragma unroll
+            for (int u = 0; u < kPairMaxChunks; ++u) {
+                const int c = u * kPairChunk + lane;
+                if (u < n_chunks && c < p.n_cols)
+                    comb[q * kPairMaxCols + c] = make_float4(mx[u], __int_as_float(arg[u]), sum[u], 0.0f);
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            for (int c = et; c < p.n_cols; c += kEpiThreads) {
+                const int r = j * p.n_cols + c;
+                if (r >= p.rows) break;
+                float m = -CUDART_INF_F, sm = 0.0f;
+                int a = 0x7fffffff;
+#pragma unroll
+                for (int qq = 0; qq < 4; ++qq) {
+                    const float4 f = comb[qq * kPairMaxCols + c];
+                    pair_merge(m, a, sm, f.x, __float_as_int(f.y), f.z);
+                }
+                p.lm_part[(size_t)r * p.part_stride + slot] = make_float4(m, __int_as_float(a), sm, 0.0f);
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");        // the buffer goes back to the transposition
+        };
+        if (p.carry) reset_state(0);
+        Item w;
+        for (int local = 0; ok && item_at(local, w); ++local) {
             const int as = local & 1;
             const uint32_t aph = (local >> 1) & 1u;
-            const int row = w.mp * kPairTileM + static_cast<int>(rank) * kTileM + q * 32 + lane;
-            const bool valid = row < p.rows;
+            const int half_h = w.h >> 1;
+            const int warp_v0 = w.n0 + static_cast<int>(rank) * half_h + q * 32;    // token of this warp's first lane
+            const bool lane_valid = (q * 32 + lane < half_h) && (warp_v0 + lane < p.n_total);
+            const int row0 = w.j * p.n_cols;                                         // first window row of the block
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(as * kAccCols);
+            if (!p.carry) reset_state(w.j);
 
             bool got = mbar_wait_bounded(acc_full_bar(as), aph, abort_flag, kWaitLimitClocks);
-            got = __all_sync(0xffffffffu, got);
+            {
+                // The four warps must agree on `got`: they meet at barriers inside flush_state, and after a time-out
+                // one warp may have seen the abort flag while another still saw the accumulator arrive.
+                uint32_t all;
+                asm volatile(
+                    "{\n\t"
+                    ".reg .pred pi, po;\n\t"
+                    "setp.ne.u32 pi, %1, 0;\n\t"
+                    "barrier.cta.red.and.pred po, 1, 128, pi;\n\t"
+                    "selp.u32 %0, 1, 0, po;\n\t"
+                    "}\n"
+                    : "=r"(all) : "r"(got ? 1u : 0u) : "memory");
+                got = all != 0;
+            }
             if (!got) { ok = false; break; }
             tc_fence_after();
 
-            if (!p.carry) { mx = -CUDART_INF_F; sum = 0.0f; arg = 0; }
-            const int tok = valid ? p.row_tok[row] : -1;
-            for (int c0 = 0; c0 < w.h; c0 += 16) {
-                uint32_t v[16];
+            const bool warp_has_rows = (q * 32 < half_h) && (warp_v0 < p.n_total);   // uniform over the warp
+#pragma unroll
+            for (int u = 0; u < kPairMaxChunks; ++u) {
+                if (u >= n_chunks || !warp_has_rows) continue;
+                const int c0 = u * kPairChunk;
+                const int cols_here = min(kPairChunk, p.n_cols - c0);               // 16 or 32
+                if (row0 + c0 >= p.rows) continue;                                   // the block's padding columns
+                // ---- TMEM -> shared memory, transposed: tbuf[column][lane]
+                for (int hlf = 0; hlf * 16 < cols_here; ++hlf) {
+                    uint32_t v[16];
+                    tmem_ld16(taddr + static_cast<uint32_t>(c0 + hlf * 16), v);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int t = 0; t < 16; ++t)
+                        tbuf[(hlf * 16 + t) * kPairPitch + lane] = lane_valid ? __uint_as_float(v[t]) : -CUDART_INF_F;
+                }
                 __syncwarp();
-                tmem_ld16(taddr + static_cast<uint32_t>(c0), v);
-                tmem_wait_ld();
-                if (!valid) continue;
-                lm_update_chunk(v, w.n0 + c0, p.n_total, tok, mx, arg, sum, p.tok_logit + row);
+                // ---- lane L: window row row0 + c0 + L against this warp's 32 vocabulary rows, in ascending order
+                const int r = row0 + c0 + lane;
+                if (lane < cols_here && r < p.rows) {
+                    float x[32];
+                    const float4* src = reinterpret_cast<const float4*>(tbuf + lane * kPairPitch);
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) {
+                        const float4 f = src[t];
+                        x[4 * t] = f.x; x[4 * t + 1] = f.y; x[4 * t + 2] = f.z; x[4 * t + 3] = f.w;
+                    }
+                    float cm = x[0];
+                    int ci = 0;
+#pragma unroll
+                    for (int t = 1; t < 32; ++t) { if (x[t] > cm) { cm = x[t]; ci = t; } }
+                    if (cm != -CUDART_INF_F) {
+                        if (cm > mx[u]) {                     // strict: an earlier (lower) token keeps a tie
+                            sum[u] *= exp2f((mx[u] - cm) * 1.4426950408889634f);
+                            mx[u] = cm;
+                            arg[u] = warp_v0 + ci;
+                        }
+                        const float base = mx[u] * 1.4426950408889634f;
+                        float acc = 0.0f;
+#pragma unroll
+                        for (int t = 0; t < 32; ++t) acc += exp2f(fmaf(x[t], 1.4426950408889634f, -base));
+                        sum[u] += acc;
+                        const int d = tokc[u] - warp_v0;
+                        if (static_cast<unsigned>(d) < 32u && warp_v0 + d < p.n_total && q * 32 + d < half_h)
+                            p.tok_logit[r] = tbuf[lane * kPairPitch + d];
+                    }
+                }
+                __syncwarp();                                  // the buffer is rewritten by the next chunk
             }
+            // accumulator drained: hand it back to the MMA thread of the leader
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(as ? leader_acc_empty1 : leader_acc_empty0);
-            if (valid && !p.carry)
-                p.lm_part[(size_t)row * p.part_stride + w.n] = make_float4(mx, __int_as_float(arg), sum, 0.0f);
-            last_row = valid ? row : -1;
+            if (!p.carry) flush_state(w.j, w.n * 2 + static_cast<int>(rank));
         }
-        // carry: the tiles of a pair ascend through the vocabulary, so the strict '>' of the update kept the
-        // lowest index; a pair without tiles is never launched
-        if (p.carry && ok && last_row >= 0)
-            p.lm_part[(size_t)last_row * p.part_stride + pair_id] = make_float4(mx, __int_as_float(arg), sum, 0.0f);
+        // carry: the tiles of a pair ascend through the vocabulary, so the strict '>' of the update kept the lowest
+        // index; a pair without tiles is never launched.  (`ok` is the same in all four warps, see above.)
+        if (p.carry && ok) flush_state(0, pair_id * 2 + static_cast<int>(rank));
     }
 
     // After a time-out copies may still be heading for the shared memory of either CTA.  Their bytes are counted on
     // the leader's full barriers, so the leader's producer thread waits (bounded) for the stages it issued last
     // before it arrives at the closing cluster barrier, which in turn keeps the partner from retiring earlier.
     __syncthreads();
-    if (leader && producer_thread && abort_flag[0] != 0) {
-        const int inflight = prod_issued < p.stages ? static_cast<int>(prod_issued) : p.stages;
-        int ws = prod_s;
-        uint32_t wph = prod_ph;
-        for (int i = 0; i < inflight; ++i) {
-            if (--ws < 0) { ws = p.stages - 1; wph ^= 1u; }
-            mbar_wait_bounded(full_bar(ws), wph, abort_flag + 1, kWaitLimitClocks);
-        }
+    if (leader && warp == 0 && lane == 0 && abort_flag[0] != 0) {
+        // K block i went to slot i % stages and completes phase (i / stages) & 1 of its full barrier
+        for (long long i = prod_issued > p.stages ? prod_issued - p.stages : 0; i < prod_issued; ++i)
+            mbar_wait_bounded(full_bar(static_cast<int>(i % p.stages)), static_cast<uint32_t>((i / p.stages) & 1),
+                              abort_flag + 1, kWaitLimitClocks);
     }
     // neither CTA may retire (or release TMEM) while its partner can still signal or read it
     tc_fence_before();

@@ -773,7 +773,7 @@ def test_random_shapes_under_every_launch_plan():
         d = cases.to_device(case, DEV)
         v = cases.make_verifier(d)
         outs = []
-        for tune in (dict(), dict(head_ctas=-1), dict(lm_single_cta=1), dict(head_ctas=3), dict(lm_swap=-1)):
+        for tune in (dict(), dict(head_ctas=-1), dict(lm_single_cta=1), dict(head_ctas=3), dict(lm_kb_per_stage=1), dict(lm_kb_per_stage=4)):
             v.set_tuning(**tune)
             cases.run(v, d)
             out = cases.run(v, d)                       # twice: nothing may linger from the first call

@@ -77,7 +77,7 @@ def test_every_launch_plan_on_a_poisoned_workspace():
         d = cases.to_device(case, DEV)
         # capacity far above the batch: most of the workspace is never written by these rounds
         v = cases.make_verifier(d, max_requests=cfg.B + 40, max_rows=case["R"] + 700, max_sel=case["T"] + 300)
-        for tune in (dict(), dict(head_ctas=-1), dict(lm_single_cta=1), dict(head_ctas=3), dict(lm_mma_m=128), dict(lm_swap=-1)):
+        for tune in (dict(), dict(head_ctas=-1), dict(lm_single_cta=1), dict(head_ctas=3), dict(lm_mma_m=128), dict(lm_kb_per_stage=1)):
             v.set_tuning(**tune)
             clean = cases.run(v, d)
             torch.cuda.synchronize()

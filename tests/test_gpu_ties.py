@@ -5,9 +5,10 @@ argmax (Section II-A; Algorithm 1, commit-and-correct), so a tie has to be broke
 lowest id (the oracle's strict '>' scan).  Duplicated rows of the LM head give bit-identical fp32 logits on the
 GPU and bit-identical fp64 logits in the oracle, so the expected answer is exact.  The duplicates are planted so
 that the equal maxima of a window row meet at each merge site of the kernels: inside one 16-column chunk of the
-epilogue, in different chunks of one tile, in different tiles of one CTA's (or CTA pair's) carried vocabulary
-range, in different CTAs / pairs, in the two halves of a pair tile, in different vocabulary shards - under 64- and
-128-row MMAs, carried and per-tile partials, and through every entry point that reduces the LM head.
+epilogue (one warp's 32 vocabulary rows in the CTA-pair kernel), in different chunks of one tile (different warps
+there), in different tiles of one CTA's (or CTA pair's) carried vocabulary range, in different CTAs / pairs, in
+the two halves of a pair tile (its two CTAs), in different vocabulary shards - under 64- and 128-row MMAs, carried
+and per-tile partials, and through every entry point that reduces the LM head.
 """
 import ctypes as C
 
@@ -161,7 +162,7 @@ def test_lowest_token_id_wins_at_every_merge_site(shape):
     if shape == "R512_pair_tiles":
         assert plan["lm_pair"] and not plan["lm_carry"] and plan["lm_n_cols"] == 256
     if shape == "R300_three_row_tiles":
-        assert plan["lm_swap"] and not plan["lm_carry"] and plan["lm_n_cols"] == 160      # two row blocks of 160
+        assert plan["lm_pair"] and not plan["lm_carry"] and plan["lm_n_cols"] == 160      # two row blocks of 160
     if R <= 128:
         assert plan["lm_carry"] and plan["lm_tiles_per_cta"] > 1
     d = cases.to_device(case, DEV)
@@ -169,7 +170,7 @@ def test_lowest_token_id_wins_at_every_merge_site(shape):
     geo = dict(B=cfg.B, K=cfg.K, T=case["T"])
 
     # one-call round: automatic plan, then other MMA heights, tile heights, kernels and launch splits
-    tunings = [dict(), dict(lm_mma_m=128), dict(lm_single_cta=1), dict(head_ctas=-1), dict(lm_swap=-1),
+    tunings = [dict(), dict(lm_mma_m=128), dict(lm_single_cta=1), dict(head_ctas=-1), dict(lm_kb_per_stage=1),
                dict(head_ctas=-1, lm_single_cta=1, lm_mma_m=128)]
     if R <= 128:
         # other tile heights (with more rows the partial buffer is sized for the automatic tile and refuses finer ones)

@@ -57,10 +57,15 @@ def test_plans_at_the_task_shapes():
     assert p["lm_tile_n"] == 240 and p["lm_tiles_per_cta"] == 4 and p["lm_units_base"] == 56
     p = plan_host(R=144, P=128, **DIMS_8B)                   # B=16: pairs with head clusters
     assert (p["kernels"], p["lm_pair"], p["lm_carry"], p["lm_ctas"], p["head_ctas"]) == (3, 1, 1, 142, 6)
-    p = plan_host(R=576, P=512, **DIMS_8B)                   # B=64: 16.9 rounds on 148 SMs, nothing to spare
-    assert (p["kernels"], p["lm_pair"], p["lm_ctas"], p["lm_rounds"]) == (4, 0, 148, 17)
-    p = plan_host(R=8704, P=8192, **DIMS_8B)                 # B=512, K=16: 74 pairs, 230.2 rounds
+    assert (p["lm_n_cols"], p["lm_row_blocks"], p["lm_parts"]) == (144, 1, 142)     # the MMA's N is the row count up to 16
+    p = plan_host(R=288, P=256, **DIMS_8B)                   # B=32: two row blocks of 144, nothing padded
+    assert (p["kernels"], p["lm_pair"], p["lm_carry"], p["lm_n_cols"], p["lm_row_blocks"]) == (3, 1, 0, 144, 2)
+    p = plan_host(R=576, P=512, **DIMS_8B)                   # B=64: three row blocks of 192; 1503 items on 72 pairs
+    assert (p["kernels"], p["lm_pair"], p["lm_ctas"], p["lm_rounds"]) == (3, 1, 144, 21)
+    assert (p["lm_n_cols"], p["lm_row_blocks"], p["lm_parts"], p["head_ctas"]) == (192, 3, 1002, 4)
+    p = plan_host(R=8704, P=8192, **DIMS_8B)                 # B=512, K=16: 74 pairs, 230.2 rounds of 256 x 256 items
     assert (p["kernels"], p["lm_pair"], p["lm_ctas"], p["lm_rounds"]) == (4, 1, 148, 231)
+    assert (p["lm_n_cols"], p["lm_row_blocks"]) == (256, 34)
 
 
 @pytest.mark.parametrize("R", [257, 288, 384, 385, 432, 504, 576, 640, 864, 1017, 1152, 1408, 2816, 8704])
@@ -80,9 +85,17 @@ def test_head_rides_along_only_when_the_lm_head_needs_no_extra_round(R):
         assert p["lm_smem_bytes"] <= SMEM and p["head_smem_bytes"] <= SMEM
 
 
-def test_pairs_for_an_even_number_of_row_tiles_or_many():
-    for R, pair in ((129, 1), (256, 1), (257, 0), (384, 0), (385, 1), (512, 1), (576, 0), (1152, 0), (1281, 1), (1409, 1)):
-        assert plan_host(R=R, P=0, **DIMS_8B)["lm_pair"] == pair, R
+def test_row_blocks_of_the_pair_kernel_pad_at_most_fifteen_rows_each():
+    for R in (129, 144, 200, 256, 257, 288, 384, 385, 576, 600, 1017, 1280, 2816, 8704):
+        p = plan_host(R=R, P=0, **DIMS_8B)
+        assert p["lm_pair"] == 1
+        nb, n = p["lm_row_blocks"], p["lm_n_cols"]
+        assert nb == -(-R // 256) and n % 16 == 0 and 16 <= n <= 256
+        assert nb * n >= R and nb * (n - 16) < R              # the narrowest width that covers the rows
+        assert nb * n <= -(-R // 256) * 256                   # the blocks stay inside the rows the workspace holds
+        assert p["lm_carry"] == (1 if nb == 1 else 0)
+        assert p["lm_parts"] == (p["lm_ctas"] if nb == 1 else 2 * p["lm_n_tiles"])
+    assert plan_host(R=128, P=0, **DIMS_8B)["lm_pair"] == 0
 
 
 def test_decision_head_in_a_launch_of_its_own():
@@ -90,13 +103,14 @@ def test_decision_head_in_a_launch_of_its_own():
     p = plan_host(R=8 * 9, P=64, **{**DIMS_8B, "V": 128256}, sm_count=148)
     assert p["head_in_lm_launch"] == 1                        # (small batches ride along; no split there)
     assert p["head_k_splits"] == 1
-    # four row tiles (B=64, K=8): 64 column tiles of 64, K split in two, 128 work items for 148 SMs
-    p = plan_host(R=576, P=512, **DIMS_8B)
+    # four row tiles of positions beside an LM head that cannot spare SMs: 64 column tiles of 64, K split in two,
+    # 128 work items for 148 SMs
+    p = plan_host(R=1100, P=512, **DIMS_8B)
     assert (p["head_in_lm_launch"], p["head_tile_n"], p["head_m_tiles"], p["head_n_tiles"]) == (0, 64, 4, 16)
     assert p["head_k_splits"] == 2 and p["head_kb_per_split"] == 48 and p["head_ctas"] == 128
     assert p["head_k_splits"] * p["head_kb_per_split"] >= 96  # the splits cover all 96 K blocks
     # six row tiles: no split; one round of 128-wide items rather than three rounds of 16-wide ones
-    p = plan_host(R=864, P=768, **DIMS_8B)
+    p = plan_host(R=1100, P=768, **DIMS_8B)
     assert (p["head_in_lm_launch"], p["head_k_splits"], p["head_tile_n"]) == (0, 1, 128)
     assert p["head_m_tiles"] * p["head_n_tiles"] <= 148
     # many row tiles: the widest tiles
