@@ -28,8 +28,9 @@
  * accept_len in both branches.
  *
  * Numerics.  Hidden states are rounded to bf16 (nearest even) before every
- * matrix product; weights are bf16; accumulation and everything after the
- * products is fp32.  CSI features and the CSI columns of W1 enter in fp32.
+ * matrix product - fp32 and fp16 inputs are rounded by the library, bf16 inputs
+ * are taken as they are; weights are bf16; accumulation and everything after
+ * the products is fp32.  CSI features and the CSI columns of W1 enter in fp32.
  *
  * Conventions.  Every function returns 0 (WISV_OK) or a negative error code; no
  * function throws, aborts or prints.  Pointers marked "dev" are CUDA device
@@ -82,6 +83,11 @@ extern "C" {
                                       WISV_MAX_K positions (or none) were verified.  k_off lives on the device, so
                                       wisv_verify cannot check it; wisv_verify_host does and returns WISV_ESHAPE */
 
+/* element type of a hidden-state array (wisv_batch.target_hidden_dtype / draft_hidden_dtype) */
+#define WISV_DT_F32  0      /* fp32: rounded to bf16 (nearest even) by the library */
+#define WISV_DT_BF16 1      /* bf16: used as it is */
+#define WISV_DT_F16  2      /* fp16 (the 16-bit upload format of Section IV-A, b_h = 16): rounded to bf16 (nearest even) */
+
 #define WISV_MAX_K   64
 #define WISV_MAX_DC  16
 
@@ -116,9 +122,9 @@ typedef struct {
     int32_t K;                     /* uniform window length, or 0 with k_off != NULL */
     const int32_t* k_off;          /* dev int32 [B+1] prefix sums of K_b (ragged), or NULL */
     int32_t T_total;               /* sum of K_b (host-known; = B*K when uniform) */
-    const float*   target_hidden;  /* dev fp32 [R, H] */
+    const void*    target_hidden;  /* dev [R, H], element type target_hidden_dtype (fp32 by default), 16-byte aligned */
     const int32_t* draft_tokens;   /* dev int32 [T] */
-    const float*   draft_hidden;   /* dev fp32 [T, H_d] (FH) or [M_sel, H_d] (SH) */
+    const void*    draft_hidden;   /* dev [T, H_d] (FH) or [M_sel, H_d] (SH), element type draft_hidden_dtype */
     const int32_t* sel_off;        /* SH: dev int32 [B+1], CSR offsets into sel_pos */
     const int32_t* sel_pos;        /* SH: dev int32 [M_sel], window-relative positions */
     int32_t M_sel;                 /* SH: number of uploaded hidden states */
@@ -127,6 +133,9 @@ typedef struct {
     const float*   uniforms;       /* stochastic: dev fp32 [T], u in [0, 1) */
     uint32_t mode;                 /* WISV_MODE_* | WISV_ACCEPT_* */
     float    tau;                  /* NaN: use the context default */
+    int32_t  target_hidden_dtype;  /* WISV_DT_*: element type of target_hidden (0 = fp32) */
+    int32_t  draft_hidden_dtype;   /* WISV_DT_*: element type of draft_hidden; the drafter uploads its hidden states with
+                                      b_h = 16 bits per element (Section IV-A, Eq. 3), i.e. WISV_DT_F16 or WISV_DT_BF16 */
 } wisv_batch;
 
 typedef struct {

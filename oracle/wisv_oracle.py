@@ -128,6 +128,20 @@ def scan(k_off, cand, has_prob, prob, tau, argmax):
     return A, corr
 
 
+def hidden_as_f32(x) -> np.ndarray:
+    """Hidden states as the fp32 array the definition starts from.
+
+    The drafter uploads 16-bit hidden states (Section IV-A, b_h = 16): an fp16 array (numpy float16) is widened
+    exactly; bf16 values arrive as uint16 bit patterns and are widened exactly as well.  The rounding to bf16 that
+    precedes every matrix product is then applied by the C routines as for fp32 inputs: it leaves bf16 values as
+    they are and rounds fp16 values to nearest even.
+    """
+    x = np.asarray(x)
+    if x.dtype == np.uint16:
+        return (x.astype(np.uint32) << np.uint32(16)).view(np.float32)
+    return np.ascontiguousarray(x, dtype=np.float32)
+
+
 def verify(*, lm_head_bits, W1_bits, b1, w2, b2, act, tau, k_len, target_hidden, draft_tokens,
            draft_hidden, csi, sel_off=None, sel_pos=None, draft_q=None, uniforms=None,
            head_row_shift: int = 0) -> Dict[str, np.ndarray]:
@@ -148,8 +162,9 @@ def verify(*, lm_head_bits, W1_bits, b1, w2, b2, act, tau, k_len, target_hidden,
     T, R = int(k_off[-1]), int(row_off[-1])
     W = _c(lm_head_bits, np.uint16)
     V, H = W.shape
-    Ht = _c(target_hidden, np.float32)
+    Ht = hidden_as_f32(target_hidden)
     assert Ht.shape == (R, H)
+    draft_hidden = hidden_as_f32(draft_hidden)
     draft_tokens = _c(draft_tokens, np.int32)
     H_d = int(np.asarray(draft_hidden).shape[1]) if np.asarray(draft_hidden).ndim == 2 else 0
     csi = _c(csi, np.float32).reshape(B, -1)

@@ -16,6 +16,21 @@ _lib = None
 ACT_RELU, ACT_GELU = 0, 1
 MODE_FH, MODE_SH = 0, 1
 ACCEPT_GREEDY, ACCEPT_STOCHASTIC = 0, 2
+DT_F32, DT_BF16, DT_F16 = 0, 1, 2
+
+
+def _hidden_dtype(t) -> int:
+    """WISV_DT_* of a hidden-state tensor (fp32, bf16 or fp16)."""
+    if t is None:
+        return DT_F32
+    name = str(t.dtype)
+    if name.endswith("float32"):
+        return DT_F32
+    if name.endswith("bfloat16"):
+        return DT_BF16
+    if name.endswith("float16"):
+        return DT_F16
+    raise ValueError("hidden states must be float32, bfloat16 or float16, not %s" % name)
 
 
 class WisvError(RuntimeError):
@@ -40,7 +55,8 @@ class _Batch(C.Structure):
     _fields_ = [("B", C.c_int32), ("K", C.c_int32), ("k_off", C.c_void_p), ("T_total", C.c_int32),
                 ("target_hidden", C.c_void_p), ("draft_tokens", C.c_void_p), ("draft_hidden", C.c_void_p),
                 ("sel_off", C.c_void_p), ("sel_pos", C.c_void_p), ("M_sel", C.c_int32), ("csi", C.c_void_p),
-                ("draft_q", C.c_void_p), ("uniforms", C.c_void_p), ("mode", C.c_uint32), ("tau", C.c_float)]
+                ("draft_q", C.c_void_p), ("uniforms", C.c_void_p), ("mode", C.c_uint32), ("tau", C.c_float),
+                ("target_hidden_dtype", C.c_int32), ("draft_hidden_dtype", C.c_int32)]
 
 
 class _Result(C.Structure):
@@ -266,7 +282,8 @@ class Verifier:
         M_sel = int(sel_pos.shape[0]) if sel_pos is not None else 0
         return _Batch(B, 0 if k_off is not None else K, _ptr(k_off), T, _ptr(target_hidden), _ptr(draft_tokens),
                       _ptr(draft_hidden), _ptr(sel_off), _ptr(sel_pos), M_sel, _ptr(csi), _ptr(draft_q),
-                      _ptr(uniforms), mode, float("nan") if tau is None else float(tau))
+                      _ptr(uniforms), mode, float("nan") if tau is None else float(tau),
+                      _hidden_dtype(target_hidden), _hidden_dtype(draft_hidden))
 
     def _outputs(self, B, R, T, P, device, extras: bool, pin: bool = False):
         torch = self._torch

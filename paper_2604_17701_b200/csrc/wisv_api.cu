@@ -54,7 +54,9 @@ struct Plan {
 // error word comes back in one packed block (one copy), because at small batches a round is a few hundred
 // microseconds and each separate copy costs several of them in submission and DMA latency.
 struct HostStaging {
-    float* target_hidden = nullptr; float* draft_hidden = nullptr;
+    float* target_hidden = nullptr; float* draft_hidden = nullptr;   // sized for fp32 rows; 16-bit rows use half of it
+    cudaStream_t copy_stream = nullptr;            // large batches: hidden states travel group by group on this stream
+    cudaEvent_t copy_ev[8] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
     uint8_t* dev_in = nullptr;        // packed small inputs, layout chosen per call
     uint8_t* pin = nullptr;           // pinned, device-mapped host: [in_cap | out_cap]
     uint8_t* pin_dev = nullptr;       // the same block as the device sees it
@@ -400,6 +402,8 @@ void free_ctx(wisv_ctx* c)
     }
     HostStaging& h = c->hs;
     cudaFree(h.target_hidden); cudaFree(h.draft_hidden); cudaFree(h.dev_in);
+    for (int i = 0; i < 8; ++i) if (h.copy_ev[i]) cudaEventDestroy(h.copy_ev[i]);
+    if (h.copy_stream) cudaStreamDestroy(h.copy_stream);
     if (h.pin) cudaFreeHost(h.pin);
     (void)cudaGetLastError();
     delete c;
@@ -418,14 +422,16 @@ int dev_alloc(T** p, size_t n)
 // at most kZeroCopyBytes), else `staged`.
 constexpr size_t kZeroCopyBytes = 1u << 20;
 constexpr size_t kSmallInputsInPlace = 8u << 10;   // packed small inputs up to this size are not copied either
-const float* mapped_or(const float* host, size_t bytes, const float* staged)
+constexpr size_t kPipelineBytes = 32u << 20;       // host-buffer calls with at least this much hidden state travel in groups
+constexpr long long kPipelineFirstRows = 256;      // window rows of the first group; each later group is twice the one before
+const void* mapped_or(const void* host, size_t bytes, const void* staged)
 {
     if (!host || bytes == 0 || bytes > kZeroCopyBytes) return staged;
     cudaPointerAttributes at;
     if (cudaPointerGetAttributes(&at, host) != cudaSuccess) { (void)cudaGetLastError(); return staged; }
     if (at.type != cudaMemoryTypeHost || !at.devicePointer) return staged;
     if (reinterpret_cast<uintptr_t>(at.devicePointer) & 15u) return staged;
-    return static_cast<const float*>(at.devicePointer);
+    return at.devicePointer;
 }
 
 inline size_t pad16(size_t n) { return (n + 15) & ~size_t(15); }
@@ -444,11 +450,14 @@ size_t out_arena_layout(int B, int R, int T, int P, size_t* off)
 }
 
 // The same for the small inputs: k_off, draft_tokens, sel_off, sel_pos, csi, draft_q, uniforms.
-enum { IN_KOFF = 0, IN_TOK, IN_SELOFF, IN_SELPOS, IN_CSI, IN_Q, IN_U, IN_FIELDS };
+// IN_KOFF_G / IN_SELOFF_G: the offsets again, rebased to zero for each group of requests of a pipelined call.
+constexpr int kMaxCopyGroups = 8;
+enum { IN_KOFF = 0, IN_TOK, IN_SELOFF, IN_SELPOS, IN_CSI, IN_Q, IN_U, IN_KOFF_G, IN_SELOFF_G, IN_FIELDS };
 size_t in_arena_layout(int B, int T, int P, int d_c, size_t* off, size_t* bytes)
 {
     const size_t sz[IN_FIELDS] = {4u * ((size_t)B + 1), 4u * (size_t)T, 4u * ((size_t)B + 1), 4u * (size_t)P,
-                                  4u * (size_t)B * (size_t)d_c, 4u * (size_t)T, 4u * (size_t)T};
+                                  4u * (size_t)B * (size_t)d_c, 4u * (size_t)T, 4u * (size_t)T,
+                                  4u * ((size_t)B + kMaxCopyGroups), 4u * ((size_t)B + kMaxCopyGroups)};
     size_t at = 0;
     for (int i = 0; i < IN_FIELDS; ++i) { if (off) off[i] = at; if (bytes) bytes[i] = sz[i]; at += pad16(sz[i]); }
     return at;
@@ -462,6 +471,8 @@ int validate_batch(const wisv_ctx* c, const wisv_batch* b, const wisv_result* r,
     if (!c || !b || (!r && phase != PHASE_SHARD)) return WISV_EINVAL;
     if (b->B < 0 || b->K < 0) return WISV_ESHAPE;
     if (b->mode & ~3u) return WISV_EINVAL;
+    if (b->target_hidden_dtype < 0 || b->target_hidden_dtype > WISV_DT_F16 || b->draft_hidden_dtype < 0 ||
+        b->draft_hidden_dtype > WISV_DT_F16) return WISV_EINVAL;
     const bool sh = (b->mode & WISV_MODE_SH) != 0;
     const bool stoch = (b->mode & WISV_ACCEPT_STOCHASTIC) != 0;
     if (b->K == 0 && !b->k_off && b->B > 0 && b->T_total != 0) return WISV_EINVAL;
@@ -892,6 +903,7 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
     pp.ix = ix; pp.R = pack_rows; pp.P = P; pp.H = cf.H; pp.H_d = cf.H_d; pp.V = cf.V; pp.shift = cf.head_row_shift;
     pp.mode_sh = sh ? 1 : 0; pp.R_total = R; pp.T_total = T;
     pp.target_hidden = b->target_hidden; pp.draft_hidden = b->draft_hidden; pp.draft_tokens = b->draft_tokens;
+    pp.th_dtype = b->target_hidden_dtype; pp.dh_dtype = b->draft_hidden_dtype;
     pp.sel_off = b->sel_off; pp.sel_pos = b->sel_pos;
     pp.X = c->X; pp.Z = c->Z; pp.row_tok = c->row_tok; pp.row_flag = c->row_flag; pp.tok_logit = c->tok_logit;
     pp.pos_req = c->pos_req; pp.pos_i = c->pos_i;
@@ -1204,9 +1216,11 @@ int wisv_verify_host(wisv_ctx* c, const wisv_batch* hb, const wisv_result* hr, v
     db.k_off = hb->k_off ? reinterpret_cast<int32_t*>(in_base + ioff[IN_KOFF]) : nullptr;
     // a small hidden-state array in pinned memory is read in place by the pack kernel (one pass over PCIe, no
     // separate copy to wait for); a large or pageable one goes through the copy engine
-    const size_t th_bytes = sizeof(float) * (size_t)R * cf.H, dh_bytes = sizeof(float) * (size_t)P * cf.H_d;
-    const float* th_dev = mapped_or(hb->target_hidden, th_bytes, h.target_hidden);
-    const float* dh_dev = mapped_or(hb->draft_hidden, dh_bytes, h.draft_hidden);
+    auto elem = [](int dt) -> size_t { return dt == WISV_DT_F32 ? 4u : 2u; };
+    const size_t th_es = elem(hb->target_hidden_dtype), dh_es = elem(hb->draft_hidden_dtype);
+    const size_t th_bytes = th_es * (size_t)R * cf.H, dh_bytes = dh_es * (size_t)P * cf.H_d;
+    const void* th_dev = mapped_or(hb->target_hidden, th_bytes, h.target_hidden);
+    const void* dh_dev = mapped_or(hb->draft_hidden, dh_bytes, h.draft_hidden);
     db.target_hidden = hb->target_hidden ? th_dev : nullptr;
     db.draft_tokens = hb->draft_tokens ? reinterpret_cast<int32_t*>(in_base + ioff[IN_TOK]) : nullptr;
     db.draft_hidden = hb->draft_hidden ? dh_dev : nullptr;
@@ -1237,27 +1251,125 @@ int wisv_verify_host(wisv_ctx* c, const wisv_batch* hb, const wisv_result* hr, v
             if (kb < 0 || kb > WISV_MAX_K) return WISV_ESHAPE;
         }
     }
-    for (int i = 0; i < IN_FIELDS; ++i)
+    if (sh) {
+        if (hb->sel_off[0] != 0 || hb->sel_off[B] != P) return WISV_ESHAPE;
+        for (int i = 0; i < B; ++i)
+            if (hb->sel_off[i + 1] < hb->sel_off[i]) return WISV_ESHAPE;
+    }
+    // Large batches: the hidden states cross PCIe for milliseconds, and windows are verified independently (Section
+    // II-A), so the batch is cut into groups of whole requests, small ones first: group g is verified while group
+    // g + 1 is still on its way (copies on a stream of the context's own, one event per group).
+    int gb[kMaxCopyGroups + 1];
+    int n_groups = 1;
+    gb[0] = 0; gb[1] = B;
+    auto tok_of = [&](int b) { return hb->k_off ? (long long)hb->k_off[b] : (long long)b * hb->K; };
+    const bool staged = th_dev == h.target_hidden && (P == 0 || dh_dev == h.draft_hidden);
+    if (staged && th_bytes + dh_bytes >= kPipelineBytes && B >= 2) {
+        n_groups = 0;
+        long long target = kPipelineFirstRows, step = kPipelineFirstRows;
+        int prev = 0;
+        while (prev < B && n_groups < kMaxCopyGroups - 1) {
+            int b = prev + 1;
+            while (b < B && tok_of(b + 1) + b + 1 <= target) ++b;       // whole requests up to `target` window rows
+            if ((long long)R - (tok_of(b) + b) < 3 * kPipelineFirstRows) b = B;    // no small group at the end
+            gb[++n_groups] = b;
+            prev = b;
+            step *= 2; target += step;
+        }
+        if (prev < B) gb[++n_groups] = B;
+    }
+    if (n_groups > 1) {
+        // per-group offsets, rebased to zero, behind the plain ones in the packed block
+        int32_t* kg = reinterpret_cast<int32_t*>(pin_in + ioff[IN_KOFF_G]);
+        int32_t* sg = reinterpret_cast<int32_t*>(pin_in + ioff[IN_SELOFF_G]);
+        size_t at = 0;
+        for (int g = 0; g < n_groups; ++g)
+            for (int b = gb[g]; b <= gb[g + 1]; ++b, ++at) {
+                kg[at] = hb->k_off ? hb->k_off[b] - hb->k_off[gb[g]] : 0;
+                sg[at] = sh ? hb->sel_off[b] - hb->sel_off[gb[g]] : 0;
+            }
+    }
+    for (int i = 0; i < IN_KOFF_G; ++i)
         if (src[i] && ibytes[i] > 0) memcpy(pin_in + ioff[i], src[i], ibytes[i]);
     if (!small_in_place) WISV_CUDA(cudaMemcpyAsync(h.dev_in, pin_in, in_used, cudaMemcpyHostToDevice, st));
-    if (th_dev != h.target_hidden)
-        ;   // the pack kernel reads the caller's pinned array in place
-    else if (hb->target_hidden)
-        WISV_CUDA(cudaMemcpyAsync(h.target_hidden, hb->target_hidden, th_bytes, cudaMemcpyHostToDevice, st));
-    if (dh_dev != h.draft_hidden)
-        ;
-    else if (hb->draft_hidden && P > 0)
-        WISV_CUDA(cudaMemcpyAsync(h.draft_hidden, hb->draft_hidden, dh_bytes, cudaMemcpyHostToDevice, st));
     memset(pin_out, 0, 4);
-    c->err_copy_next = reinterpret_cast<int32_t*>(h.pin_dev + h.in_cap);
     // The merge/scan kernel stores a fresh sequence number next to the results when all of them are written;
     // watching that word costs less than a stream synchronisation at the end of a round of a few hundred
     // microseconds.  The stream is polled now and then as well, so a failed launch or kernel ends the wait.
     volatile int32_t* host_flag = reinterpret_cast<volatile int32_t*>(pin_out + 4);
     c->done_seq = c->done_seq == 0x7fffffff ? 1 : c->done_seq + 1;
     *host_flag = 0;
-    c->done_flag_next = reinterpret_cast<volatile int32_t*>(h.pin_dev + h.in_cap + 4);
-    const int rc = wisv_verify(c, &db, &dr, cuda_stream);
+    int rc = WISV_OK;
+    if (n_groups == 1) {
+        if (th_dev != h.target_hidden)
+            ;   // the pack kernel reads the caller's pinned array in place
+        else if (hb->target_hidden)
+            WISV_CUDA(cudaMemcpyAsync(h.target_hidden, hb->target_hidden, th_bytes, cudaMemcpyHostToDevice, st));
+        if (dh_dev != h.draft_hidden)
+            ;
+        else if (hb->draft_hidden && P > 0)
+            WISV_CUDA(cudaMemcpyAsync(h.draft_hidden, hb->draft_hidden, dh_bytes, cudaMemcpyHostToDevice, st));
+        c->err_copy_next = reinterpret_cast<int32_t*>(h.pin_dev + h.in_cap);
+        c->done_flag_next = reinterpret_cast<volatile int32_t*>(h.pin_dev + h.in_cap + 4);
+        rc = wisv_verify(c, &db, &dr, cuda_stream);
+    } else {
+        if (!h.copy_stream) {
+            WISV_CUDA(cudaStreamCreateWithFlags(&h.copy_stream, cudaStreamNonBlocking));
+            for (int i = 0; i < kMaxCopyGroups; ++i) WISV_CUDA(cudaEventCreateWithFlags(&h.copy_ev[i], cudaEventDisableTiming));
+        }
+        // the staging buffers were last read by the previous call, which had completed before it returned; the
+        // copies must still not overtake work the caller queued on `st` that this call's inputs may depend on
+        WISV_CUDA(cudaEventRecord(h.copy_ev[0], st));
+        WISV_CUDA(cudaStreamWaitEvent(h.copy_stream, h.copy_ev[0], 0));
+        const uint8_t* th_src = static_cast<const uint8_t*>(hb->target_hidden);
+        const uint8_t* dh_src = static_cast<const uint8_t*>(hb->draft_hidden);
+        uint8_t* th_dst = reinterpret_cast<uint8_t*>(h.target_hidden);
+        uint8_t* dh_dst = reinterpret_cast<uint8_t*>(h.draft_hidden);
+        size_t off_at = 0;
+        for (int g = 0; g < n_groups && rc == WISV_OK; ++g) {
+            const int b0 = gb[g], b1 = gb[g + 1];
+            const long long t0 = tok_of(b0), t1 = tok_of(b1);
+            const long long r0 = t0 + b0, r1 = t1 + b1;
+            const long long e0 = sh ? hb->sel_off[b0] : t0, e1 = sh ? hb->sel_off[b1] : t1;    // evaluated positions
+            const size_t row_b = th_es * cf.H, pos_b = dh_es * cf.H_d;
+            WISV_CUDA(cudaMemcpyAsync(th_dst + r0 * row_b, th_src + r0 * row_b, (size_t)(r1 - r0) * row_b,
+                                      cudaMemcpyHostToDevice, h.copy_stream));
+            if (e1 > e0)
+                WISV_CUDA(cudaMemcpyAsync(dh_dst + e0 * pos_b, dh_src + e0 * pos_b, (size_t)(e1 - e0) * pos_b,
+                                          cudaMemcpyHostToDevice, h.copy_stream));
+            WISV_CUDA(cudaEventRecord(h.copy_ev[g], h.copy_stream));
+            WISV_CUDA(cudaStreamWaitEvent(st, h.copy_ev[g], 0));
+            wisv_batch gbt = db;
+            wisv_result grs = dr;
+            gbt.B = b1 - b0;
+            gbt.T_total = (int32_t)(t1 - t0);
+            gbt.k_off = hb->k_off ? reinterpret_cast<int32_t*>(in_base + ioff[IN_KOFF_G]) + off_at : nullptr;
+            gbt.sel_off = sh ? reinterpret_cast<int32_t*>(in_base + ioff[IN_SELOFF_G]) + off_at : nullptr;
+            off_at += (size_t)(b1 - b0) + 1;
+            gbt.target_hidden = th_dst + r0 * row_b;
+            gbt.draft_hidden = hb->draft_hidden ? dh_dst + e0 * pos_b : nullptr;
+            gbt.draft_tokens = db.draft_tokens ? db.draft_tokens + t0 : nullptr;
+            gbt.sel_pos = db.sel_pos ? db.sel_pos + e0 : nullptr;
+            gbt.M_sel = sh ? (int32_t)(e1 - e0) : 0;
+            gbt.csi = db.csi ? db.csi + (size_t)b0 * cf.d_c : nullptr;
+            gbt.draft_q = db.draft_q ? db.draft_q + t0 : nullptr;
+            gbt.uniforms = db.uniforms ? db.uniforms + t0 : nullptr;
+            grs.accept_len = dr.accept_len + b0; grs.correction_token = dr.correction_token + b0;
+            if (dr.argmax) grs.argmax = dr.argmax + r0;
+            if (dr.lse) grs.lse = dr.lse + r0;
+            if (dr.p_draft) grs.p_draft = dr.p_draft + t0;
+            if (dr.head_prob) grs.head_prob = dr.head_prob + e0;
+            if (dr.mismatch_mask) grs.mismatch_mask = dr.mismatch_mask + b0;
+            if (dr.n_mismatch) grs.n_mismatch = dr.n_mismatch + b0;
+            if (dr.status) grs.status = dr.status + b0;
+            if (g == n_groups - 1) {
+                // the last group's merge/scan kernel mirrors the error word and announces completion
+                c->err_copy_next = reinterpret_cast<int32_t*>(h.pin_dev + h.in_cap);
+                c->done_flag_next = reinterpret_cast<volatile int32_t*>(h.pin_dev + h.in_cap + 4);
+            }
+            rc = wisv_verify(c, &gbt, &grs, cuda_stream);
+        }
+    }
     c->err_copy_next = nullptr;
     c->done_flag_next = nullptr;
     if (rc != WISV_OK) return rc;

@@ -10,6 +10,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <math_constants.h>
 #include <stdint.h>
 
@@ -41,8 +42,9 @@ struct PackParams {
     int32_t R, P, H, H_d, V, shift, mode_sh;
     int32_t R_total, T_total;     // window rows and draft tokens of the batch (bounds for indices derived from k_off)
     int32_t vocab_base, vocab_total;   // this context's LM-head rows are tokens [vocab_base, vocab_base + V) of vocab_total
-    const float* target_hidden;   // [R, H]
-    const float* draft_hidden;    // [P, H_d]
+    const void* target_hidden;    // [R, H], element type th_dtype (0 fp32, 1 bf16, 2 fp16)
+    const void* draft_hidden;     // [P, H_d], element type dh_dtype
+    int32_t th_dtype, dh_dtype;
     const int32_t* draft_tokens;  // [T]
     const int32_t* sel_off;       // [B+1] (SH)
     const int32_t* sel_pos;       // [P]   (SH)
@@ -83,6 +85,31 @@ __device__ __forceinline__ void cast_row(const float* __restrict__ src, __nv_bfl
     }
 }
 
+// 16-bit sources: bf16 rows are copied, fp16 rows converted (exactly) to fp32 and rounded to bf16; 8 elements per step
+__device__ __forceinline__ void copy_row_bf16(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst, int n) {
+    for (int i = threadIdx.x * 8; i < n; i += blockDim.x * 8)
+        *reinterpret_cast<uint4*>(dst + i) = *reinterpret_cast<const uint4*>(src + i);
+}
+__device__ __forceinline__ void cast_row_f16(const __half* __restrict__ src, __nv_bfloat16* __restrict__ dst, int n) {
+    for (int i = threadIdx.x * 8; i < n; i += blockDim.x * 8) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(src + i);
+        const __half2* h = reinterpret_cast<const __half2*>(&raw);
+        __nv_bfloat162 o[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const float2 f = __half22float2(h[u]);
+            o[u] = __floats2bfloat162_rn(f.x, f.y);
+        }
+        *reinterpret_cast<uint4*>(dst + i) = *reinterpret_cast<const uint4*>(o);
+    }
+}
+// row `row` (n elements) of a hidden-state array of the given element type -> bf16
+__device__ __forceinline__ void pack_row(const void* base, int dtype, size_t row, __nv_bfloat16* dst, int n) {
+    if (dtype == 0) cast_row(static_cast<const float*>(base) + row * n, dst, n);
+    else if (dtype == 1) copy_row_bf16(static_cast<const __nv_bfloat16*>(base) + row * n, dst, n);
+    else cast_row_f16(static_cast<const __half*>(base) + row * n, dst, n);
+}
+
 __global__ void __launch_bounds__(256) pack_kernel(const PackParams p)
 {
     __shared__ int s_src_row;
@@ -110,7 +137,7 @@ __global__ void __launch_bounds__(256) pack_kernel(const PackParams p)
             p.row_flag[r] = flag;
             p.tok_logit[r] = 0.0f;
         }
-        cast_row(p.target_hidden + (size_t)r * p.H, p.X + (size_t)r * p.H, p.H);
+        pack_row(p.target_hidden, p.th_dtype, (size_t)r, p.X + (size_t)r * p.H, p.H);
     } else {
         const int j = blk - p.R;          // evaluated position
         if (threadIdx.x == 0) {
@@ -132,8 +159,8 @@ __global__ void __launch_bounds__(256) pack_kernel(const PackParams p)
         }
         __syncthreads();
         const size_t zw = (size_t)(p.H_d + p.H);
-        cast_row(p.draft_hidden + (size_t)j * p.H_d, p.Z + (size_t)j * zw, p.H_d);
-        cast_row(p.target_hidden + (size_t)s_src_row * p.H, p.Z + (size_t)j * zw + p.H_d, p.H);
+        pack_row(p.draft_hidden, p.dh_dtype, (size_t)j, p.Z + (size_t)j * zw, p.H_d);
+        pack_row(p.target_hidden, p.th_dtype, (size_t)s_src_row, p.Z + (size_t)j * zw + p.H_d, p.H);
     }
 }
 

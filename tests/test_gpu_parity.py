@@ -583,6 +583,92 @@ def test_window_longer_than_the_limit_in_device_offsets_is_cut_and_flagged():
     v.close()
 
 
+def _as16(a, kind):
+    """numpy view of a hidden-state array in a 16-bit upload format, and the same as a torch CPU tensor."""
+    if kind == "f16":
+        h = np.ascontiguousarray(a, np.float32).astype(np.float16)
+        return h, torch.from_numpy(h.copy())
+    bits = gen.f32_to_bf16_bits(a)
+    return bits, torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16)
+
+
+@pytest.mark.parametrize("th,dh", [("bf16", "f16"), ("f16", "bf16"), ("f32", "f16"), ("bf16", "f32")])
+@pytest.mark.parametrize("kw", [dict(B=9, K=5), dict(B=30, K=6, mode="SH"), dict(B=70, K=0, K_lo=1, K_hi=7, V=3000)],
+                         ids=["R54", "R210_SH", "R350_ragged"])
+def test_sixteen_bit_hidden_states(kw, th, dh):
+    """The drafter uploads hidden states with 16 bits per element (Section IV-A); the target's may be 16-bit too.
+    bf16 is used as it is, fp16 is rounded to bf16 like fp32: against the oracle on the same 16-bit arrays, through
+    the device entry point and the host-buffer one."""
+    cfg = _small(seed=83, **kw)
+    case = cases.make_case(cfg, oracle_ref_argmax)
+    ocase, dev_t = dict(case), {}
+    for key, kind in (("target_hidden", th), ("draft_hidden", dh)):
+        if kind == "f32":
+            dev_t[key] = torch.from_numpy(np.ascontiguousarray(case[key]))
+        else:
+            ocase[key], dev_t[key] = _as16(case[key], kind)
+    ref = run_oracle(ocase)
+    d = cases.to_device(case, DEV)
+    d["target_hidden"], d["draft_hidden"] = dev_t["target_hidden"].to(DEV), dev_t["draft_hidden"].to(DEV)
+    v = cases.make_verifier(d)
+    out = cases.run(v, d)
+    torch.cuda.synchronize()
+    assert v.device_error() == 0
+    compare(ocase, ref, out, cfg.tau)
+    pin = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    ho = v.verify_host(dev_t["target_hidden"].pin_memory(), pin(case["draft_tokens"]), dev_t["draft_hidden"].pin_memory(),
+                       pin(case["csi"]), B=cfg.B, K=cfg.K if cfg.K_hi == 0 else 0,
+                       k_off=pin(case["k_off"]) if cfg.K_hi > 0 else None, T=case["T"], sel_off=pin(case["sel_off"]),
+                       sel_pos=pin(case["sel_pos"]), extras=True)
+    for k in ("accept_len", "correction_token", "argmax", "lse", "p_draft", "head_prob", "n_mismatch", "status"):
+        assert torch.equal(getattr(ho, k), getattr(out, k).cpu()), k
+    v.close()
+
+
+@pytest.mark.parametrize("kw", [dict(B=320, K=9), dict(B=520, K=0, K_lo=2, K_hi=12, mode="SH", stochastic=True),
+                                dict(B=380, K=9, h16=True)], ids=["uniform", "ragged_SH_stoch", "f16_uploads"])
+def test_host_entry_point_pipelines_large_batches_group_by_group(kw):
+    """More than 32 MB of hidden states: the host-buffer call cuts the batch into groups of whole requests and
+    verifies one group while the next is in flight.  Windows are independent, so the result must equal the oracle and
+    the one-piece device round (up to the fp32 summation order of the log-sum-exp, which follows the launch plan)."""
+    kw = dict(kw)
+    h16 = kw.pop("h16", False)
+    cfg = _small(seed=91, H=2048, H_d=1024, V=1000, d_J=64, **kw)
+    case = cases.make_case(cfg, oracle_ref_argmax)
+    if cfg.stochastic:
+        base = run_oracle(case)
+        case["draft_q"] = (base["p_draft"] * np.random.default_rng(5).uniform(0.5, 4.0, size=case["T"])).astype(np.float32)
+    ocase = dict(case)
+    th_t = torch.from_numpy(np.ascontiguousarray(case["target_hidden"]))
+    dh_t = torch.from_numpy(np.ascontiguousarray(case["draft_hidden"]))
+    if h16:
+        ocase["draft_hidden"], dh_t = _as16(case["draft_hidden"], "f16")
+    n_bytes = th_t.numel() * th_t.element_size() + dh_t.numel() * dh_t.element_size()
+    assert n_bytes > (32 << 20)
+    ref = run_oracle(ocase)
+    d = cases.to_device(case, DEV)
+    d["draft_hidden"] = dh_t.to(DEV)
+    v = cases.make_verifier(d)
+    out = cases.run(v, d)
+    torch.cuda.synchronize()
+    compare(ocase, ref, out, cfg.tau)
+    pin = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    n0 = v.launch_count()
+    for _ in range(2):                                   # twice: staging, events and offsets are reused
+        ho = v.verify_host(th_t.pin_memory(), pin(case["draft_tokens"]), dh_t.pin_memory(), pin(case["csi"]), B=cfg.B,
+                           K=cfg.K if cfg.K_hi == 0 else 0, k_off=pin(case["k_off"]) if cfg.K_hi > 0 else None,
+                           T=case["T"], sel_off=pin(case["sel_off"]), sel_pos=pin(case["sel_pos"]),
+                           draft_q=pin(case["draft_q"]), uniforms=pin(case["uniforms"]), extras=True)
+    assert v.launch_count() - n0 >= 2 * 3 * 3            # at least three groups of at least three kernels per call
+    assert v.device_error() == 0
+    compare(ocase, ref, ho, cfg.tau)
+    assert torch.equal(ho.argmax, out.argmax.cpu()) and torch.equal(ho.accept_len, out.accept_len.cpu())
+    assert torch.equal(ho.correction_token, out.correction_token.cpu()) and torch.equal(ho.mismatch_mask, out.mismatch_mask.cpu())
+    assert float((ho.lse - out.lse.cpu()).abs().max()) < 1e-4
+    assert float((ho.head_prob - out.head_prob.cpu()).abs().max()) < 1e-5
+    v.close()
+
+
 def test_capacity_and_argument_errors():
     cfg = _small(B=4, K=4)
     case = cases.make_case(cfg, oracle_ref_argmax)

@@ -380,3 +380,54 @@ def test_candidate_counts_with_empty_windows():
     assert out["n_mismatch"].tolist() == [2, 0, 1, 0, 0]
     assert out["accept_len"].tolist() == [0, 0, 0, 0, 0]
     assert np.array_equal(out["correction_token"], ref[[0, 3, 4, 6, 7]])     # first row of every window
+
+
+# ----------------------------------------------------------------------------- 16-bit hidden states (Section IV-A, b_h = 16)
+
+def test_sixteen_bit_hidden_states_follow_the_same_rounding_rule():
+    """fp16 uploads are widened exactly and then rounded to bf16 (nearest even) like fp32 inputs; bf16 uploads are used
+    as they are.  Second opinion: torch's own fp16 -> bf16 conversion and a float64 matmul."""
+    import torch
+    g = np.random.default_rng(12)
+    V, H, R = 64, 48, 6
+    W = gen.f32_to_bf16_bits(g.standard_normal((V, H), dtype=np.float32) * 0.1)
+    x16 = g.standard_normal((R, H)).astype(np.float16)
+    # halfway cases of the fp16 -> bf16 rounding: low three mantissa bits 100, kept bit even and odd
+    bits = x16.view(np.uint16).copy()
+    bits[0, :8] = (bits[0, :8] & np.uint16(0xFFF0)) | np.uint16(0x0004)       # kept bit 0: rounds down
+    bits[0, 8:16] = (bits[0, 8:16] & np.uint16(0xFFF0)) | np.uint16(0x000C)   # kept bit 1: rounds up
+    x16 = bits.view(np.float16)
+    got = oracle.lm_head(W, oracle.hidden_as_f32(x16), want_logits=True)["logits"]
+    xt = torch.from_numpy(x16.copy()).to(torch.bfloat16).to(torch.float64)       # library conversion, nearest even
+    Wt = torch.from_numpy(gen.bf16_bits_to_f32(W)).to(torch.float64)
+    assert np.allclose(got, (xt @ Wt.T).numpy(), rtol=0, atol=1e-12)
+    # the two halfway groups really round in different directions
+    r = xt[0].numpy()
+    lo = x16[0].astype(np.float64)
+    assert np.all(np.abs(r[:8]) < np.abs(lo[:8])) and np.all(np.abs(r[8:16]) > np.abs(lo[8:16]))
+    # bf16 bit patterns are taken as they are
+    xb = gen.f32_to_bf16_bits(g.standard_normal((R, H), dtype=np.float32))
+    a = oracle.lm_head(W, oracle.hidden_as_f32(xb), want_logits=True)["logits"]
+    b = oracle.lm_head(W, gen.bf16_bits_to_f32(xb), want_logits=True)["logits"]
+    assert np.array_equal(a, b)
+    assert np.allclose(a, (torch.from_numpy(gen.bf16_bits_to_f32(xb)).to(torch.float64) @ Wt.T).numpy(), rtol=0, atol=1e-12)
+
+
+def test_round_with_sixteen_bit_uploads_equals_round_on_their_fp32_values():
+    cfg = gen.VerifyConfig("h16", B=5, K=4, H=64, H_d=32, d_c=2, d_J=32, V=300, match_rate=0.5, seed=77)
+    k_len = gen.synth.window_lengths(cfg)
+    w = gen.make_weights(cfg)
+    h = gen.make_hidden(cfg, k_len)
+    ref_am = oracle.lm_head(w["lm_head"], h["target_hidden"])["argmax"]
+    toks = gen.make_draft_tokens(cfg, k_len, ref_am)
+    kw = dict(lm_head_bits=w["lm_head"], W1_bits=w["W1"], b1=w["b1"], w2=w["w2"], b2=float(w["b2"]), act=oracle.ACT_GELU,
+              tau=0.5, k_len=k_len, draft_tokens=toks, csi=h["csi"])
+    hd16 = h["draft_hidden"].astype(np.float16)
+    ht_bits = gen.f32_to_bf16_bits(h["target_hidden"])
+    a = oracle.verify(target_hidden=ht_bits, draft_hidden=hd16, **kw)
+    b = oracle.verify(target_hidden=gen.bf16_bits_to_f32(ht_bits), draft_hidden=hd16.astype(np.float32), **kw)
+    for k in ("accept_len", "correction_token", "argmax", "lse", "head_prob", "p_draft"):
+        assert np.array_equal(a[k], b[k]), k
+    # and the fp16 upload is a different input from the fp32 original: the head sees the rounded values
+    c = oracle.verify(target_hidden=gen.bf16_bits_to_f32(ht_bits), draft_hidden=h["draft_hidden"], **kw)
+    assert np.max(np.abs(c["head_logit"] - a["head_logit"])) > 0
