@@ -43,14 +43,14 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 SINGLE_CTA_SOURCES = ("wisv_gemm.cuh", "wisv_ptx.cuh")
 CTA_PAIR_SOURCES = ("wisv_gemm2.cuh", "wisv_gemm.cuh", "wisv_ptx.cuh")
 NCU_TRAFFIC = {
-    # LM-head and decision-head CTAs in one launch, 9 window rows: 1.0642 GB read + 4.9 MB written per launch
-    "8b_b1": {"bytes": 1069100000, "files": SINGLE_CTA_SOURCES, "kernel_hash": "eed3461d3bffc1f3"},
-    # CTA pairs + decision-head clusters, 144 window rows: 1.0829 GB read + 3.8 MB written per launch
-    "8b_b16": {"bytes": 1086800000, "files": CTA_PAIR_SOURCES, "kernel_hash": "26e869a2e0a21f84"},
-    # single-CTA kernel, 576 window rows: 1.0584 GB read + 8.3 MB written per launch
-    "8b_b64": {"bytes": 1066600000, "files": SINGLE_CTA_SOURCES, "kernel_hash": "eed3461d3bffc1f3"},
-    # CTA-pair kernel, 8704 window rows: 3.263 GB read + 72.8 MB written per launch (3.3-8.5 GB between captures)
-    "8b_b512": {"bytes": 3335600000, "files": CTA_PAIR_SOURCES, "kernel_hash": "26e869a2e0a21f84"},
+    # LM-head and decision-head CTAs in one launch, 9 window rows: 1.0642 GB read + 4.0-5.9 MB written per launch
+    "8b_b1": {"bytes": 1069100000, "files": SINGLE_CTA_SOURCES, "kernel_hash": "94d71ebe0866b145"},
+    # CTA pairs (one row block of 144) + decision-head clusters: 1.0763 GB read + 3.6-6.2 MB written per launch
+    "8b_b16": {"bytes": 1081200000, "files": CTA_PAIR_SOURCES, "kernel_hash": "4a707a11da85279b"},
+    # CTA pairs (three row blocks of 192) + decision-head clusters: 1.1362 GB read + 12.3 MB written per launch
+    "8b_b64": {"bytes": 1148500000, "files": CTA_PAIR_SOURCES, "kernel_hash": "4a707a11da85279b"},
+    # CTA pairs (34 row blocks of 256): 3.49-3.59 GB read + 138-142 MB written (the partials) per launch
+    "8b_b512": {"bytes": 3681000000, "files": CTA_PAIR_SOURCES, "kernel_hash": "4a707a11da85279b"},
 }
 
 
@@ -530,10 +530,8 @@ def measure(cfg, w, wdev, args, rank, world, local_rank, ranks, with_baseline, b
 
 
 def lm_kernel_name(R, one_launch):
-    # which LM-head kernel the library's plan uses (same rule as the planner: CTA pairs for an even number of
-    # 128-row tiles or at least 11 of them)
-    tiles128 = -(-R // 128)
-    on_pairs = tiles128 >= 2 and (tiles128 % 2 == 0 or tiles128 >= 11)
+    # which LM-head kernel the library's plan uses: single CTAs up to 128 window rows, CTA pairs above
+    on_pairs = R > 128
     if one_launch:
         return ("lmhead_pair_kernel (CTA pairs + decision-head clusters)" if on_pairs
                 else "round_small_kernel (LM-head CTAs + decision-head CTAs)")
