@@ -121,7 +121,7 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [0] abort, [1] drain scratch
     float* trans_base = reinterpret_cast<float*>(smem + ring_bytes + 1024);      // 4 x [32 columns][36]
 
-    const int warp = threadIdx.x >> 5;
+    const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0);   // the same in all lanes, and the compiler knows it
     const int lane = threadIdx.x & 31;
     // carry: this pair's contiguous range of 32-row units and how it is cut into tiles
     const int my_units = p.units_base + (pair_id < p.units_rem ? 1 : 0);
@@ -189,30 +189,33 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (each CTA)
-        // One pass of this loop (barrier test, expect_tx, TMA issues: each a round trip of its own) costs the thread
-        // about 500 clocks whatever the tile sizes, more than the MMAs of one K block take when the row block is
-        // narrow; a stage of kbs K blocks spreads that over kbs blocks.  Plain counters and nested loops only: a 64-bit
-        // division per K block in this loop doubled the kernel's time.
+        // The WHOLE warp runs these loops and one elected lane issues: tcgen05.mma, tcgen05.commit and the TMA
+        // instructions take their operands from uniform registers, which the compiler can only use in code that the
+        // warp runs together.  Written as the work of one thread inside `if (lane == 0)`, the same loops cost 470
+        // clocks per stage plus 75 per TMA issue here and 57-74 clocks per MMA in the warp below (measured), more
+        // than the tensor pipe needs for the MMAs of a narrow row block.  Plain counters and nested loops only: a
+        // 64-bit division per K block in this loop doubled the kernel's time.
         Item w;
         int pre = 0;                               // stages whose weight half-tiles were requested before the wait
-        if (lane == 0) {
-            for (int i = 0; pre < p.stages && item_at(i, w); ++i) {
-                const int half_h = w.h >> 1;
-                const int w_row0 = w.n0 + static_cast<int>(rank) * half_h;
-                const CUtensorMap* mapW = (w.h == p.tile_m) ? &tmW : &tmW2;
-                for (int kb = 0; kb < p.k_blocks && pre < p.stages; kb += p.kbs, ++pre) {
-                    const int nb = min(p.kbs, p.k_blocks - kb);
-                    const uint32_t dst = smem_base + stage_bytes * static_cast<uint32_t>(pre);
-                    if (leader)                    // both CTAs' bytes
-                        mbar_expect_tx(full_bar(pre), 2u * static_cast<uint32_t>(nb) * (static_cast<uint32_t>(half_h) * kBlockK * 2u + b_bytes));
+        for (int i = 0; pre < p.stages && item_at(i, w); ++i) {
+            const int half_h = w.h >> 1;
+            const int w_row0 = w.n0 + static_cast<int>(rank) * half_h;
+            const CUtensorMap* mapW = (w.h == p.tile_m) ? &tmW : &tmW2;
+            for (int kb = 0; kb < p.k_blocks && pre < p.stages; kb += p.kbs, ++pre) {
+                const int nb = min(p.kbs, p.k_blocks - kb);
+                const uint32_t dst = smem_base + stage_bytes * static_cast<uint32_t>(pre);
+                const uint32_t tx = 2u * static_cast<uint32_t>(nb) * (static_cast<uint32_t>(half_h) * kBlockK * 2u + b_bytes);
+                if (elect_one()) {
+                    if (leader) mbar_expect_tx(full_bar(pre), tx);          // both CTAs' bytes
                     for (int u = 0; u < nb; ++u)
                         tma_load_2d_pair(dst + static_cast<uint32_t>(u) * a_bytes, mapW, (kb + u) * kBlockK, w_row0, full_bar(pre));
                 }
+                __syncwarp();
             }
         }
         griddep_wait();
         griddep_launch_dependents();
-        if (lane == 0) {
+        {
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
@@ -221,26 +224,35 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 const int w_row0 = w.n0 + static_cast<int>(rank) * half_h;
                 const int x_row0 = w.j * p.n_cols + static_cast<int>(rank) * (p.n_cols / 2);   // its half of the row block
                 const CUtensorMap* mapW = (w.h == p.tile_m) ? &tmW : &tmW2;
+                const uint32_t tx_w = static_cast<uint32_t>(half_h) * kBlockK * 2u + b_bytes;
                 for (int kb = 0; kb < p.k_blocks; kb += p.kbs) {
                     const int nb = min(p.kbs, p.k_blocks - kb);
                     const uint32_t dst = smem_base + stage_bytes * static_cast<uint32_t>(s);
-                    if (prod_issued >= pre) {
-                        if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, kWaitLimitClocks)) { ok = false; break; }
-                        if (leader)
-                            mbar_expect_tx(full_bar(s), 2u * static_cast<uint32_t>(nb) * (static_cast<uint32_t>(half_h) * kBlockK * 2u + b_bytes));
+                    const bool fresh = prod_issued >= pre;    // else: first pass over the ring, the stage is free and
+                                                              // its weight half-tiles are on their way
+                    if (fresh) {
+                        ok = __all_sync(0xffffffffu, mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, kWaitLimitClocks));
+                        if (!ok) break;
+                    }
+                    if (elect_one()) {
+                        if (fresh) {
+                            if (leader) mbar_expect_tx(full_bar(s), 2u * static_cast<uint32_t>(nb) * tx_w);
+                            for (int u = 0; u < nb; ++u)
+                                tma_load_2d_pair(dst + static_cast<uint32_t>(u) * a_bytes, mapW, (kb + u) * kBlockK, w_row0, full_bar(s));
+                        }
                         for (int u = 0; u < nb; ++u)
-                            tma_load_2d_pair(dst + static_cast<uint32_t>(u) * a_bytes, mapW, (kb + u) * kBlockK, w_row0, full_bar(s));
-                    }   // else: first pass over the ring, the stage is free and its weight half-tiles are on their way
-                    for (int u = 0; u < nb; ++u)
-                        tma_load_2d_pair(dst + x_off + static_cast<uint32_t>(u) * b_bytes, &tmX, (kb + u) * kBlockK, x_row0, full_bar(s));
+                            tma_load_2d_pair(dst + x_off + static_cast<uint32_t>(u) * b_bytes, &tmX, (kb + u) * kBlockK, x_row0, full_bar(s));
+                    }
+                    __syncwarp();
                     ++prod_issued;
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer (leader CTA only)
-        if (lane == 0 && leader) {
+        // ------------------------------------------------------------ MMA issuer (leader CTA only; see the producer
+        // for why the whole warp runs the loop)
+        if (leader) {
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
@@ -250,28 +262,37 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             for (int local = 0; ok && item_at(local, w); ++local) {
                 const int as = local & 1;
                 const uint32_t aph = (local >> 1) & 1u;
-                if (!mbar_wait_bounded(acc_empty_bar(as), aph ^ 1u, abort_flag, kWaitLimitClocks)) { ok = false; break; }
+                ok = __all_sync(0xffffffffu, mbar_wait_bounded(acc_empty_bar(as), aph ^ 1u, abort_flag, kWaitLimitClocks));
+                if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(as * kAccCols);
                 for (int kb = 0; kb < p.k_blocks; kb += p.kbs) {
                     const int nb = min(p.kbs, p.k_blocks - kb);
-                    if (!mbar_wait_bounded(full_bar(s), ph, abort_flag, kWaitLimitClocks)) { ok = false; break; }
+                    ok = __all_sync(0xffffffffu, mbar_wait_bounded(full_bar(s), ph, abort_flag, kWaitLimitClocks));
+                    if (!ok) break;
                     tc_fence_after();
                     const uint32_t st_addr = smem_base + stage_bytes * s;
-                    for (int u = 0; u < nb; ++u) {
-                        const uint64_t a_desc = smem_desc_k128(st_addr + static_cast<uint32_t>(u) * a_bytes);          // weights: the M side
-                        const uint64_t b_desc = smem_desc_k128(st_addr + x_off + static_cast<uint32_t>(u) * b_bytes);  // window rows: the N side
+                    const uint64_t a_desc0 = smem_desc_k128(st_addr);             // weights: the M side
+                    const uint64_t b_desc0 = smem_desc_k128(st_addr + x_off);     // window rows: the N side
+                    const bool last = kb + nb >= p.k_blocks;
+                    if (elect_one()) {
+                        for (int u = 0; u < nb; ++u) {
+                            const uint64_t a_desc = a_desc0 + static_cast<uint64_t>((static_cast<uint32_t>(u) * a_bytes) >> 4);
+                            const uint64_t b_desc = b_desc0 + static_cast<uint64_t>((static_cast<uint32_t>(u) * b_bytes) >> 4);
 #pragma unroll
-                        for (int k = 0; k < kBlockK / kUmmaK; ++k)
-                            umma_bf16_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | u | k) != 0 ? 1u : 0u);
+                            for (int k = 0; k < kBlockK / kUmmaK; ++k)
+                                umma_bf16_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | u | k) != 0 ? 1u : 0u);
+                        }
+                        umma_commit_pair(empty_bar(s));                    // frees the stage in both CTAs
+                        if (last) umma_commit_pair(acc_full_bar(as));      // accumulator ready in both CTAs
                     }
-                    umma_commit_pair(empty_bar(s));          // frees the stage in both CTAs
+                    __syncwarp();
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
-                if (ok) umma_commit_pair(acc_full_bar(as));  // accumulator ready in both CTAs
             }
             if (!ok) {
-                umma_commit_pair(drain_bar);
+                if (elect_one()) umma_commit_pair(drain_bar);
+                __syncwarp();
                 mbar_wait_bounded(drain_bar, 0, abort_flag + 1, kWaitLimitClocks);
             }
         }
