@@ -162,7 +162,7 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
     volatile int* last_flag = abort_flag + 2;                                    // split-K: this CTA finishes the tile
     float* epi_const = reinterpret_cast<float*>(smem + ring_bytes + 1024);
 
-    const int warp = threadIdx.x >> 5;
+    const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0);   // the same in all lanes, and the compiler knows it
     const int lane = threadIdx.x & 31;
     const int total_tiles = p.m_tiles * p.n_tiles * p.k_splits;      // work items
     // item t -> row tile m (fastest), K split ks, column tile n
@@ -237,91 +237,103 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
+        // The whole warp runs the loops and one elected lane issues.  The TMA, tcgen05.mma and tcgen05.commit
+        // instructions take their operands from uniform registers, which exist only for code the warp runs
+        // together: the same loops written as one thread's work (`if (lane == 0)`) cost about twice the clocks
+        // per stage here and 57-74 clocks per MMA in the warp below (measured), more than narrow MMAs take.
         long long pre = 0;                     // stages whose weight tile was requested before the wait
         Item w;
         if (!kWaitLast) {
-            if (lane == 0) {
-                for (int i = 0; pre < p.stages && item_at(i, w); ++i) {
-                    const uint32_t tx = a_bytes + static_cast<uint32_t>(w.h) * kBlockK * 2;
-                    for (int kb = w.kb0; kb < w.kb1 && pre < p.stages; ++kb, ++pre) {
-                        const uint32_t a_dst = smem_base + stage_bytes * static_cast<uint32_t>(pre);
+            for (int i = 0; pre < p.stages && item_at(i, w); ++i) {
+                const uint32_t tx = a_bytes + static_cast<uint32_t>(w.h) * kBlockK * 2;
+                for (int kb = w.kb0; kb < w.kb1 && pre < p.stages; ++kb, ++pre) {
+                    const uint32_t a_dst = smem_base + stage_bytes * static_cast<uint32_t>(pre);
+                    if (elect_one()) {
                         mbar_expect_tx(full_bar(static_cast<int>(pre)), tx);
                         tma_load_2d(a_dst + a_bytes, b_map(w.h), kb * kBlockK, w.n0, full_bar(static_cast<int>(pre)));
                     }
+                    __syncwarp();
                 }
             }
             griddep_wait();                    // from here on the activation rows may be read
             griddep_launch_dependents();
         }
-        if (lane == 0) {
-            int s = 0;
-            uint32_t ph = 0;
-            long long issued = 0;
-            bool ok = true;
-            for (int i = 0; ok && item_at(i, w); ++i) {
-                const uint32_t tx = a_bytes + static_cast<uint32_t>(w.h) * kBlockK * 2;
-                for (int kb = w.kb0; kb < w.kb1; ++kb) {
-                    const uint32_t a_dst = smem_base + stage_bytes * s;
-                    if (issued < pre) {
-                        // first pass over the ring: the stage is free and its weight tile is already on its way
-                        tma_load_2d(a_dst, &tmA, kb * kBlockK, w.m * kTileM, full_bar(s));
-                    } else {
-                        if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, kWaitLimitClocks)) { ok = false; break; }
-                        mbar_expect_tx(full_bar(s), tx);
-                        tma_load_2d(a_dst, &tmA, kb * kBlockK, w.m * kTileM, full_bar(s));
-                        tma_load_2d(a_dst + a_bytes, b_map(w.h), kb * kBlockK, w.n0, full_bar(s));
-                    }
-                    ++issued;
-                    if (++s == p.stages) { s = 0; ph ^= 1u; }
+        int s = 0;
+        uint32_t ph = 0;
+        long long issued = 0;
+        bool ok = true;
+        for (int i = 0; ok && item_at(i, w); ++i) {
+            const uint32_t tx = a_bytes + static_cast<uint32_t>(w.h) * kBlockK * 2;
+            const CUtensorMap* mapB = b_map(w.h);
+            for (int kb = w.kb0; kb < w.kb1; ++kb) {
+                const uint32_t a_dst = smem_base + stage_bytes * s;
+                // not fresh: first pass over the ring, the stage is free and its weight tile is already on its way
+                const bool fresh = issued >= pre;
+                if (fresh) {
+                    ok = __all_sync(0xffffffffu, mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, kWaitLimitClocks));
+                    if (!ok) break;
                 }
+                if (elect_one()) {
+                    if (fresh) mbar_expect_tx(full_bar(s), tx);
+                    tma_load_2d(a_dst, &tmA, kb * kBlockK, w.m * kTileM, full_bar(s));
+                    if (fresh) tma_load_2d(a_dst + a_bytes, mapB, kb * kBlockK, w.n0, full_bar(s));
+                }
+                __syncwarp();
+                ++issued;
+                if (++s == p.stages) { s = 0; ph ^= 1u; }
             }
-            if (!ok) {
-                // let copies already in flight land before the CTA retires
-                const int inflight = issued < p.stages ? static_cast<int>(issued) : p.stages;
-                int ws = s;
-                uint32_t wph = ph;
-                for (int i = 0; i < inflight; ++i) {
-                    if (--ws < 0) { ws = p.stages - 1; wph ^= 1u; }
-                    mbar_wait_bounded(full_bar(ws), wph, abort_flag + 1, kWaitLimitClocks);
-                }
+        }
+        if (!ok) {
+            // let copies already in flight land before the CTA retires
+            const int inflight = issued < p.stages ? static_cast<int>(issued) : p.stages;
+            int ws = s;
+            uint32_t wph = ph;
+            for (int i = 0; i < inflight; ++i) {
+                if (--ws < 0) { ws = p.stages - 1; wph ^= 1u; }
+                mbar_wait_bounded(full_bar(ws), wph, abort_flag + 1, kWaitLimitClocks);
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            int s = 0;
-            uint32_t ph = 0;
-            bool ok = true;
-            Item w;
-            for (int local = 0; ok && item_at(local, w); ++local) {
-                const uint32_t idesc = idesc_bf16_f32(static_cast<uint32_t>(tile_mma_m(w.m)), static_cast<uint32_t>(w.h));
-                const int as = local & 1;
-                const uint32_t aph = (local >> 1) & 1u;
-                if (!mbar_wait_bounded(acc_empty_bar(as), aph ^ 1u, abort_flag, kWaitLimitClocks)) { ok = false; break; }
+        // ------------------------------------------------------------ MMA issuer (whole warp, one elected lane: see
+        // the producer)
+        int s = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        Item w;
+        for (int local = 0; ok && item_at(local, w); ++local) {
+            const uint32_t idesc = idesc_bf16_f32(static_cast<uint32_t>(tile_mma_m(w.m)), static_cast<uint32_t>(w.h));
+            const int as = local & 1;
+            const uint32_t aph = (local >> 1) & 1u;
+            ok = __all_sync(0xffffffffu, mbar_wait_bounded(acc_empty_bar(as), aph ^ 1u, abort_flag, kWaitLimitClocks));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(as * kAccCols);
+            const int kb0 = w.kb0, kb1 = w.kb1;
+            for (int kb = kb0; kb < kb1; ++kb) {
+                ok = __all_sync(0xffffffffu, mbar_wait_bounded(full_bar(s), ph, abort_flag, kWaitLimitClocks));
+                if (!ok) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(as * kAccCols);
-                const int kb0 = w.kb0, kb1 = w.kb1;
-                for (int kb = kb0; kb < kb1; ++kb) {
-                    if (!mbar_wait_bounded(full_bar(s), ph, abort_flag, kWaitLimitClocks)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t a_addr = smem_base + stage_bytes * s;
-                    const uint64_t a_desc = smem_desc_k128(a_addr);
-                    const uint64_t b_desc = smem_desc_k128(a_addr + a_bytes);
+                const uint32_t a_addr = smem_base + stage_bytes * s;
+                const uint64_t a_desc = smem_desc_k128(a_addr);
+                const uint64_t b_desc = smem_desc_k128(a_addr + a_bytes);
+                if (elect_one()) {
 #pragma unroll
                     for (int k = 0; k < kBlockK / kUmmaK; ++k) {
                         // advancing K by 16 bf16 = 32 bytes = 2 descriptor units inside the swizzle atom
                         umma_bf16(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, ((kb - kb0) | k) != 0 ? 1u : 0u);
                     }
                     umma_commit(empty_bar(s));       // stage is free once these MMAs have read it
-                    if (++s == p.stages) { s = 0; ph ^= 1u; }
+                    if (kb + 1 == kb1) umma_commit(acc_full_bar(as));
                 }
-                if (ok) umma_commit(acc_full_bar(as));
+                __syncwarp();
+                if (++s == p.stages) { s = 0; ph ^= 1u; }
             }
-            if (!ok) {
-                // drain whatever was issued before TMEM is released
-                umma_commit(drain_bar);
-                mbar_wait_bounded(drain_bar, 0, abort_flag + 1, kWaitLimitClocks);
-            }
+        }
+        if (!ok) {
+            // drain whatever was issued before TMEM is released
+            if (elect_one()) umma_commit(drain_bar);
+            __syncwarp();
+            mbar_wait_bounded(drain_bar, 0, abort_flag + 1, kWaitLimitClocks);
         }
     } else {
         // ------------------------------------------------------------ epilogue (warps 2..5)
