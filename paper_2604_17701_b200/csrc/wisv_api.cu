@@ -542,9 +542,11 @@ PairParams pair_params(const wisv_ctx* c, const Plan& pl, int R)
     sp.rows = R; sp.n_cols = pl.n_cols; sp.row_blocks = pl.n_blocks; sp.n_total = cf.V;
     sp.k_blocks = (cf.H + kBlockK - 1) / kBlockK; sp.carry = pl.carry; sp.n_tiles = pl.n_tiles;
     {
-        // raster groups: keep a group's bf16 rows within 32 MB of L2 while the weights stream past them
+        // raster groups: keep a group's bf16 rows within 48 MB of L2 while the weights stream past them (measured at
+        // 8704 rows: 3 groups of 25 MB and 2 of 36 MB read 4-6.5 GB and 2.6-5.4 GB from HBM per launch, the second
+        // 1 % faster; one group of 71 MB reads 11 GB and is 10 % slower)
         const long long block_bytes = (long long)pl.n_cols * cf.H * 2;
-        int bg_max = (int)((32ll << 20) / block_bytes);
+        int bg_max = (int)((48ll << 20) / block_bytes);
         if (bg_max < 1) bg_max = 1;
         const int groups = (pl.n_blocks + bg_max - 1) / bg_max;
         sp.b_group = (pl.n_blocks + groups - 1) / groups;
