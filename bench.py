@@ -474,6 +474,17 @@ def measure(cfg, w, wdev, args, rank, world, local_rank, ranks, with_baseline, b
     h2d = sum(int(t.numel() * t.element_size()) for t in list(hc.values()) + [hk] if t is not None)
     d2h = 2 * 4 * cfg.B
     same = bool(torch.equal(host_out.accept_len, fast_out.accept_len.cpu()))
+    # ---- (3b) the same call with the hidden states as the uplink delivers them (Section IV-A: b_h = 16 bits per
+    # element): the drafter's as fp16, the target's as bf16; half the bytes cross PCIe
+    hc16 = dict(hc)
+    hc16["target_hidden"] = hc["target_hidden"].to(torch.bfloat16).pin_memory()
+    hc16["draft_hidden"] = hc["draft_hidden"].to(torch.float16).pin_memory()
+    host_call16 = v.bind_host(hc16["target_hidden"], hc16["draft_tokens"], hc16["draft_hidden"], hc16["csi"], **hkw)
+    for _ in range(min(args.warmup, 10) + 1):
+        host_call16()
+    e2e16_regions = [region(host_call16, steps) for _ in range(e2e_repeats)]
+    e2e16_ms = float(statistics.median(e2e16_regions))
+    h2d16 = sum(int(t.numel() * t.element_size()) for t in list(hc16.values()) + [hk] if t is not None)
     clocks = sampler.stop() if rank == 0 else None
 
     rec = None
@@ -518,7 +529,12 @@ def measure(cfg, w, wdev, args, rank, world, local_rank, ranks, with_baseline, b
                "clocks": clocks, "gpu_launches": int(launches),
                "e2e": {"value": aggregate(world, T, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                        "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": steps, "repeats": e2e_repeats,
-                       "ms_per_step_regions": region_stats(e2e_regions), "matches_device_path": same},
+                       "ms_per_step_regions": region_stats(e2e_regions), "matches_device_path": same,
+                       "hidden_dtype": "f32",
+                       "sixteen_bit_hidden": {"value": aggregate(world, T, e2e16_ms), "unit": UNIT,
+                                              "ms_per_step": e2e16_ms, "h2d_bytes_per_step": h2d16,
+                                              "d2h_bytes_per_step": d2h, "hidden_dtype": "target bf16, draft f16",
+                                              "ms_per_step_regions": region_stats(e2e16_regions)}},
                "roofline": roof,
                "accepted_tokens_per_s": world * dec["accepted_tokens"] / (ms_step * 1e-3),
                "decisions": dec}
