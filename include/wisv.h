@@ -268,6 +268,9 @@ typedef struct {
                                 there (0 = chosen automatically), -1 = always two launches */
     int32_t lm_mma_m;        /* 128: never use 64-row MMAs (the default for GEMMs with at most 64 valid rows) */
     int32_t lm_kb_per_stage; /* CTA-pair LM-head kernel: K blocks (of 64) per shared-memory stage: 1, 2 or 4 */
+    int32_t lm_teams;        /* CTA-pair LM-head kernel with 2 or more row blocks: 1 = one team of pairs per row block,
+                                each dealing out the whole vocabulary with carried row state (whenever all window rows
+                                fit in L2), -1 = never (round-robin work items), 0 = chosen automatically */
 } wisv_tuning;
 int wisv_set_tuning(wisv_ctx* ctx, const wisv_tuning* tuning);
 

@@ -68,7 +68,7 @@ class _Result(C.Structure):
 class _Tuning(C.Structure):
     _fields_ = [("lm_tile_n", C.c_int32), ("lm_stages", C.c_int32), ("head_tile_n", C.c_int32),
                 ("head_stages", C.c_int32), ("lm_single_cta", C.c_int32), ("head_ctas", C.c_int32),
-                ("lm_mma_m", C.c_int32), ("lm_kb_per_stage", C.c_int32)]
+                ("lm_mma_m", C.c_int32), ("lm_kb_per_stage", C.c_int32), ("lm_teams", C.c_int32)]
 
 
 class LinkParams(C.Structure):
@@ -482,8 +482,9 @@ class Verifier:
         return n
 
     def set_tuning(self, lm_tile_n: int = 0, lm_stages: int = 0, head_tile_n: int = 0, head_stages: int = 0,
-                   lm_single_cta: int = 0, head_ctas: int = 0, lm_mma_m: int = 0, lm_kb_per_stage: int = 0):
-        t = _Tuning(lm_tile_n, lm_stages, head_tile_n, head_stages, lm_single_cta, head_ctas, lm_mma_m, lm_kb_per_stage)
+                   lm_single_cta: int = 0, head_ctas: int = 0, lm_mma_m: int = 0, lm_kb_per_stage: int = 0, lm_teams: int = 0):
+        t = _Tuning(lm_tile_n, lm_stages, head_tile_n, head_stages, lm_single_cta, head_ctas, lm_mma_m, lm_kb_per_stage,
+                    lm_teams)
         _check(self.lib.wisv_set_tuning(self._h, C.byref(t)), "wisv_set_tuning")
 
     def launch_count(self) -> int:

@@ -32,6 +32,7 @@ constexpr int kNumRowVariants = kTileM / 8;        // a_rows = 8, 16, ..., 128
 constexpr int kStages = 4;                         // profiled stages per call
 constexpr int kSplitTileN = 64;                    // head tile height when K is split over CTAs
 constexpr int kSplitMaxRowTiles = 4;               // K is split for decision heads of up to this many row tiles
+constexpr long long kTeamRowBytes = 32ll << 20;    // CTA-pair LM head: teams only while all bf16 window rows fit in this
 constexpr int kPairKbPerStage = 2;                 // CTA-pair LM head: K blocks per shared-memory stage
 
 struct Plan {
@@ -43,6 +44,7 @@ struct Plan {
     int n_cols;      // pairs: N of the MMA = width of a row block (a multiple of 16)
     int n_blocks;    // pairs: row blocks of n_cols rows
     int kbs;         // pairs: K blocks per shared-memory stage
+    int team_pairs;  // pairs with carried ranges: pairs per team (one team per row block)
     int k_splits;    // work items per (m, n) tile along K (decision head with one row tile)
     int kb_per_split;
     int units_base, units_rem, tiles_per_cta;   // carry: contiguous ranges of 16-row units per CTA
@@ -109,7 +111,7 @@ struct wisv_ctx {
     long long prof_calls = 0;
     cudaEvent_t* prof_ev = nullptr;   // [prof_n][kStages + 1]
     long long launches = 0;
-    wisv_tuning tune = {0, 0, 0, 0, 0, 0, 0, 0};
+    wisv_tuning tune = {0, 0, 0, 0, 0, 0, 0, 0, 0};
     HostStaging hs;
 };
 
@@ -216,12 +218,27 @@ Plan plan_lm(const wisv_ctx* c, int R, bool single_only = false, int sms = 0, in
         p.n_cols = round_up((R + p.n_blocks - 1) / p.n_blocks, 16);
         p.m_tiles = p.n_blocks;
         pair_ring(c, &p);
-        if (p.n_blocks == 1) {
+        const int units = (V + 31) / 32;
+        const int n_tiles_256 = (V + kPairTileN - 1) / kPairTileN;
+        // teams (one per row block, each dealing out the whole vocabulary): when they need no more tiles per pair than
+        // round-robin items need rounds, and all window rows (every team reads its own) stay in L2
+        int team_pairs = pairs_free / p.n_blocks;
+        if (team_pairs > units) team_pairs = units;
+        bool teams = false;
+        if (p.n_blocks > 1 && team_pairs >= 1 && c->tune.lm_teams >= 0) {
+            const int umax = (units + team_pairs - 1) / team_pairs;
+            const long long team_tiles = (umax + kPairTileN / 32 - 1) / (kPairTileN / 32);
+            const long long item_rounds = ((long long)p.n_blocks * n_tiles_256 + pairs_free - 1) / pairs_free;
+            const bool fits = (long long)p.n_blocks * p.n_cols * c->cfg.H * 2 <= kTeamRowBytes;
+            teams = fits && (team_tiles <= item_rounds || c->tune.lm_teams > 0);
+        }
+        if (p.n_blocks == 1 || teams) {
             // One row block (HBM-bound): like the single-CTA kernel with one row tile, every pair gets one contiguous
             // range of the vocabulary, here in units of 32 rows (each CTA of a pair loads half a tile, a multiple of
-            // 16 rows), cut into tiles of nearly equal height; one partial per (row, CTA).
-            const int units = (V + 31) / 32;
-            const int pairs = units < pairs_free ? units : pairs_free;
+            // 16 rows), cut into tiles of nearly equal height; one partial per (row, CTA).  Teams: the same inside
+            // each team.
+            const int pairs = p.n_blocks == 1 ? (units < pairs_free ? units : pairs_free) : team_pairs;
+            p.team_pairs = pairs;
             p.units_base = units / pairs;
             p.units_rem = units % pairs;
             const int umax = p.units_base + (p.units_rem ? 1 : 0);
@@ -229,7 +246,7 @@ Plan plan_lm(const wisv_ctx* c, int R, bool single_only = false, int sms = 0, in
             p.tiles_per_cta = (umax + cap - 1) / cap;
             p.tile_n = (umax + p.tiles_per_cta - 1) / p.tiles_per_cta * 32;
             p.n_tiles = pairs * p.tiles_per_cta;
-            p.ctas = 2 * pairs;
+            p.ctas = 2 * pairs * p.n_blocks;
             p.carry = 1;
             p.parts = 2 * pairs;
             return p;
@@ -238,7 +255,7 @@ Plan plan_lm(const wisv_ctx* c, int R, bool single_only = false, int sms = 0, in
         // partial per (row, vocabulary tile, CTA).
         p.carry = 0;
         p.tile_n = kPairTileN;
-        p.n_tiles = (V + kPairTileN - 1) / kPairTileN;
+        p.n_tiles = n_tiles_256;
         const long long items = (long long)p.n_blocks * p.n_tiles;
         p.ctas = 2 * (int)(items < pairs_free ? items : pairs_free);
         p.parts = 2 * p.n_tiles;
@@ -339,9 +356,10 @@ Plan plan_head_beside(const wisv_ctx* c, int P, int want)
     return h;
 }
 
-// rounds of tiles the slowest CTA (or pair) of a plan without carried ranges works through
+// rounds of tiles the slowest CTA (or pair) of a plan works through
 long long plan_waves(const Plan& p)
 {
+    if (p.pair && p.carry) return p.tiles_per_cta;        // teams: every pair walks its own range
     const long long units = p.pair ? p.ctas / 2 : p.ctas;
     const long long items = (long long)p.m_tiles * p.n_tiles * (p.k_splits > 0 ? p.k_splits : 1);
     return units > 0 ? (items + units - 1) / units : 0;
@@ -553,6 +571,7 @@ PairParams pair_params(const wisv_ctx* c, const Plan& pl, int R)
     }
     sp.stages = pl.stages; sp.kbs = pl.kbs > 0 ? pl.kbs : 1; sp.units_base = pl.units_base; sp.units_rem = pl.units_rem;
     sp.tiles_per_pair = pl.tiles_per_cta > 0 ? pl.tiles_per_cta : 1; sp.tile_m = pl.tile_n;
+    sp.team_pairs = pl.team_pairs > 0 ? pl.team_pairs : 1;
     sp.part_stride = pl.parts; sp.err = c->err;
     sp.lm_part = c->lm_part; sp.row_tok = c->row_tok; sp.tok_logit = c->tok_logit;
     return sp;
@@ -708,6 +727,11 @@ int wisv_create(const wisv_config* cfg, const wisv_weights* w, wisv_ctx** out)
             const size_t e = (size_t)cfg->max_rows * 2 * nt;
             if (e > lm_elems) lm_elems = e;
         }
+        if (cfg->max_rows > kPairTileM) {
+            // teams of pairs: R rows x 2 partials x at most (pairs / ceil(R / 256)) pairs per team <= 512 per pair
+            const size_t e = (size_t)2 * kPairMaxCols * (c->sm_count / 2 > 0 ? c->sm_count / 2 : 1);
+            if (e > lm_elems) lm_elems = e;
+        }
         head_elems = (size_t)c->max_pos * ((cfg->d_J + 15) / 16);
     }
     c->lm_part_elems = lm_elems;
@@ -821,8 +845,9 @@ int wisv_plan_host(const wisv_config* cfg, int32_t sm_count, int32_t max_smem_by
     out->lm_pair = a.pair; out->lm_carry = a.carry; out->lm_tile_n = a.tile_n; out->lm_ctas = a.ctas;
     out->lm_m_tiles = a.m_tiles; out->lm_n_tiles = a.n_tiles; out->lm_stages = a.stages; out->lm_smem_bytes = (int32_t)a.smem;
     out->lm_units_base = a.units_base; out->lm_units_rem = a.units_rem; out->lm_tiles_per_cta = a.tiles_per_cta;
-    out->lm_rounds = a.carry ? 0 : (int32_t)plan_waves(a);
-    out->lm_rounds_alone = alone.carry ? 0 : (int32_t)plan_waves(alone);
+    // rounds of tiles: round-robin items, or the tiles of a pair's range when teams of pairs deal out the vocabulary
+    out->lm_rounds = (a.carry && a.n_blocks <= 1) ? 0 : (int32_t)plan_waves(a);
+    out->lm_rounds_alone = (alone.carry && alone.n_blocks <= 1) ? 0 : (int32_t)plan_waves(alone);
     if (P > 0) {
         out->head_carry = h.carry; out->head_tile_n = h.tile_n; out->head_ctas = h.ctas; out->head_m_tiles = h.m_tiles;
         out->head_n_tiles = h.n_tiles; out->head_k_splits = h.k_splits; out->head_kb_per_split = h.kb_per_split;
@@ -838,12 +863,13 @@ int64_t wisv_launch_count(const wisv_ctx* c) { return c ? c->launches : 0; }
 int wisv_set_tuning(wisv_ctx* c, const wisv_tuning* t)
 {
     if (!c) return WISV_EINVAL;
-    if (!t) { c->tune = wisv_tuning{0, 0, 0, 0, 0, 0, 0, 0}; return WISV_OK; }
+    if (!t) { c->tune = wisv_tuning{0, 0, 0, 0, 0, 0, 0, 0, 0}; return WISV_OK; }
     const int32_t tn[2] = {t->lm_tile_n, t->head_tile_n};
     for (int i = 0; i < 2; ++i)
         if (tn[i] != 0 && (tn[i] < 16 || tn[i] > kMaxTileN || tn[i] % 16)) return WISV_ESHAPE;
     if (t->lm_stages < 0 || t->head_stages < 0 || t->lm_stages == 1 || t->head_stages == 1) return WISV_ESHAPE;
     if (t->lm_mma_m != 0 && t->lm_mma_m != 64 && t->lm_mma_m != 128) return WISV_ESHAPE;
+    if (t->lm_teams < -1 || t->lm_teams > 1) return WISV_ESHAPE;
     if (t->lm_kb_per_stage != 0 && t->lm_kb_per_stage != 1 && t->lm_kb_per_stage != 2 && t->lm_kb_per_stage != 4) return WISV_ESHAPE;
     c->tune = *t;
     return WISV_OK;

@@ -16,11 +16,16 @@
 // '>' keeps the lowest token id).  The running (max, argidx, sum exp) of a window row lives in the registers of
 // the lane that owns its column, per warp; the four warps of a CTA are then merged in vocabulary order.
 //
-// Two ways of dealing out the work:
+// Three ways of dealing out the work:
 //  * one row block (up to 256 rows, bound by HBM): every pair owns one contiguous range of the vocabulary (units of
 //    32 rows, tiles of tile_m or tile_m - 32 rows, balanced to one unit), carries its running row state across its
 //    tiles and writes one partial per (row, CTA) at the end;
-//  * several row blocks (bound by the tensor pipe): work items (vocabulary tile of 256 rows, row block) are dealt
+//  * a few row blocks (2-4 in practice): the pairs form one team per row block and every team deals out the
+//    vocabulary as above, so a row still gets one partial per CTA of its team (48 instead of 1002 at 576 rows and 8B
+//    shapes) and nothing is merged or written between tiles; the k-th pairs of all teams stream the same range at the
+//    same time and share its weight tiles through L2.  Chosen when the teams need no more tiles per pair than the
+//    round-robin below needs rounds;
+//  * many row blocks (bound by the tensor pipe): work items (vocabulary tile of 256 rows, row block) are dealt
 //    out round-robin, row blocks of a group fastest, so the pairs that run at the same time share a weight tile
 //    through L2 and a group's activation rows stay resident there; one partial per (row, vocabulary tile, CTA).
 //
@@ -51,6 +56,10 @@ struct PairParams {
     // one row block (carry = 1): vocabulary ranges in units of 32 rows per pair - units_base units, one more for the
     // first units_rem pairs - cut into tiles_per_pair tiles of tile_m or tile_m - 32 rows
     int32_t carry, units_base, units_rem, tiles_per_pair, tile_m;
+    // carry with several row blocks: the pairs form row_blocks teams of team_pairs pairs; team j streams the whole
+    // vocabulary for row block j, its k-th pair the k-th range, so the pairs that work on one range at the same time
+    // (one per team) share its weight tiles through L2.  One row block: one team of all pairs.
+    int32_t team_pairs;
     // several row blocks (carry = 0): n_tiles vocabulary tiles of 256 rows; items run group by group (all vocabulary
     // tiles of a group of b_group row blocks before the next group)
     int32_t n_tiles, b_group;
@@ -123,9 +132,12 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
 
     const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0);   // the same in all lanes, and the compiler knows it
     const int lane = threadIdx.x & 31;
-    // carry: this pair's contiguous range of 32-row units and how it is cut into tiles
-    const int my_units = p.units_base + (pair_id < p.units_rem ? 1 : 0);
-    const int my_unit0 = pair_id * p.units_base + (pair_id < p.units_rem ? pair_id : p.units_rem);
+    // carry: this pair's team (row block) and place in it, its contiguous range of 32-row units and how that is cut
+    // into tiles
+    const int team = p.carry ? pair_id / p.team_pairs : 0;
+    const int team_k = p.carry ? pair_id - team * p.team_pairs : 0;
+    const int my_units = p.units_base + (team_k < p.units_rem ? 1 : 0);
+    const int my_unit0 = team_k * p.units_base + (team_k < p.units_rem ? team_k : p.units_rem);
     const int my_tiles = p.carry ? (my_units < p.tiles_per_pair ? my_units : p.tiles_per_pair) : 0;
     const int my_hq = p.carry ? my_units / p.tiles_per_pair : 0;
     const int my_hr = p.carry ? my_units % p.tiles_per_pair : 0;
@@ -135,7 +147,7 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     auto item_at = [&](int i, Item& w) -> bool {
         if (p.carry) {
             if (i >= my_tiles) return false;
-            w.n = pair_id; w.j = 0;
+            w.n = team_k; w.j = team;
             w.h = (my_hq + (i < my_hr ? 1 : 0)) * 32;
             w.n0 = (my_unit0 + i * my_hq + (i < my_hr ? i : my_hr)) * 32;
             return true;
@@ -344,7 +356,7 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             }
             asm volatile("bar.sync 1, 128;" ::: "memory");        // the buffer goes back to the transposition
         };
-        if (p.carry) reset_state(0);
+        if (p.carry) reset_state(team);
         Item w;
         for (int local = 0; ok && item_at(local, w); ++local) {
             const int as = local & 1;
@@ -431,7 +443,7 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         }
         // carry: the tiles of a pair ascend through the vocabulary, so the strict '>' of the update kept the lowest
         // index; a pair without tiles is never launched.  (`ok` is the same in all four warps, see above.)
-        if (p.carry && ok) flush_state(0, pair_id * 2 + static_cast<int>(rank));
+        if (p.carry && ok) flush_state(team, team_k * 2 + static_cast<int>(rank));
     }
 
     // After a time-out copies may still be heading for the shared memory of either CTA.  Their bytes are counted on

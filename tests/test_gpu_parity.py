@@ -239,7 +239,10 @@ def test_more_row_tiles_share_a_launch_when_it_costs_no_extra_round_of_tiles(kw)
     torch.cuda.synchronize()
     assert v.device_error() == 0
     assert torch.equal(sep.argmax, out.argmax) and torch.equal(sep.accept_len, out.accept_len)
-    assert torch.equal(sep.correction_token, out.correction_token) and torch.equal(sep.lse, out.lse)
+    assert torch.equal(sep.correction_token, out.correction_token)
+    # with fewer pairs for the LM head its teams cut the vocabulary into other ranges: the sums of exponentials are
+    # added in another order
+    assert float((sep.lse - out.lse).abs().max()) < 1e-5
     assert float((sep.head_prob - out.head_prob).abs().max()) < 1e-5
     v.close()
 
@@ -840,7 +843,8 @@ def test_random_shapes_under_every_launch_plan():
     for it in range(40):
         ragged = rng.random() < 0.3
         K = int(rng.integers(1, 13))
-        target_rows = int(rng.choice([5, 16, 17, 63, 64, 65, 127, 128, 129, 200, 255, 256, 257, 300, 384, 385, 520]))
+        target_rows = int(rng.choice([5, 16, 17, 63, 64, 65, 127, 128, 129, 200, 255, 256, 257, 300, 384, 385, 520, 780,
+                                      1040]))
         kw = dict(B=max(1, target_rows // (K + 1)), K=0 if ragged else K, H=int(rng.choice([64, 72, 128, 256])),
                   H_d=int(rng.choice([8, 40, 64, 128])), d_c=int(rng.choice([0, 2, 3])),
                   d_J=int(rng.choice([16, 48, 50, 128, 200, 272])),
@@ -859,7 +863,8 @@ def test_random_shapes_under_every_launch_plan():
         d = cases.to_device(case, DEV)
         v = cases.make_verifier(d)
         outs = []
-        for tune in (dict(), dict(head_ctas=-1), dict(lm_single_cta=1), dict(head_ctas=3), dict(lm_kb_per_stage=1), dict(lm_kb_per_stage=4)):
+        for tune in (dict(), dict(head_ctas=-1), dict(lm_single_cta=1), dict(head_ctas=3), dict(lm_kb_per_stage=1),
+                     dict(lm_kb_per_stage=4), dict(lm_teams=-1), dict(lm_teams=1, head_ctas=-1)):
             v.set_tuning(**tune)
             cases.run(v, d)
             out = cases.run(v, d)                       # twice: nothing may linger from the first call

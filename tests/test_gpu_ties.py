@@ -146,8 +146,8 @@ def _assert_planted(argmax, expect, what):
         assert am[r] == g[0], "%s: tie %s %s on row %d resolved to %d" % (what, name, g, r, am[r])
 
 
-SHAPES = {"R9_mma64": (1, 8), "R100_mma128": (20, 4), "R200_pair_ranges": (40, 4), "R300_three_row_tiles": (60, 4),
-          "R512_pair_tiles": (64, 7)}
+SHAPES = {"R9_mma64": (1, 8), "R100_mma128": (20, 4), "R200_pair_ranges": (40, 4), "R300_two_teams": (60, 4),
+          "R512_two_teams": (64, 7), "R1040_pair_items": (130, 7)}
 
 
 @pytest.mark.gpu
@@ -159,10 +159,15 @@ def test_lowest_token_id_wins_at_every_merge_site(shape):
     R = case["R"]
     if shape == "R200_pair_ranges":
         assert plan["lm_pair"] and plan["lm_carry"] and plan["lm_tiles_per_cta"] > 1
-    if shape == "R512_pair_tiles":
-        assert plan["lm_pair"] and not plan["lm_carry"] and plan["lm_n_cols"] == 256
-    if shape == "R300_three_row_tiles":
-        assert plan["lm_pair"] and not plan["lm_carry"] and plan["lm_n_cols"] == 160      # two row blocks of 160
+    if shape == "R512_two_teams":
+        assert plan["lm_pair"] and plan["lm_carry"] and (plan["lm_n_cols"], plan["lm_row_blocks"]) == (256, 2)
+    if shape == "R300_two_teams":
+        # two row blocks of 160, a team of pairs each, every pair with several tiles in its vocabulary range
+        assert plan["lm_pair"] and plan["lm_carry"] and (plan["lm_n_cols"], plan["lm_row_blocks"]) == (160, 2)
+        assert plan["lm_tiles_per_cta"] > 1 and plan["lm_parts"] == plan["lm_ctas"] // 2
+    if shape == "R1040_pair_items":
+        # five row blocks: work items (vocabulary tile of 256, row block) dealt out round-robin, partials per tile
+        assert plan["lm_pair"] and not plan["lm_carry"] and plan["lm_row_blocks"] == 5
     if R <= 128:
         assert plan["lm_carry"] and plan["lm_tiles_per_cta"] > 1
     d = cases.to_device(case, DEV)
@@ -175,6 +180,9 @@ def test_lowest_token_id_wins_at_every_merge_site(shape):
     if R <= 128:
         # other tile heights (with more rows the partial buffer is sized for the automatic tile and refuses finer ones)
         tunings += [dict(lm_tile_n=64), dict(lm_tile_n=176, lm_stages=3)]
+    if R > 256:
+        # the other way of dealing out the pair kernel's work: round-robin items instead of teams, and the reverse
+        tunings += [dict(lm_teams=-1), dict(lm_teams=1), dict(lm_teams=-1, lm_kb_per_stage=4)]
     for tune in tunings:
         v.set_tuning(**tune)
         out = cases.run(v, d)
@@ -226,10 +234,13 @@ def test_lowest_token_id_wins_at_every_merge_site(shape):
 def test_owner_map_matches_the_planner():
     """The helper that places the ties must describe the ranges the planner deals out (every token owned once,
     chunks and tiles inside the stated heights).  Host arithmetic only."""
-    for R, P in ((9, 8), (100, 80), (200, 160)):
+    for R, P in ((9, 8), (100, 80), (200, 160), (300, 240), (512, 448)):
         plan = wisv.plan_host(H=H, V=V, H_d=64, d_c=2, d_J=64, R=R, P=P, sm_count=SM, max_smem_bytes=SMEM)
         own = _owner_fn(plan)
         groups = plan["lm_ctas"] // 2 if plan["lm_pair"] else plan["lm_ctas"]
+        if R > 256:
+            assert plan["lm_carry"] and plan["lm_row_blocks"] == 2
+            groups //= plan["lm_row_blocks"]                  # teams of pairs: ownership inside a team
         seen = {}
         for v in range(0, V, 7):
             c, t, ch, half = own(v)

@@ -58,11 +58,15 @@ def test_plans_at_the_task_shapes():
     p = plan_host(R=144, P=128, **DIMS_8B)                   # B=16: pairs with head clusters
     assert (p["kernels"], p["lm_pair"], p["lm_carry"], p["lm_ctas"], p["head_ctas"]) == (3, 1, 1, 142, 6)
     assert (p["lm_n_cols"], p["lm_row_blocks"], p["lm_parts"]) == (144, 1, 142)     # the MMA's N is the row count up to 16
-    p = plan_host(R=288, P=256, **DIMS_8B)                   # B=32: two row blocks of 144, nothing padded
-    assert (p["kernels"], p["lm_pair"], p["lm_carry"], p["lm_n_cols"], p["lm_row_blocks"]) == (3, 1, 0, 144, 2)
-    p = plan_host(R=576, P=512, **DIMS_8B)                   # B=64: three row blocks of 192; 1503 items on 72 pairs
-    assert (p["kernels"], p["lm_pair"], p["lm_ctas"], p["lm_rounds"]) == (3, 1, 144, 21)
-    assert (p["lm_n_cols"], p["lm_row_blocks"], p["lm_parts"], p["head_ctas"]) == (192, 3, 1002, 4)
+    p = plan_host(R=288, P=256, **DIMS_8B)                   # B=32: two row blocks of 144, nothing padded; two teams
+    assert (p["kernels"], p["lm_pair"], p["lm_carry"], p["lm_n_cols"], p["lm_row_blocks"]) == (3, 1, 1, 144, 2)
+    assert (p["lm_ctas"], p["lm_parts"], p["lm_rounds"], p["head_ctas"]) == (144, 72, 14, 2)   # of 36 pairs
+    p = plan_host(R=576, P=512, **DIMS_8B)                   # B=64: three row blocks of 192; three teams of 24 pairs,
+    assert (p["kernels"], p["lm_pair"], p["lm_carry"], p["lm_ctas"], p["lm_rounds"]) == (3, 1, 1, 144, 21)   # 21 tiles each
+    assert (p["lm_n_cols"], p["lm_row_blocks"], p["lm_parts"], p["head_ctas"]) == (192, 3, 48, 4)
+    assert (p["lm_units_base"], p["lm_units_rem"], p["lm_tiles_per_cta"]) == (167, 0, 21)     # 4008 units of 32 rows / 24
+    p = plan_host(R=1100, P=1000, **DIMS_8B)                 # five row blocks: 14 pairs per team would need 36 tiles
+    assert (p["lm_carry"], p["lm_row_blocks"], p["lm_parts"], p["lm_rounds"]) == (0, 5, 1002, 34)   # against 34 rounds
     p = plan_host(R=8704, P=8192, **DIMS_8B)                 # B=512, K=16: 74 pairs, 230.2 rounds of 256 x 256 items
     assert (p["kernels"], p["lm_pair"], p["lm_ctas"], p["lm_rounds"]) == (4, 1, 148, 231)
     assert (p["lm_n_cols"], p["lm_row_blocks"]) == (256, 34)
@@ -72,9 +76,18 @@ def test_plans_at_the_task_shapes():
 def test_head_rides_along_only_when_the_lm_head_needs_no_extra_round(R):
     for P in (R - R // 9, max(1, R // 3)):
         p = plan_host(R=R, P=P, **DIMS_8B)
-        assert p["lm_carry"] == 0
         groups = p["lm_ctas"] // 2 if p["lm_pair"] else p["lm_ctas"]
-        assert p["lm_rounds"] == -(-(p["lm_m_tiles"] * p["lm_n_tiles"]) // groups)
+        if p["lm_carry"]:
+            # teams of pairs, one per row block: a round is one tile of a pair's own vocabulary range, and the plan
+            # is taken only when that is no more than round-robin items would need
+            assert p["lm_row_blocks"] in (2, 3, 4) and groups % p["lm_row_blocks"] == 0
+            assert p["lm_rounds"] == p["lm_tiles_per_cta"]
+            assert p["lm_rounds"] <= -(-(p["lm_row_blocks"] * -(-128256 // 256)) // groups)
+            team = groups // p["lm_row_blocks"]
+            assert p["lm_parts"] == 2 * team
+            assert team * p["lm_units_base"] + p["lm_units_rem"] == -(-128256 // 32)
+        else:
+            assert p["lm_rounds"] == -(-(p["lm_m_tiles"] * p["lm_n_tiles"]) // groups)
         if p["head_in_lm_launch"]:
             assert p["kernels"] == 3 and p["lm_rounds"] == p["lm_rounds_alone"]
             assert p["lm_ctas"] + p["head_ctas"] + (p["head_ctas"] % 2 if p["lm_pair"] else 0) <= 148
@@ -93,8 +106,8 @@ def test_row_blocks_of_the_pair_kernel_pad_at_most_fifteen_rows_each():
         assert nb == -(-R // 256) and n % 16 == 0 and 16 <= n <= 256
         assert nb * n >= R and nb * (n - 16) < R              # the narrowest width that covers the rows
         assert nb * n <= -(-R // 256) * 256                   # the blocks stay inside the rows the workspace holds
-        assert p["lm_carry"] == (1 if nb == 1 else 0)
-        assert p["lm_parts"] == (p["lm_ctas"] if nb == 1 else 2 * p["lm_n_tiles"])
+        assert p["lm_carry"] == (1 if nb <= 4 else 0)         # one team of pairs per row block up to four blocks
+        assert p["lm_parts"] == (p["lm_ctas"] // nb if nb <= 4 else 2 * p["lm_n_tiles"])
     assert plan_host(R=128, P=0, **DIMS_8B)["lm_pair"] == 0
 
 
