@@ -297,7 +297,9 @@ def run_reference(args, rank, world):
 # ------------------------------------------------------------------------------------- CUDA arm
 
 NOMINAL_PEAKS = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0}       # HGX B200 data-sheet figures (dense bf16)
-DEFAULT_LEGS = ("8b_b64", "8b_sh256", "8b_b512")                 # tensor-bound configurations of the same 8B model
+# further configurations of the same 8B model: 144 rows (one row block on CTA pairs, still bound by HBM), then the
+# tensor-bound ones
+DEFAULT_LEGS = ("8b_b16", "8b_b64", "8b_sh256", "8b_b512")
 SHM_DIR = "/dev/shm"
 
 
