@@ -45,6 +45,7 @@ struct Plan {
     int n_blocks;    // pairs: row blocks of n_cols rows
     int kbs;         // pairs: K blocks per shared-memory stage
     int team_pairs;  // pairs with carried ranges: pairs per team (one team per row block)
+    int box3d;       // pairs: one TMA box per operand and stage (3-D tensor maps)
     int k_splits;    // work items per (m, n) tile along K (decision head with one row tile)
     int kb_per_split;
     int units_base, units_rem, tiles_per_cta;   // carry: contiguous ranges of 16-row units per CTA
@@ -106,6 +107,10 @@ struct wisv_ctx {
     CUtensorMap tmX[kNumRowVariants], tmZ[kNumRowVariants];   // box heights 8, 16, ..., 128 rows
     CUtensorMap tmW[kNumTileVariants];
     CUtensorMap tmW1[kNumTileVariants];
+    // CTA-pair LM head, boxes of 2 ([0]) or 4 ([1]) K blocks: window rows (8..128 per box) and weight rows (16..128)
+    CUtensorMap tmX3[2][kNumRowVariants];
+    CUtensorMap tmW3[2][kNumTileVariants / 2];
+    bool have_box3d = false;
     // profiling
     int prof_n = 0;
     long long prof_calls = 0;
@@ -131,6 +136,21 @@ int encode_2d(EncodeTiledFn fn, CUtensorMap* out, const void* base, uint64_t inn
     cuuint32_t box[2] = {box_inner, box_outer};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? WISV_OK : WISV_ECUDA;
+}
+
+// The same matrix seen as (column inside a K block of 64, row, K block): a box of `box_kb` K blocks of `box_rows` rows
+// lands in shared memory block after block, each block in the layout the 2-D box gives.  Only for inner % 64 == 0.
+int encode_3d(EncodeTiledFn fn, CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer, uint32_t box_rows,
+              uint32_t box_kb)
+{
+    cuuint64_t dims[3] = {(cuuint64_t)kBlockK, outer, inner / kBlockK};
+    cuuint64_t strides[2] = {inner * 2, (cuuint64_t)kBlockK * 2};
+    cuuint32_t box[3] = {(cuuint32_t)kBlockK, box_rows, box_kb};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? WISV_OK : WISV_ECUDA;
@@ -190,6 +210,7 @@ void pair_ring(const wisv_ctx* c, Plan* p)
     if (ss > kMaxStages) ss = kMaxStages;
     if (c->tune.lm_stages >= 2 && c->tune.lm_stages < ss) ss = c->tune.lm_stages;
     p->kbs = kbs;
+    p->box3d = (c->have_box3d && (kbs == 2 || kbs == 4)) ? 1 : 0;
     p->stages = ss;
     p->smem = pair_fixed_bytes() + (size_t)ss * stage;
 }
@@ -551,6 +572,16 @@ inline int map_lo(const Plan& pl) { return pl.tile_n / 16 - 2 > 0 ? pl.tile_n / 
 // tensor maps of the pair kernel's weight tiles: each CTA of a pair loads half of a tile's rows
 inline int pair_map_hi(const Plan& pl) { return pl.tile_n / 32 - 1; }
 inline int pair_map_lo(const Plan& pl) { return pl.tile_n / 32 - 2 > 0 ? pl.tile_n / 32 - 2 : 0; }
+// tensor maps of the CTA-pair LM head: half a row block of window rows; half a tile of tile_n (or tile_n - 32) weight rows
+inline const CUtensorMap& pair_tm_x(const wisv_ctx* c, const Plan& pl)
+{
+    return pl.box3d ? c->tmX3[pl.kbs / 4][pl.n_cols / 16 - 1] : c->tmX[pl.n_cols / 16 - 1];
+}
+inline const CUtensorMap& pair_tm_w(const wisv_ctx* c, const Plan& pl, bool lower)
+{
+    const int i = lower ? pair_map_lo(pl) : pair_map_hi(pl);
+    return pl.box3d ? c->tmW3[pl.kbs / 4][i] : c->tmW[i];
+}
 
 PairParams pair_params(const wisv_ctx* c, const Plan& pl, int R)
 {
@@ -572,6 +603,7 @@ PairParams pair_params(const wisv_ctx* c, const Plan& pl, int R)
     sp.stages = pl.stages; sp.kbs = pl.kbs > 0 ? pl.kbs : 1; sp.units_base = pl.units_base; sp.units_rem = pl.units_rem;
     sp.tiles_per_pair = pl.tiles_per_cta > 0 ? pl.tiles_per_cta : 1; sp.tile_m = pl.tile_n;
     sp.team_pairs = pl.team_pairs > 0 ? pl.team_pairs : 1;
+    sp.box3d = pl.box3d;
     sp.part_stride = pl.parts; sp.err = c->err;
     sp.lm_part = c->lm_part; sp.row_tok = c->row_tok; sp.tok_logit = c->tok_logit;
     return sp;
@@ -781,6 +813,18 @@ int wisv_create(const wisv_config* cfg, const wisv_weights* w, wisv_ctx** out)
             if (rc == WISV_OK)
                 rc = encode_2d(encode, &c->tmW1[i], c->W1p, (uint64_t)hd_h, (uint64_t)cfg->d_J, kBlockK, tn);
         }
+        if (rc == WISV_OK && cfg->H % kBlockK == 0 && cfg->H >= 2 * kBlockK) {
+            // (a driver that refuses these maps only costs the wider boxes, not the context)
+            int rc3 = WISV_OK;
+            for (int q = 0; q < 2 && rc3 == WISV_OK; ++q) {
+                const uint32_t kb = q ? 4u : 2u;
+                for (int i = 0; i < kNumRowVariants && rc3 == WISV_OK; ++i)
+                    rc3 = encode_3d(encode, &c->tmX3[q][i], c->X, (uint64_t)cfg->H, (uint64_t)c->rows_alloc, 8u * (i + 1), kb);
+                for (int i = 0; i < kNumTileVariants / 2 && rc3 == WISV_OK; ++i)
+                    rc3 = encode_3d(encode, &c->tmW3[q][i], w->lm_head, (uint64_t)cfg->H, (uint64_t)cfg->V, 16u * (i + 1), kb);
+            }
+            c->have_box3d = rc3 == WISV_OK;
+        }
     } while (0);
     if (rc != WISV_OK) { free_ctx(c); return rc; }
     *out = c;
@@ -957,7 +1001,7 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
         if (pl.pair) {
             const PairParams sp = pair_params(c, pl, R);
             const int rc = launch_pdl(lmhead_pair_kernel, dim3(pl.ctas + round_up(ph.ctas, 2)), dim3(kGemmThreads), smem,
-                                      st, c->tmX[pl.n_cols / 16 - 1], c->tmW[pair_map_hi(pl)], c->tmW[pair_map_lo(pl)],
+                                      st, pair_tm_x(c, pl), pair_tm_w(c, pl, false), pair_tm_w(c, pl, true),
                                       sp, c->tmZ[ph.a_rows / 8 - 1], c->tmW1[map_hi(ph)], c->tmW1[map_lo(ph)], gh,
                                       pl.ctas, ph.ctas);
             if (rc != WISV_OK) return rc;
@@ -976,7 +1020,7 @@ int run_round(wisv_ctx* c, const wisv_batch* b, const wisv_result* r, void* cuda
         GemmParams none;
         memset(&none, 0, sizeof none);
         const int rc = launch_pdl(lmhead_pair_kernel, dim3(pl.ctas), dim3(kGemmThreads), pl.smem, st,
-                                  c->tmX[pl.n_cols / 16 - 1], c->tmW[pair_map_hi(pl)], c->tmW[pair_map_lo(pl)], sp,
+                                  pair_tm_x(c, pl), pair_tm_w(c, pl, false), pair_tm_w(c, pl, true), sp,
                                   c->tmZ[0], c->tmW1[0], c->tmW1[0], none, pl.ctas, 0);
         if (rc != WISV_OK) return rc;
         c->launches++;

@@ -53,6 +53,10 @@ struct PairParams {
     int32_t k_blocks;
     int32_t stages;
     int32_t kbs;         // K blocks per stage (1, 2 or 4): one barrier round trip, on both sides of the ring, serves kbs K blocks
+    int32_t box3d;       // 1: the tensor maps are 3-D (column in a K block, row, K block) with boxes of kbs K blocks, so one
+                         // TMA instruction per operand fills a stage (each instruction costs the producer about 80 clocks
+                         // on top of about 440 per stage); needs H % 64 == 0.  A weight block then takes its real height
+                         // in shared memory, not a 128-row slot.
     // one row block (carry = 1): vocabulary ranges in units of 32 rows per pair - units_base units, one more for the
     // first units_rem pairs - cut into tiles_per_pair tiles of tile_m or tile_m - 32 rows
     int32_t carry, units_base, units_rem, tiles_per_pair, tile_m;
@@ -216,11 +220,17 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             for (int kb = 0; kb < p.k_blocks && pre < p.stages; kb += p.kbs, ++pre) {
                 const int nb = min(p.kbs, p.k_blocks - kb);
                 const uint32_t dst = smem_base + stage_bytes * static_cast<uint32_t>(pre);
-                const uint32_t tx = 2u * static_cast<uint32_t>(nb) * (static_cast<uint32_t>(half_h) * kBlockK * 2u + b_bytes);
+                // a 3-D box always brings kbs K blocks (zeros past the end of K)
+                const uint32_t tx = 2u * static_cast<uint32_t>(p.box3d ? p.kbs : nb) *
+                                    (static_cast<uint32_t>(half_h) * kBlockK * 2u + b_bytes);
                 if (elect_one()) {
                     if (leader) mbar_expect_tx(full_bar(pre), tx);          // both CTAs' bytes
-                    for (int u = 0; u < nb; ++u)
-                        tma_load_2d_pair(dst + static_cast<uint32_t>(u) * a_bytes, mapW, (kb + u) * kBlockK, w_row0, full_bar(pre));
+                    if (p.box3d) {
+                        tma_load_3d_pair(dst, mapW, 0, w_row0, kb, full_bar(pre));
+                    } else {
+                        for (int u = 0; u < nb; ++u)
+                            tma_load_2d_pair(dst + static_cast<uint32_t>(u) * a_bytes, mapW, (kb + u) * kBlockK, w_row0, full_bar(pre));
+                    }
                 }
                 __syncwarp();
             }
@@ -247,13 +257,21 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                         if (!ok) break;
                     }
                     if (elect_one()) {
-                        if (fresh) {
-                            if (leader) mbar_expect_tx(full_bar(s), 2u * static_cast<uint32_t>(nb) * tx_w);
+                        if (p.box3d) {
+                            if (fresh) {
+                                if (leader) mbar_expect_tx(full_bar(s), 2u * static_cast<uint32_t>(p.kbs) * tx_w);
+                                tma_load_3d_pair(dst, mapW, 0, w_row0, kb, full_bar(s));
+                            }
+                            tma_load_3d_pair(dst + x_off, &tmX, 0, x_row0, kb, full_bar(s));
+                        } else {
+                            if (fresh) {
+                                if (leader) mbar_expect_tx(full_bar(s), 2u * static_cast<uint32_t>(nb) * tx_w);
+                                for (int u = 0; u < nb; ++u)
+                                    tma_load_2d_pair(dst + static_cast<uint32_t>(u) * a_bytes, mapW, (kb + u) * kBlockK, w_row0, full_bar(s));
+                            }
                             for (int u = 0; u < nb; ++u)
-                                tma_load_2d_pair(dst + static_cast<uint32_t>(u) * a_bytes, mapW, (kb + u) * kBlockK, w_row0, full_bar(s));
+                                tma_load_2d_pair(dst + x_off + static_cast<uint32_t>(u) * b_bytes, &tmX, (kb + u) * kBlockK, x_row0, full_bar(s));
                         }
-                        for (int u = 0; u < nb; ++u)
-                            tma_load_2d_pair(dst + x_off + static_cast<uint32_t>(u) * b_bytes, &tmX, (kb + u) * kBlockK, x_row0, full_bar(s));
                     }
                     __syncwarp();
                     ++prod_issued;
@@ -278,6 +296,8 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(as * kAccCols);
+                // bytes between the weight blocks of a stage
+                const uint32_t a_blk = p.box3d ? static_cast<uint32_t>(w.h >> 1) * kBlockK * 2u : a_bytes;
                 for (int kb = 0; kb < p.k_blocks; kb += p.kbs) {
                     const int nb = min(p.kbs, p.k_blocks - kb);
                     ok = __all_sync(0xffffffffu, mbar_wait_bounded(full_bar(s), ph, abort_flag, kWaitLimitClocks));
@@ -289,7 +309,7 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                     const bool last = kb + nb >= p.k_blocks;
                     if (elect_one()) {
                         for (int u = 0; u < nb; ++u) {
-                            const uint64_t a_desc = a_desc0 + static_cast<uint64_t>((static_cast<uint32_t>(u) * a_bytes) >> 4);
+                            const uint64_t a_desc = a_desc0 + static_cast<uint64_t>((static_cast<uint32_t>(u) * a_blk) >> 4);
                             const uint64_t b_desc = b_desc0 + static_cast<uint64_t>((static_cast<uint32_t>(u) * b_bytes) >> 4);
 #pragma unroll
                             for (int k = 0; k < kBlockK / kUmmaK; ++k)
