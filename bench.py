@@ -45,14 +45,14 @@ CTA_PAIR_SOURCES = ("wisv_gemm2.cuh", "wisv_gemm.cuh", "wisv_ptx.cuh")
 NCU_TRAFFIC = {
     # LM-head and decision-head CTAs in one launch, 9 window rows: 1.0642 GB read + 3.8-4.8 MB written per launch
     "8b_b1": {"bytes": 1068500000, "files": SINGLE_CTA_SOURCES, "kernel_hash": "93b8d429d9cf04b3"},
-    # CTA pairs (one row block of 144) + decision-head clusters: 1.0762 GB read + 4.4-4.8 MB written per launch
-    "8b_b16": {"bytes": 1080800000, "files": CTA_PAIR_SOURCES, "kernel_hash": "9286f23afc62be64"},
-    # CTA pairs (three teams, row blocks of 192) + decision-head clusters: 1.1196 GB read + 4.1-4.3 MB written per launch
-    "8b_b64": {"bytes": 1123800000, "files": CTA_PAIR_SOURCES, "kernel_hash": "9286f23afc62be64"},
-    # CTA pairs (34 row blocks of 256, two raster groups): 3.89-4.04 GB read + 138-141 MB written (the partials) per
+    # CTA pairs (one row block of 144) + decision-head clusters: 1.0761 GB read + 3.8-3.9 MB written per launch
+    "8b_b16": {"bytes": 1079900000, "files": CTA_PAIR_SOURCES, "kernel_hash": "6701d2854056471d"},
+    # CTA pairs (three teams, row blocks of 192) + decision-head clusters: 1.1239 GB read + 4.3-4.6 MB written per launch
+    "8b_b64": {"bytes": 1128400000, "files": CTA_PAIR_SOURCES, "kernel_hash": "6701d2854056471d"},
+    # CTA pairs (34 row blocks of 256, two raster groups): 2.93-3.11 GB read + 138-142 MB written (the partials) per
     # launch in this capture; what falls out of L2 depends on where the buffers land, and other captures of the same
-    # kernel read 2.3-5.4 GB
-    "8b_b512": {"bytes": 4104000000, "files": CTA_PAIR_SOURCES, "kernel_hash": "9286f23afc62be64"},
+    # plan read 2.3-5.4 GB
+    "8b_b512": {"bytes": 3160000000, "files": CTA_PAIR_SOURCES, "kernel_hash": "6701d2854056471d"},
 }
 
 
