@@ -43,8 +43,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 SINGLE_CTA_SOURCES = ("wisv_gemm.cuh", "wisv_ptx.cuh")
 CTA_PAIR_SOURCES = ("wisv_gemm2.cuh", "wisv_gemm.cuh", "wisv_ptx.cuh")
 NCU_TRAFFIC = {
-    # LM-head and decision-head CTAs in one launch, 9 window rows: 1.0642 GB read + 3.8-4.8 MB written per launch
-    "8b_b1": {"bytes": 1068500000, "files": SINGLE_CTA_SOURCES, "kernel_hash": "93b8d429d9cf04b3"},
+    # LM-head and decision-head CTAs in one launch, 9 window rows: 1.0642 GB read + 3.8-4.4 MB written per launch
+    "8b_b1": {"bytes": 1068300000, "files": SINGLE_CTA_SOURCES, "kernel_hash": "97d6116174a73cd8"},
     # CTA pairs (one row block of 144) + decision-head clusters: 1.0761 GB read + 3.8-3.9 MB written per launch
     "8b_b16": {"bytes": 1079900000, "files": CTA_PAIR_SOURCES, "kernel_hash": "6701d2854056471d"},
     # CTA pairs (three teams, row blocks of 192) + decision-head clusters: 1.1239 GB read + 4.3-4.6 MB written per launch
