@@ -217,9 +217,9 @@ void pair_ring(const wisv_ctx* c, Plan* p)
 
 // LM head.  Up to 128 window rows: single CTAs with the rows on the M side, each with one contiguous range of the
 // vocabulary (HBM-bound).  More rows: CTA pairs with the vocabulary on the M side and the rows on the N side
-// (wisv_gemm3.cuh) - one row block with carried vocabulary ranges up to 256 rows, several row blocks dealt out as
-// (vocabulary tile, row block) items above.  The tuning switches lm_single_cta / lm_tile_n keep every size on the
-// single-CTA kernel.
+// (wisv_gemm2.cuh) - one row block with carried vocabulary ranges up to 256 rows, one team of pairs per row block
+// with carried ranges while that costs no extra tile (2-4 blocks), (vocabulary tile, row block) items dealt out
+// round-robin above.  The tuning switches lm_single_cta / lm_tile_n keep every size on the single-CTA kernel.
 Plan plan_lm(const wisv_ctx* c, int R, bool single_only = false, int sms = 0, int reserved_pairs = 0)
 {
     Plan p{};
