@@ -330,19 +330,20 @@ Plan plan_head(const wisv_ctx* c, int P)
         if (splits > kMaxKSplits) splits = kMaxKSplits;
         p.kb_per_split = (k_blocks + splits - 1) / splits;
         p.k_splits = (k_blocks + p.kb_per_split - 1) / p.kb_per_split;
-    } else if (p.m_tiles >= 8) {
-        best = kMaxTileN;
     } else {
-        // Every work item walks all of K, and below about 200 columns a K block costs the same whatever the tile
-        // width (four MMAs at their issue-bound pace); wider tiles take proportionally longer.  So: fewest rounds
-        // of items first, at equal time the wider tile (fewer re-reads of the activation rows: with six row tiles
-        // one round of 48 items 128 columns wide ran 7 % faster than one round of 96 items 64 wide).
+        // Every work item walks all of K.  Measured with 5 to 64 row tiles of positions (d_J = 1024, 96 K blocks): the
+        // kernel takes about 20 us plus, per round of items, 38 / 45 / 63 us with tiles 64 / 128 / 256 columns wide
+        // (narrow tiles need more bytes per flop, so their rounds are not shorter in proportion).  So: the width whose
+        // rounds cost least, at equal cost the wider tile - 64 columns while that is one round (up to 9 row tiles on
+        // 148 SMs), 128 up to 18 row tiles, 256 beyond.
+        static const int widths[3] = {64, 128, 256};
+        static const double per_round[3] = {38.0, 45.0, 63.0};
         double best_cost = 1e30;
-        for (int tn = 16; tn <= kMaxTileN; tn *= 2) {
+        for (int k = 0; k < 3; ++k) {
+            const int tn = widths[k];
             const long long tiles = (long long)p.m_tiles * ((N + tn - 1) / tn);
             const long long rounds = (tiles + c->sm_count - 1) / c->sm_count;
-            const double per_item = tn > 208 ? tn / 208.0 : 1.0;
-            const double cost = (double)rounds * per_item;
+            const double cost = (double)rounds * per_round[k];
             if (cost <= best_cost + 1e-9) { best_cost = cost; best = tn; }
         }
     }

@@ -122,10 +122,17 @@ def test_decision_head_in_a_launch_of_its_own():
     assert (p["head_in_lm_launch"], p["head_tile_n"], p["head_m_tiles"], p["head_n_tiles"]) == (0, 64, 4, 16)
     assert p["head_k_splits"] == 2 and p["head_kb_per_split"] == 48 and p["head_ctas"] == 128
     assert p["head_k_splits"] * p["head_kb_per_split"] >= 96  # the splits cover all 96 K blocks
-    # six row tiles: no split; one round of 128-wide items rather than three rounds of 16-wide ones
+    # six row tiles: no split; one round of 96 items 64 columns wide (a round of narrower tiles is shorter)
     p = plan_host(R=1100, P=768, **DIMS_8B)
+    assert (p["head_in_lm_launch"], p["head_k_splits"], p["head_tile_n"]) == (0, 1, 64)
+    assert p["head_m_tiles"] * p["head_n_tiles"] == 96
+    # thirteen row tiles: 64-wide items would need two rounds, 128-wide ones fit in one
+    p = plan_host(R=1800, P=1600, **DIMS_8B)
     assert (p["head_in_lm_launch"], p["head_k_splits"], p["head_tile_n"]) == (0, 1, 128)
-    assert p["head_m_tiles"] * p["head_n_tiles"] <= 148
+    assert p["head_m_tiles"] * p["head_n_tiles"] == 104
+    # twenty row tiles: one round of 256-wide items rather than two of 128-wide ones
+    p = plan_host(R=2880, P=2560, **DIMS_8B)
+    assert (p["head_k_splits"], p["head_tile_n"], p["head_m_tiles"] * p["head_n_tiles"]) == (1, 256, 80)
     # many row tiles: the widest tiles
     p = plan_host(R=8704, P=8192, **DIMS_8B)
     assert (p["head_k_splits"], p["head_tile_n"]) == (1, 256)
