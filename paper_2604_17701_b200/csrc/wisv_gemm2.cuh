@@ -2,7 +2,7 @@
 // (tcgen05 cta_group::2, M = 256: 128 weight rows per CTA) and the WINDOW ROWS on the N side, for batches of
 // more than 128 window rows.
 //
-// Why: one tcgen05.mma (K = 16) occupies the tensor pipe for max(57, N / 2) SM clocks per CTA whatever its M
+// Why: one tcgen05.mma (K = 16) occupies the tensor pipe for N / 2 SM clocks per CTA whatever its M once N >= 128
 // (measured: 128 x N and 64 x N cost the same).  With the window rows on the 128-row M side a batch pays for its
 // row count rounded up to 128 (256 for a pair): 144 rows cost as much as 256, 288 rows as much as 384, 576 as
 // much as 640.  On the N side the granularity is 16 rows: the batch is cut into ceil(R / 256) row blocks of equal
@@ -25,7 +25,7 @@
 //    shapes) and nothing is merged or written between tiles; the k-th pairs of all teams stream the same range at the
 //    same time and share its weight tiles through L2.  Chosen when the teams need no more tiles per pair than the
 //    round-robin below needs rounds;
-//  * many row blocks (bound by the tensor pipe): work items (vocabulary tile of 256 rows, row block) are dealt
+//  * many row blocks (bound by the tensor pipe at N = 256): work items (vocabulary tile of 256 rows, row block) are dealt
 //    out round-robin, row blocks of a group fastest, so the pairs that run at the same time share a weight tile
 //    through L2 and a group's activation rows stay resident there; one partial per (row, vocabulary tile, CTA).
 //
@@ -67,7 +67,7 @@ struct PairParams {
     // several row blocks (carry = 0): n_tiles vocabulary tiles of 256 rows; items run group by group (all vocabulary
     // tiles of a group of b_group row blocks before the next group)
     int32_t n_tiles, b_group;
-    int32_t part_stride; // partials per row: 2 per pair (carry) or 2 per vocabulary tile
+    int32_t part_stride; // partials per row: 2 per pair of a team (carry) or 2 per vocabulary tile
     int32_t* err;
     float4* lm_part;
     const int32_t* row_tok;
