@@ -322,7 +322,7 @@ Plan plan_head(const wisv_ctx* c, int P)
     } else if (p.m_tiles <= kSplitMaxRowTiles &&
                c->sm_count / (p.m_tiles * ((N + kSplitTileN - 1) / kSplitTileN)) >= 2) {
         // a few row tiles (B=64, K=8: four): still far fewer column tiles than SMs, and every CTA would walk all of
-        // K at the issue-bound pace of narrow tiles, so K is split here too while the work items fit the GPU once
+        // K at the pace of narrow tiles (set by barrier round trips, not by the MMAs), so K is split here too while the work items fit the GPU once
         best = kSplitTileN;
         const int nt = (N + best - 1) / best;
         int splits = c->sm_count / (p.m_tiles * nt);

@@ -225,7 +225,7 @@ __device__ __forceinline__ void gemm_rowreduce_body(const CUtensorMap& tmA, cons
     // end instead, so that "head kernel complete" implies "LM-head kernel complete" for the merge/scan
     // kernel that follows.  Decision-head CTAs that share a launch with the LM head follow the pack
     // kernel directly and wait here like the others.
-    // The producer thread of the early waiters waits a little later: weight tiles do not depend on the
+    // The producer warp of the early waiters waits a little later: weight tiles do not depend on the
     // pack kernel, so it first puts one ring-full of them in flight.
     // (The whole producer warp waits later, not just its issuing lane: lanes of one warp that sit in
     // griddepcontrol.wait hold back the lane that diverged from them.)

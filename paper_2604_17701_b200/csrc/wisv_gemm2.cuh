@@ -200,7 +200,7 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         griddep_launch_dependents();
     }
 
-    // producer thread only: stages issued so far (read again by the drain before the kernel ends)
+    // producer warp: stages issued so far, the same in all its lanes (read again by the drain before the kernel ends)
     long long prod_issued = 0;
 
     if (warp == 0) {
@@ -455,7 +455,7 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 }
                 __syncwarp();                                  // the buffer is rewritten by the next chunk
             }
-            // accumulator drained: hand it back to the MMA thread of the leader
+            // accumulator drained: hand it back to the MMA warp of the leader
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(as ? leader_acc_empty1 : leader_acc_empty0);
@@ -467,7 +467,7 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     }
 
     // After a time-out copies may still be heading for the shared memory of either CTA.  Their bytes are counted on
-    // the leader's full barriers, so the leader's producer thread waits (bounded) for the stages it issued last
+    // the leader's full barriers, so one lane of the leader's producer warp waits (bounded) for the stages it issued last
     // before it arrives at the closing cluster barrier, which in turn keeps the partner from retiring earlier.
     __syncthreads();
     if (leader && warp == 0 && lane == 0 && abort_flag[0] != 0) {
