@@ -82,6 +82,14 @@ __host__ __device__ inline uint32_t pair_fixed_bytes() {
     return 1024u + 1024u + 4u * kPairChunk * kPairPitch * 4u;
 }
 
+// 2^x for x <= 0 by the hardware approximation alone (relative error 2^-22; results below 2^-126 become 0):
+// exp2f() wraps the same instruction in a range fix-up that a sum of exponentials of non-positive numbers does not need.
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 __device__ __forceinline__ void pair_merge(float& mx, int& arg, float& sum, float omx, int oarg, float osum) {
     if (omx == -CUDART_INF_F && osum == 0.0f) return;
     if (omx > mx) {
@@ -413,17 +421,26 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 const int c0 = u * kPairChunk;
                 const int cols_here = min(kPairChunk, p.n_cols - c0);               // 16 or 32
                 if (row0 + c0 >= p.rows) continue;                                   // the block's padding columns
-                // ---- TMEM -> shared memory, transposed: tbuf[column][lane]
-                for (int hlf = 0; hlf * 16 < cols_here; ++hlf) {
-                    uint32_t v[16];
-                    tmem_ld16(taddr + static_cast<uint32_t>(c0 + hlf * 16), v);
+                // ---- TMEM -> shared memory, transposed: tbuf[column][lane] (both halves requested before the one wait)
+                {
+                    uint32_t va[16], vb[16];
+                    tmem_ld16(taddr + static_cast<uint32_t>(c0), va);
+                    if (cols_here > 16) tmem_ld16(taddr + static_cast<uint32_t>(c0 + 16), vb);
                     tmem_wait_ld();
 #pragma unroll
                     for (int t = 0; t < 16; ++t)
-                        tbuf[(hlf * 16 + t) * kPairPitch + lane] = lane_valid ? __uint_as_float(v[t]) : -CUDART_INF_F;
+                        tbuf[t * kPairPitch + lane] = lane_valid ? __uint_as_float(va[t]) : -CUDART_INF_F;
+                    if (cols_here > 16) {
+#pragma unroll
+                        for (int t = 0; t < 16; ++t)
+                            tbuf[(16 + t) * kPairPitch + lane] = lane_valid ? __uint_as_float(vb[t]) : -CUDART_INF_F;
+                    }
                 }
                 __syncwarp();
-                // ---- lane L: window row row0 + c0 + L against this warp's 32 vocabulary rows, in ascending order
+                // ---- lane L: window row row0 + c0 + L against this warp's 32 vocabulary rows.  Few warps share a
+                // scheduler here, so the chains are kept short: the maximum by a tree (the right operand of every
+                // merge holds the higher tokens, so strict '>' keeps the lowest token id of a tie), the sum in four
+                // independent accumulators.
                 const int r = row0 + c0 + lane;
                 if (lane < cols_here && r < p.rows) {
                     float x[32];
@@ -433,10 +450,26 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                         const float4 f = src[t];
                         x[4 * t] = f.x; x[4 * t + 1] = f.y; x[4 * t + 2] = f.z; x[4 * t + 3] = f.w;
                     }
-                    float cm = x[0];
-                    int ci = 0;
+                    float tm[16];
+                    int ti[16];
 #pragma unroll
-                    for (int t = 1; t < 32; ++t) { if (x[t] > cm) { cm = x[t]; ci = t; } }
+                    for (int t = 0; t < 16; ++t) {
+                        const bool g = x[2 * t + 1] > x[2 * t];
+                        tm[t] = g ? x[2 * t + 1] : x[2 * t];
+                        ti[t] = g ? 2 * t + 1 : 2 * t;
+                    }
+#pragma unroll
+                    for (int w2 = 8; w2 >= 1; w2 >>= 1) {
+#pragma unroll
+                        for (int t = 0; t < w2; ++t) {
+                            const bool g = tm[2 * t + 1] > tm[2 * t];
+                            const float m2 = g ? tm[2 * t + 1] : tm[2 * t];
+                            const int i2 = g ? ti[2 * t + 1] : ti[2 * t];
+                            tm[t] = m2; ti[t] = i2;
+                        }
+                    }
+                    const float cm = tm[0];
+                    const int ci = ti[0];
                     if (cm != -CUDART_INF_F) {
                         if (cm > mx[u]) {                     // strict: an earlier (lower) token keeps a tie
                             sum[u] *= exp2f((mx[u] - cm) * 1.4426950408889634f);
@@ -444,10 +477,10 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                             arg[u] = warp_v0 + ci;
                         }
                         const float base = mx[u] * 1.4426950408889634f;
-                        float acc = 0.0f;
+                        float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-                        for (int t = 0; t < 32; ++t) acc += exp2f(fmaf(x[t], 1.4426950408889634f, -base));
-                        sum[u] += acc;
+                        for (int t = 0; t < 32; ++t) acc[t & 3] += ex2_approx(fmaf(x[t], 1.4426950408889634f, -base));
+                        sum[u] += (acc[0] + acc[1]) + (acc[2] + acc[3]);
                         const int d = tokc[u] - warp_v0;
                         if (static_cast<unsigned>(d) < 32u && warp_v0 + d < p.n_total && q * 32 + d < half_h)
                             p.tok_logit[r] = tbuf[lane * kPairPitch + d];
