@@ -7,6 +7,7 @@ import torch
 
 import gen
 import oracle
+import paper_2604_17701_b200 as wisv
 from gen import cases
 from parity import compare, oracle_ref_argmax, run_oracle
 
@@ -756,8 +757,8 @@ def _check_properties(case, out):
     return A
 
 
-def _sampled_parity(name, n_sample, seed_pick=0):
-    cfg = gen.config(name)
+def _sampled_parity(name, n_sample, seed_pick=0, cfg=None):
+    cfg = cfg if cfg is not None else gen.config(name)
     case = cases.make_case(cfg, _lib_ref, weights=_shared_weights(cfg))
     d = cases.to_device(case, DEV)
     v = cases.make_verifier(d)
@@ -790,8 +791,8 @@ def test_8b_batch1_full_oracle():
 
 @pytest.mark.parametrize("name", ["8b_b16", "8b_b32"])
 def test_8b_two_and_three_row_tiles_sampled(name):
-    # 144 rows: CTA pairs with balanced vocabulary ranges + decision-head clusters; 288 rows: three row tiles on
-    # the single-CTA kernel with decision-head CTAs in the same launch
+    # 144 rows: CTA pairs with balanced vocabulary ranges + decision-head clusters; 288 rows: two teams of pairs, one
+    # per row block of 144, with decision-head clusters in the same launch
     case, out, A, stats = _sampled_parity(name, 12)
     assert stats["tainted_requests"] < stats["requests"]
 
@@ -832,6 +833,17 @@ def test_8b_batch512_sampled(name):
         expect = a * (1 - a ** k) / (1 - a)
         var = np.var(A)
         assert abs(A.mean() - expect) < 4 * np.sqrt(var / len(A)) + 0.05
+
+
+@pytest.mark.parametrize("B,K", [(100, 16), (1100, 16)], ids=["R1700_seven_row_blocks", "R18700_three_raster_groups"])
+def test_8b_row_counts_beyond_the_bench_configurations_sampled(B, K):
+    # 1700 rows: round-robin work items in one raster group, the decision head in its own launch with 128-column tiles;
+    # 18700 rows: 74 row blocks in three raster groups, twice the rows of the largest bench configuration
+    cfg = gen.config("8b_b512").with_(B=B, K=K, name="8b_b%d" % B, seed=4242 + B)
+    case, out, A, stats = _sampled_parity(cfg.name, 12, cfg=cfg)
+    v_plan = wisv.plan_host(H=cfg.H, V=cfg.V, H_d=cfg.H_d, d_c=cfg.d_c, d_J=cfg.d_J, R=case["R"], P=case["T"])
+    assert v_plan["lm_pair"] == 1 and v_plan["lm_carry"] == 0 and v_plan["lm_row_blocks"] == -(-case["R"] // 256)
+    assert stats["tainted_requests"] < stats["requests"]
 
 
 def test_random_shapes_under_every_launch_plan():
