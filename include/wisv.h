@@ -280,8 +280,10 @@ int wisv_set_tuning(wisv_ctx* ctx, const wisv_tuning* tuning);
  * opt-in shared memory per block, for the dimensions in cfg (H, V, H_d, d_c, d_J).  For tests and capacity
  * planning.  *_carry = 1: every CTA (or CTA pair) owns one contiguous range of the weight rows, units_base units
  * each (the first units_rem one more; a unit is 16 rows, 32 for pairs), cut into tiles_per_cta tiles of at most
- * tile_n rows.  lm_rounds / lm_rounds_alone: rounds of tiles the slowest CTA works through with and without
- * decision-head CTAs in the launch (0 when carried ranges are used).
+ * tile_n rows.  With lm_pair = 1, lm_carry = 1 and lm_row_blocks > 1 the pairs form one team per row block and the
+ * ranges are those of one team (lm_ctas / 2 / lm_row_blocks pairs each).  lm_rounds / lm_rounds_alone: rounds of tiles
+ * the slowest CTA (pair) works through with and without decision-head CTAs in the launch (the tiles of a pair's own
+ * range for teams; 0 when one row tile or block uses carried ranges).
  */
 typedef struct {
     int32_t kernels;                 /* kernels per round: 3 or 4 */
