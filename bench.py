@@ -47,6 +47,8 @@ NCU_TRAFFIC = {
     "8b_b1": {"bytes": 1068300000, "files": SINGLE_CTA_SOURCES, "kernel_hash": "7de628215d9b7ebf"},
     # CTA pairs (one row block of 144) + decision-head clusters: 1.0758 GB read + 4.6-5.4 MB written per launch
     "8b_b16": {"bytes": 1080800000, "files": CTA_PAIR_SOURCES, "kernel_hash": "901db3c2a09c4c22"},
+    # CTA pairs (two teams, row blocks of 144) + a decision-head cluster: 1.1039 GB read + 3.9-4.7 MB written per launch
+    "8b_b32": {"bytes": 1108200000, "files": CTA_PAIR_SOURCES, "kernel_hash": "901db3c2a09c4c22"},
     # CTA pairs (three teams, row blocks of 192) + decision-head clusters: 1.1218 GB read + 3.7-3.9 MB written per launch
     "8b_b64": {"bytes": 1125600000, "files": CTA_PAIR_SOURCES, "kernel_hash": "901db3c2a09c4c22"},
     # CTA pairs (34 row blocks of 256, two raster groups): 4.48-4.93 GB read + 139-142 MB written (the partials) per
